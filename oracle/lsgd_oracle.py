@@ -1,0 +1,340 @@
+"""CPU oracle for the Leader (Stochastic) Gradient Descent step.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, obviously-correct NumPy restatement of what one synchronous LSGD step computes,
+written from the paper (Section 2.2, Eq. (1), Algorithm 1; Section 3.1.1 and the supplement's
+"Definitions and Notation" for the eta-scaled form of the step and for communication periods;
+the supplement's matrix-completion section for the written-out update).  Only the tests, the
+smoke check and the CPU-baseline leg of the benchmark may import it; the product path never does,
+and this file imports nothing from the CUDA package.
+
+Arithmetic convention: worker parameters, gradients and losses are *stored* as float32.  Every
+stored value is produced by evaluating its defining formula in float64 from the float32 inputs
+and rounding once.  Reductions are float64.  There is no blocking, fusion or reordering beyond
+what the formulas state.
+
+Readings of the paper taken here (each is also exercised by a pin in tests/test_oracle_pins.py):
+  * pulls are scaled by the learning rate: x+ = x - eta (g + lambda (x - z))  (Section 3.1.1,
+    supplement "Definitions and Notation", and the written-out matrix-completion update
+    X+ = (1 - eta lambda) X + eta lambda Z - eta grad F(X); Eq. (1) prints them unscaled).
+  * gamma = gamma_G = 0 and tau_G = tau: leaders are re-elected and both pulls applied on steps
+    t = 0, tau, 2 tau, ... ("the leader is updated only at the beginning of each period");
+    all other steps are plain (S)GD steps.
+  * on a pull step the gradient, both leaders and both pulls are all taken at x_t (Eq. (1): every
+    right-hand term carries subscript t), i.e. a simultaneous (Jacobi) update of all workers.
+  * argmin ties go to the lowest worker index; the order on losses is
+    -inf < finite < +inf < NaN, and -0.0 == +0.0.
+
+Pins: see tests/test_oracle_pins.py.  Parity unpinned (self-consistent definitions only, no
+external fact fixes them): the placement of bf16 roundings in the MLP objective's "bf16emu" mode,
+and the 1/(2|B|) / 1/N constants of the observed-entry matrix-completion objective.
+"""
+from __future__ import annotations
+
+import math
+from typing import Callable, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+F32 = np.float32
+F64 = np.float64
+
+
+# ----------------------------------------------------------------------------------------------
+# Election (Section 2.2: local leader = argmin within the group, global leader = argmin over all)
+# ----------------------------------------------------------------------------------------------
+def _better(a: float, b: float) -> bool:
+    """True iff loss a strictly precedes loss b in the order -inf < finite < +inf < NaN."""
+    if math.isnan(a):
+        return False
+    if math.isnan(b):
+        return True
+    return a < b            # IEEE: -0.0 < +0.0 is False, so the two zeros tie
+
+
+def elect(loss: np.ndarray, group_of: Sequence[int], G: int) -> Tuple[np.ndarray, int]:
+    """Local leaders ll[j] = argmin_{i in group j} loss_i and global leader gl = argmin_i loss_i.
+
+    One left-to-right scan; a later worker replaces the incumbent only if strictly better, so
+    ties resolve to the lowest index."""
+    P = len(loss)
+    ll = [-1] * G
+    gl = -1
+    for i in range(P):
+        li = float(loss[i])
+        j = int(group_of[i])
+        if ll[j] < 0 or _better(li, float(loss[ll[j]])):
+            ll[j] = i
+        if gl < 0 or _better(li, float(loss[gl])):
+            gl = i
+    return np.asarray(ll, dtype=np.int32), int(gl)
+
+
+# ----------------------------------------------------------------------------------------------
+# The update (Eq. (1), eta-scaled pulls; plain SGD form between communications)
+# ----------------------------------------------------------------------------------------------
+def update(x: np.ndarray, g: np.ndarray, group_of: Sequence[int], ll: Sequence[int], gl: int,
+           eta: float, lambda_l: float, lambda_g: float, pull: bool) -> None:
+    """In-place on x (float32 [P, ld]).
+
+    pull:  x_i <- x_i - eta g_i - eta lambda_l (x_i - x_{ll[group(i)]}) - eta lambda_g (x_i - x_gl)
+    else:  x_i <- x_i - eta g_i
+    with every right-hand side taken from x at time t (leader rows are snapshotted first)."""
+    eta = float(F32(eta))
+    lambda_l = float(F32(lambda_l))
+    lambda_g = float(F32(lambda_g))
+    P = x.shape[0]
+    if pull:
+        snap_l = {int(r): x[int(r)].astype(F64) for r in set(int(v) for v in ll)}
+        snap_g = x[int(gl)].astype(F64)
+    for i in range(P):
+        xi = x[i].astype(F64)
+        new = xi - eta * g[i].astype(F64)
+        if pull:
+            zl = snap_l[int(ll[int(group_of[i])])]
+            new = new - eta * lambda_l * (xi - zl) - eta * lambda_g * (xi - snap_g)
+        x[i] = new.astype(F32)
+
+
+# ----------------------------------------------------------------------------------------------
+# Objectives
+# ----------------------------------------------------------------------------------------------
+class Objective:
+    """grad(x, t) -> float32 [P, ld] stochastic gradients at step t; loss(x, n) -> float32 [P]
+    election losses for the n-th election."""
+
+    def grad(self, x: np.ndarray, t: int) -> np.ndarray:
+        raise NotImplementedError
+
+    def loss(self, x: np.ndarray, n: int) -> np.ndarray:
+        raise NotImplementedError
+
+
+class External(Objective):
+    """Gradients and election losses are supplied: one fixed g, a ring of loss vectors."""
+
+    def __init__(self, g: np.ndarray, loss_ring: np.ndarray):
+        self.g, self.loss_ring = g, loss_ring
+
+    def grad(self, x, t):
+        return self.g
+
+    def loss(self, x, n):
+        return self.loss_ring[n % len(self.loss_ring)]
+
+
+class Quadratic(Objective):
+    """f(x) = 1/2 sum_k a_k (x_k - b_k)^2  (the positive-definite quadratic model of Section 3.3
+    with a diagonal Hessian);  g = a (x - b) + sigma eps;  election loss = f(x_i) exactly."""
+
+    def __init__(self, a: np.ndarray, b: np.ndarray, sigma: float, noise: Optional[np.ndarray]):
+        self.a, self.b = a.astype(F64), b.astype(F64)
+        self.sigma = float(F32(sigma))
+        self.noise = noise                              # float32 [ring, P, ld] or None (batch LGD)
+
+    def grad(self, x, t):
+        g = np.empty_like(x)
+        for i in range(x.shape[0]):
+            gi = self.a * (x[i].astype(F64) - self.b)
+            if self.noise is not None:
+                gi = gi + self.sigma * self.noise[t % len(self.noise)][i].astype(F64)
+            g[i] = gi.astype(F32)
+        return g
+
+    def loss(self, x, n):
+        out = np.empty(x.shape[0], dtype=F32)
+        for i in range(x.shape[0]):
+            r = x[i].astype(F64) - self.b
+            out[i] = F32(0.5 * np.sum(self.a * r * r))
+        return out
+
+
+class MatComp(Objective):
+    """Factorised completion on observed entries.  Parameter row = [X (n_rows x rank) | Y (n_cols x
+    rank)], both row-major.  Minibatch loss (1/(2|B|)) sum_{(r,c,v) in B} (<X_r, Y_c> - v)^2, so
+    dX_r += e Y_c / |B| and dY_c += e X_r / |B| with e = <X_r, Y_c> - v, accumulated over the
+    batch in list order (duplicates add).  Election loss = mean squared residual over a fixed
+    held-out list."""
+
+    def __init__(self, n_rows, n_cols, rank, obs_r, obs_c, obs_v, batch_pos, heldout_pos):
+        self.n_rows, self.n_cols, self.rank = n_rows, n_cols, rank
+        self.obs_r, self.obs_c, self.obs_v = obs_r, obs_c, obs_v
+        self.batch_pos, self.heldout_pos = batch_pos, heldout_pos
+
+    def _factors(self, xi):
+        nx = self.n_rows * self.rank
+        X = xi[:nx].astype(F64).reshape(self.n_rows, self.rank)
+        Y = xi[nx:nx + self.n_cols * self.rank].astype(F64).reshape(self.n_cols, self.rank)
+        return X, Y
+
+    def grad(self, x, t):
+        g = np.zeros_like(x)
+        nx = self.n_rows * self.rank
+        for i in range(x.shape[0]):
+            pos = self.batch_pos[t % len(self.batch_pos)][i]
+            r, c, v = self.obs_r[pos], self.obs_c[pos], self.obs_v[pos].astype(F64)
+            X, Y = self._factors(x[i])
+            e = np.sum(X[r] * Y[c], axis=1) - v
+            gX = np.zeros_like(X)
+            gY = np.zeros_like(Y)
+            np.add.at(gX, r, e[:, None] * Y[c] / len(pos))
+            np.add.at(gY, c, e[:, None] * X[r] / len(pos))
+            g[i, :nx] = gX.ravel().astype(F32)
+            g[i, nx:nx + gY.size] = gY.ravel().astype(F32)
+        return g
+
+    def loss(self, x, n):
+        pos = self.heldout_pos
+        r, c, v = self.obs_r[pos], self.obs_c[pos], self.obs_v[pos].astype(F64)
+        out = np.empty(x.shape[0], dtype=F32)
+        for i in range(x.shape[0]):
+            X, Y = self._factors(x[i])
+            e = np.sum(X[r] * Y[c], axis=1) - v
+            out[i] = F32(np.sum(e * e) / len(pos))
+        return out
+
+
+def bf16_round(a: np.ndarray) -> np.ndarray:
+    """Round float32 to the nearest bfloat16 (ties to even), returned as float32 (finite inputs)."""
+    u = np.ascontiguousarray(a, dtype=F32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(F32).reshape(np.shape(a))
+
+
+class Mlp(Objective):
+    """Population of ReLU MLP classifiers with mean softmax cross-entropy.
+
+    Parameter row = [W1 | b1 | W2 | b2 | ...], W_l stored [out, in] row-major at the float offsets
+    given by ``segs`` (list of dicts with keys w, b, n_in, n_out).  Layer: z = h_prev W^T + b,
+    h = relu(z) (no relu on the last layer).
+    mode "fp32": everything float64-evaluated from float32 storage.
+    mode "bf16emu": every matrix-product operand -- weights, the input batch, the stored hidden
+    activations, and the back-propagated dz / dh -- is first rounded to bfloat16; products are
+    accumulated in float64; bias gradients are column sums of the *rounded* dz / dh; the relu mask
+    is taken from the stored (rounded) activation."""
+
+    def __init__(self, segs, data_x, data_y, batch_idx, held_x, held_y, mode="bf16emu"):
+        self.segs = segs
+        self.data_x, self.data_y, self.batch_idx = data_x, data_y, batch_idx
+        self.held_x, self.held_y = held_x, held_y
+        self.rd = bf16_round if mode == "bf16emu" else (lambda a: np.asarray(a, dtype=F32))
+        self.last_train_loss = None
+
+    def _weights(self, xi):
+        Ws, bs = [], []
+        for s in self.segs:
+            W = xi[s["w"]:s["w"] + s["n_in"] * s["n_out"]].reshape(s["n_out"], s["n_in"])
+            Ws.append(self.rd(W).astype(F64))
+            bs.append(xi[s["b"]:s["b"] + s["n_out"]].astype(F64))
+        return Ws, bs
+
+    def _forward(self, xi, inp):
+        Ws, bs = self._weights(xi)
+        hs = [self.rd(inp).astype(F64)]
+        L = len(Ws)
+        for l in range(L):
+            z = hs[-1] @ Ws[l].T + bs[l]
+            if l < L - 1:
+                hs.append(self.rd(np.maximum(z, 0.0).astype(F32)).astype(F64))
+        return Ws, hs, z
+
+    @staticmethod
+    def _softmax_ce(z, y):
+        zs = z - z.max(axis=1, keepdims=True)
+        lse = np.log(np.exp(zs).sum(axis=1, keepdims=True))
+        logp = zs - lse
+        n = z.shape[0]
+        ce = -logp[np.arange(n), y].sum() / n
+        return ce, np.exp(logp)
+
+    def grad(self, x, t):
+        g = np.zeros_like(x)
+        losses = np.empty(x.shape[0], dtype=F32)
+        for i in range(x.shape[0]):
+            idx = self.batch_idx[t % len(self.batch_idx)][i]
+            y = self.data_y[idx]
+            Ws, hs, z = self._forward(x[i], self.data_x[idx])
+            ce, p = self._softmax_ce(z, y)
+            losses[i] = F32(ce)
+            n = len(idx)
+            dz = p.copy()
+            dz[np.arange(n), y] -= 1.0
+            dz /= n
+            delta = self.rd(dz.astype(F32)).astype(F64)
+            for l in range(len(Ws) - 1, -1, -1):
+                s = self.segs[l]
+                dW = delta.T @ hs[l]                               # [out, in]
+                g[i, s["w"]:s["w"] + dW.size] = dW.ravel().astype(F32)
+                g[i, s["b"]:s["b"] + s["n_out"]] = delta.sum(axis=0).astype(F32)
+                if l > 0:
+                    dh = (delta @ Ws[l]) * (hs[l] > 0.0)
+                    delta = self.rd(dh.astype(F32)).astype(F64)
+        self.last_train_loss = losses
+        return g
+
+    def loss(self, x, n):
+        out = np.empty(x.shape[0], dtype=F32)
+        for i in range(x.shape[0]):
+            _, _, z = self._forward(x[i], self.held_x)
+            out[i] = F32(self._softmax_ce(z, self.held_y)[0])
+        return out
+
+
+class FromCallables(Objective):
+    """Any differentiable f: grad_fn(x_i) -> gradient, loss_fn(x_i) -> scalar (batch LGD)."""
+
+    def __init__(self, grad_fn: Callable, loss_fn: Callable):
+        self.grad_fn, self.loss_fn = grad_fn, loss_fn
+
+    def grad(self, x, t):
+        return np.stack([np.asarray(self.grad_fn(x[i].astype(F64)), dtype=F64).astype(F32)
+                         for i in range(x.shape[0])])
+
+    def loss(self, x, n):
+        return np.asarray([F32(self.loss_fn(x[i].astype(F64))) for i in range(x.shape[0])], dtype=F32)
+
+
+# ----------------------------------------------------------------------------------------------
+# The loop
+# ----------------------------------------------------------------------------------------------
+class LsgdOracle:
+    """State (x, t, ll, gl) and one synchronous step:
+
+      1. g_i = stochastic gradient at x_i^t                                  (Eq. (1), Algorithm 1)
+      2. if t mod tau == 0: election losses at x^t, then local / global argmin   (Section 2.2)
+      3. fused update (pull form iff t mod tau == 0)                          (Eq. (1))
+      4. t <- t + 1
+    """
+
+    def __init__(self, x0: np.ndarray, objective: Objective, group_of: Sequence[int], G: int,
+                 eta: float, lambda_l: float, lambda_g: float, tau: int):
+        assert tau >= 1
+        self.x = np.array(x0, dtype=F32, copy=True)
+        self.obj = objective
+        self.group_of = np.asarray(group_of, dtype=np.int32)
+        self.G = int(G)
+        self.eta, self.lambda_l, self.lambda_g, self.tau = eta, lambda_l, lambda_g, int(tau)
+        self.t = 0
+        self.n_elections = 0
+        self.ll: Optional[np.ndarray] = None
+        self.gl: Optional[int] = None
+        self.loss: Optional[np.ndarray] = None
+        self.history: List[dict] = []           # one record per election
+
+    def step(self, forced_loss: Optional[np.ndarray] = None) -> None:
+        g = self.obj.grad(self.x, self.t)
+        pull = (self.t % self.tau == 0)
+        if pull:
+            self.loss = np.asarray(self.obj.loss(self.x, self.n_elections) if forced_loss is None
+                                   else forced_loss, dtype=F32)
+            self.ll, self.gl = elect(self.loss, self.group_of, self.G)
+            self.history.append({"t": self.t, "loss": self.loss.copy(), "ll": self.ll.copy(),
+                                 "gl": self.gl})
+            self.n_elections += 1
+        update(self.x, g, self.group_of, self.ll if pull else (), self.gl if pull else -1,
+               self.eta, self.lambda_l, self.lambda_g, pull)
+        self.t += 1
+
+    def run(self, steps: int) -> np.ndarray:
+        for _ in range(steps):
+            self.step()
+        return self.x
