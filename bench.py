@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the LSGD step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4|c1] [--tau T]
+    python bench.py --impl reference ...        # the CPU oracle, timed on the host cores
+
+Default workload: the large fused-update stress (P = 16 workers in G = 4 groups, d = 2^26 fp32
+parameters per worker, supplied gradients and election losses, tau = 1).  One step = election +
+fused update over the whole population.  Prints ONE JSON line (rank 0).
+
+With N > 1 (torchrun, one process per GPU) every rank runs an independent replica of the workload:
+the method keeps the whole population on one device and has no exchange step, so there is no
+collective on the data path -- only the barrier and the max-over-ranks of the timing.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "lsgd_step_worker_params_per_s"
+UNIT = "worker-params/s"
+
+
+# ------------------------------------------------------------------------------------ helpers ----
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.lines = []
+        self.idx = device_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        inside = [l for (ts, l) in self.lines if t0 - 0.05 <= ts <= t1 + 0.15] or [l for (_, l) in self.lines]
+        for l in inside:
+            f = [c.strip() for c in l.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except Exception:
+                continue
+            for name, v in zip(self.NAMES, f[3:7]):
+                if v == "Active":
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def aggregate(per_rank_units: float, elapsed_ms_max: float, world: int) -> float:
+    """Whole-job throughput: the units all ranks processed over the slowest rank's time."""
+    return per_rank_units * world / (elapsed_ms_max * 1e-3)
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# --------------------------------------------------------------------------------- workloads ----
+def workload_spec(args):
+    if args.workload == "c4":
+        return dict(kind="external", P=16, G=4, d=1 << 26, eta=0.01, lambda_l=0.1, lambda_g=0.05,
+                    tau=args.tau or 1, name="C4 fused-update stress: P=16 G=4 d=2^26 fp32, supplied g and losses")
+    if args.workload == "c1":
+        return dict(kind="quadratic", P=64, G=8, d=1 << 20, eta=0.05, lambda_l=0.1, lambda_g=0.05,
+                    tau=args.tau or 4, name="C1 multi-leader quadratic: P=64 G=8 d=2^20 fp32, noise sigma=0.01")
+    raise SystemExit("unknown workload")
+
+
+def bytes_per_worker_param(spec, fused=True):
+    # update: read x + read g (or noise) + write x; quadratic adds a, b once per column
+    return 12.0 + (8.0 / spec["P"] if spec["kind"] == "quadratic" else 0.0)
+
+
+# ------------------------------------------------------------------------------ CPU oracle leg ----
+def oracle_sample_run(spec, steps, warmup, sample_cols):
+    """Times the oracle, as it stands, on a column sample of the workload (same P, G, tau)."""
+    from oracle import lsgd_oracle as orc
+    from paper_1905_10395_b200 import inputs
+    if spec["kind"] == "external":
+        w = inputs.make_external(spec["P"], spec["G"], sample_cols, eta=spec["eta"], lambda_l=spec["lambda_l"],
+                                 lambda_g=spec["lambda_g"], tau=spec["tau"], steps=steps, config_id=4)
+        obj = orc.External(w.arrays["g"], w.arrays["loss_ring"])
+    else:
+        w = inputs.make_quadratic(spec["P"], spec["G"], sample_cols, eta=spec["eta"], lambda_l=spec["lambda_l"],
+                                  lambda_g=spec["lambda_g"], tau=spec["tau"], steps=steps, sigma=0.01,
+                                  noise_ring=2, config_id=1)
+        obj = orc.Quadratic(w.arrays["a"], w.arrays["b"], 0.01, w.arrays["noise"])
+    o = orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
+    for _ in range(warmup):
+        o.step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        o.step()
+    dt = time.perf_counter() - t0
+    return spec["P"] * sample_cols * steps / dt, dt
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    spec = workload_spec(args)
+    steps, warmup = args.steps, args.warmup
+    sample = args.sample_cols or (1 << 22)
+    value, dt = oracle_sample_run(spec, steps, warmup, sample)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": spec["name"], "tau": spec["tau"],
+                   "sample": f"each step covers {sample} of the {spec['d']} columns of every worker"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{steps} steps x {spec['P']} workers x {sample} columns"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------- GPU arm ----
+def run_ours(args):
+    import torch
+    from paper_1905_10395_b200 import api, inputs
+    from paper_1905_10395_b200.runner import Population
+
+    rank, world, local = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local if world > 1 else 0)
+    torch.cuda.set_device(dev)
+    api.lib()                                       # fail loudly if the CUDA library is missing
+    spec = workload_spec(args)
+    P, G, d = spec["P"], spec["G"], spec["d"]
+    steps, warmup = args.steps, max(args.warmup, 3)
+
+    # ---- inputs: generated on the host from the seed, into pinned memory (also used by the e2e leg)
+    if spec["kind"] == "external":
+        hx = torch.empty((P, d), dtype=torch.float32, pin_memory=True)
+        hg = torch.empty((P, d), dtype=torch.float32, pin_memory=True)
+        w = inputs.make_external(P, G, d, eta=spec["eta"], lambda_l=spec["lambda_l"], lambda_g=spec["lambda_g"],
+                                 tau=spec["tau"], steps=steps, config_id=4, x_out=hx.numpy(), g_out=hg.numpy())
+        x = hx.to(dev, non_blocking=True)
+        g = hg.to(dev, non_blocking=True)
+        pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith)
+        launches_per_step = lambda t: 2 if t % spec["tau"] == 0 else 1
+    else:
+        w = inputs.config(1, tau=spec["tau"])
+        pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith)
+        hx = hg = None
+        launches_per_step = lambda t: 3 if t % spec["tau"] == 0 else 1
+    torch.cuda.synchronize(dev)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    # ---- device-resident timing
+    for _ in range(warmup):
+        pop.step()
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    k_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    barrier()
+    torch.cuda.synchronize(dev)
+    wall0 = time.time()
+    ev0.record()
+    n_launch = 0
+    pull_flags = []
+    for s in range(steps):
+        t = pop.t
+        batch = pop.batches[t % len(pop.batches)] if pop.batches else None
+        pop.lsgd.grad(batch)
+        if t % spec["tau"] == 0:
+            pop.lsgd.elect(pop.loss_ring[pop.n_elections % pop.loss_ring.shape[0]] if pop.loss_ring is not None else None)
+            pop.n_elections += 1
+        k_ev[s][0].record()
+        pop.lsgd.step()
+        k_ev[s][1].record()
+        pop.t += 1
+        n_launch += launches_per_step(t)
+        pull_flags.append(t % spec["tau"] == 0)
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    wall1 = time.time()
+    barrier()
+    clocks = sampler.stop(wall0, wall1)
+    elapsed_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+    value = aggregate(P * d * steps, elapsed_ms, world)
+    k_ms = [a.elapsed_time(b) for a, b in k_ev]
+    upd_ms = float(np.mean(k_ms))
+    alg_bytes = bytes_per_worker_param(spec) * P * d
+    peak, peak_src = read_peaks()
+    achieved = alg_bytes / (upd_ms * 1e-3) / 1e9
+    if pop.lsgd.check_device() != 0:
+        raise SystemExit("device status word set during the bench")
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": elapsed_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": {0: "f64", 1: "f64", 2: "f32"}[args.arith], "data": "synthetic",
+        "config": {"workload": spec["name"], "tau": spec["tau"], "storage": "f32",
+                   "arithmetic": ["fp64 unfused", "fp64 fma", "fp32 fma"][args.arith],
+                   "l2": "inputs (>= 0.5 GiB per step) exceed the 126 MB L2; no flush between steps",
+                   "multi_gpu": "replicas only"},
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
+                     "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
+                     "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags))},
+        "gpu_launches": n_launch,
+    }
+
+    # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs, D2H of its result
+    if rank == 0 and world == 1 and not args.no_e2e and hx is not None:
+        e_steps = args.e2e_steps
+        hout = hx                                   # result is read back into the pinned x buffer
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        loss_host = torch.from_numpy(w.arrays["loss_ring"]).pin_memory()
+        dloss = torch.empty(P, dtype=torch.float32, device=dev)
+        for it in range(e_steps + 1):
+            if it == 1:
+                e0.record()
+            pop.x.copy_(hx, non_blocking=True)
+            pop.g.copy_(hg, non_blocking=True)
+            dloss.copy_(loss_host[it % loss_host.shape[0]], non_blocking=True)
+            pop.lsgd.grad(None)
+            pop.lsgd.elect(dloss)
+            pop.lsgd.step()
+            hout.copy_(pop.x, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        e_ms = e0.elapsed_time(e1) / e_steps
+        line["e2e"] = {"value": P * d / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(2 * P * d * 4 + P * 4),
+                       "d2h_bytes_per_step": int(P * d * 4), "ms_per_step": e_ms, "steps": e_steps,
+                       "note": "every step elects (a pull step) so tau does not apply"}
+    else:
+        line["e2e"] = None
+    pop.close()
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        sample = args.sample_cols or (1 << 22)
+        v, dt = oracle_sample_run(spec, 3, 1, sample)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"3 steps x {P} workers x {sample} of {d} columns, {dt:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4", choices=["c4", "c1"])
+    ap.add_argument("--tau", type=int, default=0)
+    ap.add_argument("--arith", type=int, default=0, choices=[0, 1, 2])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--sample-cols", type=int, default=0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,186 @@
+/*
+ * lsgd.h -- C ABI of the Leader SGD step for a population of P workers in G groups that all live
+ * on ONE CUDA device (sm_100a).
+ *
+ * Method: "Leader Stochastic Gradient Descent for Distributed Training of Deep Learning Models:
+ * Extension" (Teng, Gao, Chalus, Choromanska, Goldfarb, Weller).  One synchronous step is
+ *   1. every worker's stochastic gradient g_i at x_i                   (Section 2.2, Eq. (1))
+ *   2. every worker's election loss        (Section 2.2; estimated losses: Section 3.1.3)
+ *   3. local leaders (argmin inside each group) and the global leader (argmin over all workers)
+ *                                              (Section 2.2, definitions below the multi-leader objective)
+ *   4. the fused update                                                 (Eq. (1), eta-scaled as in
+ *      x_i <- x_i - eta g_i - eta lambda_l (x_i - x_ll(i)) - eta lambda_g (x_i - x_gl)   Section 3.1.1)
+ *      on steps t = 0, tau, 2 tau, ... and the plain step x_i <- x_i - eta g_i in between
+ *      (communication period: Section 3.1.2).
+ * The paper's leader broadcast is an on-device read: leaders are kept as row indices.
+ *
+ * General conventions
+ *   - Every pointer is documented as HOST or DEVICE.  DEVICE buffers are owned by the caller, must
+ *     stay alive and unmodified by others until the stream has drained, and are never freed here.
+ *   - Worker parameters are a row-major float matrix x[P][ld]; row i is worker i; ld >= d is the
+ *     row stride in floats and a multiple of 32; columns d..ld-1 are padding that callers keep 0.
+ *   - All work is enqueued on the stream given at creation; grad / elect / step never synchronise.
+ *   - Functions return an lsgd_status; nothing throws, aborts or prints.  Argument errors are
+ *     detected on the host before anything is launched.
+ *   - A handle is not thread-safe; distinct handles are independent.
+ */
+#ifndef LSGD_H_
+#define LSGD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define LSGD_API __attribute__((visibility("default")))
+#else
+#define LSGD_API
+#endif
+
+typedef struct lsgd_ctx* lsgd_handle;
+
+typedef enum {
+  LSGD_OK = 0,
+  LSGD_ERR_INVALID_ARG = 1,  /* NULL where not allowed, P < 1, tau < 1, non-finite eta, ld < d ...  */
+  LSGD_ERR_BAD_GROUPS = 2,   /* G < 1, G > P, group id out of range, or an empty group               */
+  LSGD_ERR_ALIGNMENT = 3,    /* a DEVICE pointer is not 16-byte aligned, or ld is not a multiple of 32 */
+  LSGD_ERR_STATE = 4,        /* call order: pull step before any election, step without a gradient   */
+  LSGD_ERR_CUDA = 5,         /* a CUDA runtime call or launch failed (no usable device included)     */
+  LSGD_ERR_UNSUPPORTED = 6,  /* combination not implemented (documented at the argument)             */
+  LSGD_ERR_DEVICE_FLAG = 7   /* a kernel recorded a bounded-wait / bounds failure in its status word */
+} lsgd_status;
+
+typedef enum {
+  LSGD_OBJ_EXTERNAL = 0,     /* caller writes g and supplies the loss vector                         */
+  LSGD_OBJ_QUADRATIC = 1,    /* f(x) = 1/2 sum_k a_k (x_k - b_k)^2                                    */
+  LSGD_OBJ_MATCOMP = 2,      /* factorised matrix completion on observed entries                     */
+  LSGD_OBJ_MLP = 3           /* population of ReLU MLP classifiers, bf16 GEMMs, fp32 accumulate      */
+} lsgd_objective;
+
+/* How the per-element formulas (update, quadratic gradient) are evaluated.  Storage is always fp32. */
+typedef enum {
+  LSGD_ARITH_FP64 = 0,       /* default: fp64, one IEEE operation per printed operation, one final
+                                rounding to fp32 (what a double-precision restatement of Eq. (1) gives) */
+  LSGD_ARITH_FP64_FMA = 1,   /* fp64 with fused multiply-adds                                        */
+  LSGD_ARITH_FP32 = 2        /* fp32 fused multiply-adds                                             */
+} lsgd_arithmetic;
+
+/* Diagonal quadratic (the positive-definite quadratic model of Section 3.3 with diagonal Hessian):
+ * g_i = a (x_i - b) + sigma * noise_i,  election loss f(x_i).                                      */
+typedef struct {
+  const float* a;            /* DEVICE float[ld], a_k > 0                                            */
+  const float* b;            /* DEVICE float[ld]                                                     */
+  float sigma;               /* weight of the per-step noise array given to lsgd_grad                */
+} lsgd_quadratic_desc;
+
+/* Matrix completion with factors: row i of x is [X (n_rows x rank) | Y (n_cols x rank)], row-major.
+ * Minibatch loss (1/(2B)) sum (<X_r, Y_c> - v)^2 over B observed entries per worker per step, given
+ * to lsgd_grad as positions into the observed list; election loss = mean squared residual over the
+ * fixed held-out positions.  (Low-rank completion is the paper's motivating example, Section 2.1.) */
+typedef struct {
+  int32_t n_rows, n_cols, rank;
+  int32_t n_obs;
+  const int32_t* obs_r;      /* DEVICE int32[n_obs] row of each observed entry                       */
+  const int32_t* obs_c;      /* DEVICE int32[n_obs] column                                           */
+  const float* obs_v;        /* DEVICE float[n_obs] value                                            */
+  int32_t batch;             /* B, entries per worker per step                                       */
+  int32_t n_heldout;
+  const int32_t* heldout_pos;/* DEVICE int32[n_heldout] positions into the observed list             */
+} lsgd_matcomp_desc;
+
+/* MLP population: row i of x is [W1 | b1 | W2 | b2 | W3 | b3]; W_l is [n_out][n_in] row-major
+ * (input index contiguous); each segment starts at a multiple of 32 floats (see
+ * lsgd_mlp_param_offsets).  Loss: mean softmax cross-entropy.  Matrix products take bf16 operands
+ * (weights, inputs, stored activations and back-propagated deltas are rounded to bf16, ties to
+ * even) and accumulate in fp32.                                                                   */
+#define LSGD_MLP_MAX_LAYERS 3
+typedef struct {
+  int32_t dims[LSGD_MLP_MAX_LAYERS + 1]; /* n_in, hidden, hidden, n_classes                          */
+  int32_t batch;             /* training samples per worker per step (multiple of 128)              */
+  int32_t pool;              /* number of rows of pool_x                                             */
+  const float* pool_x;       /* DEVICE float[pool][dims[0]] training samples                         */
+  const int32_t* pool_y;     /* DEVICE int32[pool] labels                                            */
+  int32_t n_heldout;         /* election batch (multiple of 128)                                     */
+  const float* held_x;       /* DEVICE float[n_heldout][dims[0]]                                     */
+  const int32_t* held_y;     /* DEVICE int32[n_heldout]                                              */
+  void* scratch;             /* DEVICE, lsgd_mlp_scratch_bytes() bytes, 1024-byte aligned            */
+  uint64_t scratch_bytes;
+} lsgd_mlp_desc;
+
+typedef struct {
+  uint32_t struct_size;      /* = sizeof(lsgd_config)                                                */
+  int32_t P;                 /* workers (the paper's n * l)                                          */
+  int32_t G;                 /* groups  (the paper's n)                                              */
+  const int32_t* group_of;   /* HOST int32[P], values in [0, G), every group non-empty; copied       */
+  int64_t d;                 /* parameters per worker                                                */
+  int64_t ld;                /* row stride in floats, ld >= d, ld % 32 == 0                          */
+  float eta;                 /* learning rate eta                                                    */
+  float lambda_l;            /* pull strength towards the local leader  (the paper's lambda)         */
+  float lambda_g;            /* pull strength towards the global leader (the paper's lambda_G)       */
+  int32_t tau;               /* communication period tau >= 1                                        */
+  int32_t objective;         /* lsgd_objective                                                       */
+  const void* objective_desc;/* HOST pointer to the matching *_desc (copied), NULL for EXTERNAL      */
+  float* x;                  /* DEVICE float[P*ld], 16-byte aligned, updated in place                */
+  float* g;                  /* DEVICE float[P*ld] gradients.  May be NULL only for QUADRATIC, whose
+                                gradient is then evaluated inside the update kernel (no g traffic)  */
+  void* stream;              /* cudaStream_t; NULL = the legacy default stream                       */
+  int32_t arithmetic;        /* lsgd_arithmetic                                                      */
+} lsgd_config;
+
+/* Validates the configuration on the host, copies the group map, builds the group tables and
+ * allocates O(P + G) words of device state plus reduction scratch for the objective's election
+ * loss.  Returns LSGD_ERR_CUDA if no CUDA device is usable.  *out is NULL on failure.            */
+LSGD_API lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out);
+
+/* Step 1: stochastic gradients of all workers at the current x (Eq. (1): g_t^{j,i}).
+ * batch is objective-specific, a DEVICE pointer valid until the stream has drained:
+ *   EXTERNAL  ignored (the caller has written g);
+ *   QUADRATIC const float noise[P*ld] (standard normal draws) or NULL for the exact gradient;
+ *             with cfg.g == NULL nothing is launched: the gradient is evaluated in lsgd_step;
+ *   MATCOMP   const int32_t pos[P*batch], positions into the observed list (duplicates add up);
+ *   MLP       const int32_t idx[P*batch], rows of pool_x.                                          */
+LSGD_API lsgd_status lsgd_grad(lsgd_handle h, const void* batch);
+
+/* Steps 2+3: election.  loss is a DEVICE float[P] of election losses, or NULL to evaluate the
+ * objective's own election loss at the current x first (not available for EXTERNAL).  Writes the
+ * local leaders and the global leader to device state.  Order on losses: -inf < finite < +inf <
+ * NaN, -0 == +0; ties go to the lowest worker index.  Callers normally call it on the steps with
+ * t % tau == 0 only; electing more often is legal (the analysis allows any guiding point).        */
+LSGD_API lsgd_status lsgd_elect(lsgd_handle h, const float* loss);
+
+/* Step 4: the fused update, pull form iff t % tau == 0 (t = number of lsgd_step calls so far),
+ * then t <- t + 1.  On a pull step every right-hand side is x at time t, although x is updated in
+ * place.  LSGD_ERR_STATE if a pull step comes before any election, or if no gradient was
+ * provided since the previous step (EXTERNAL is exempt: g is the caller's).                      */
+LSGD_API lsgd_status lsgd_step(lsgd_handle h);
+
+/* Frees the device state.  The caller's buffers are untouched.  NULL is accepted.                */
+LSGD_API lsgd_status lsgd_destroy(lsgd_handle h);
+
+/* Accessors.  They synchronise the stream and are not part of the step.                          */
+LSGD_API lsgd_status lsgd_get_leaders(lsgd_handle h, int32_t* local_leaders /* HOST int32[G] */,
+                             int32_t* global_leader /* HOST int32[1] */);
+LSGD_API lsgd_status lsgd_get_loss(lsgd_handle h, float* loss /* HOST float[P]: losses of the last election */);
+LSGD_API lsgd_status lsgd_get_step(lsgd_handle h, int64_t* t);
+/* Times each worker has been global / local leader so far (the leader statistics of Section 4.2). */
+LSGD_API lsgd_status lsgd_get_leader_counts(lsgd_handle h, int32_t* global_counts /* HOST int32[P] */,
+                                   int32_t* local_counts /* HOST int32[P] */);
+/* Reads and clears the device status word; LSGD_ERR_DEVICE_FLAG if any kernel has set it.        */
+LSGD_API lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out /* HOST, may be NULL */);
+/* Replaces eta (learning-rate schedules are the caller's, Section 4).                            */
+LSGD_API lsgd_status lsgd_set_eta(lsgd_handle h, float eta);
+
+LSGD_API const char* lsgd_status_string(lsgd_status s);
+
+/* MLP helpers (host only).  Offsets in floats of W_l and b_l inside a parameter row, and the row
+ * length d.  n_layers = 3.                                                                        */
+LSGD_API lsgd_status lsgd_mlp_param_offsets(const int32_t* dims /* HOST int32[4] */, int64_t* w_off /* [3] */,
+                                   int64_t* b_off /* [3] */, int64_t* d_out);
+LSGD_API uint64_t lsgd_mlp_scratch_bytes(const int32_t* dims, int32_t P, int32_t batch, int32_t n_heldout);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LSGD_H_ */

@@ -1,0 +1,88 @@
+// Leader election (Section 2.2): local leader = argmin of the election loss inside each group,
+// global leader = argmin over all workers = best of the local leaders.
+//
+// Each loss is packed with its worker index into one 64-bit key, (orderable(loss) << 32) | index,
+// so that an unsigned minimum is the argmin with ties resolved to the lowest index.  orderable()
+// maps floats monotonically to uint32 with -0 and +0 equal and every NaN above +inf.  One warp
+// handles one group at a time: lanes stride over the group's members and a shuffle tree takes the
+// minimum; warp 0 then reduces the G group keys.  A single CTA does the whole election (P is the
+// number of workers, at most a few thousand); the work is latency, not bandwidth.
+//
+// Optionally the kernel first finishes a two-stage loss reduction: loss_i = scale * sum_b
+// partials[i][b], summed in fp64 in index order by one lane per worker, so the value does not depend
+// on scheduling.
+#include "internal.h"
+
+namespace lsgd {
+namespace {
+
+constexpr int kElectThreads = 256;
+
+__device__ __forceinline__ uint32_t orderable(float v) {
+  if (v != v) return 0xFFFFFFFFu;            // NaN: after +inf
+  uint32_t u = __float_as_uint(v + 0.0f);    // -0 + 0 = +0 in round-to-nearest
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ unsigned long long warp_min(unsigned long long k) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, k, o);
+    k = other < k ? other : k;
+  }
+  return k;
+}
+
+__global__ void __launch_bounds__(kElectThreads) elect_kernel(ElectArgs p) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  if (p.partials != nullptr) {
+    for (int i = threadIdx.x; i < p.P; i += blockDim.x) {
+      const double* row = p.partials + (int64_t)i * p.n_partials;
+      double acc = 0.0;
+      for (int b = 0; b < p.n_partials; ++b) acc += row[b];
+      p.loss_out[i] = (float)(acc * p.partial_scale);
+    }
+  } else if (p.loss_in != p.loss_out) {
+    for (int i = threadIdx.x; i < p.P; i += blockDim.x) p.loss_out[i] = p.loss_in[i];
+  }
+  __syncthreads();
+  for (int j = warp; j < p.G; j += nwarps) {
+    const int m0 = p.tab.group_start[j], m1 = p.tab.group_start[j + 1];
+    unsigned long long best = ~0ull;
+    for (int m = m0 + lane; m < m1; m += 32) {
+      const int i = p.tab.rows_by_group[m];
+      const unsigned long long k = ((unsigned long long)orderable(p.loss_out[i]) << 32) | (uint32_t)i;
+      best = k < best ? k : best;
+    }
+    best = warp_min(best);
+    if (lane == 0) {
+      p.group_keys[j] = best;
+      const int l = (int)(uint32_t)best;
+      p.ll[j] = l;
+      atomicAdd(p.count_local + l, 1);
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    unsigned long long best = ~0ull;
+    for (int j = lane; j < p.G; j += 32) {
+      const unsigned long long k = p.group_keys[j];
+      best = k < best ? k : best;
+    }
+    best = warp_min(best);
+    if (lane == 0) {
+      const int l = (int)(uint32_t)best;
+      *p.gl = l;
+      atomicAdd(p.count_global + l, 1);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_elect(const ElectArgs& a, cudaStream_t s) {
+  elect_kernel<<<1, kElectThreads, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace lsgd

@@ -1,0 +1,119 @@
+// Internal declarations shared by the host API and the kernel launchers.  Not installed.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "lsgd.h"
+
+namespace lsgd {
+
+// Status-word bits set by kernels (reported as LSGD_ERR_DEVICE_FLAG).
+enum : uint32_t {
+  FLAG_BAD_LEADER = 1u << 0,   // a leader index outside [0, P) reached the update kernel
+  FLAG_WAIT_TIMEOUT = 1u << 1, // a bounded mbarrier / tensor-pipe wait ran out
+  FLAG_BAD_INDEX = 1u << 2,    // a batch position / sample index out of range (entry skipped)
+};
+
+struct GroupTables {
+  // Workers sorted by group: members of group j are rows_by_group[group_start[j] .. group_start[j+1]).
+  const int32_t* rows_by_group;  // DEVICE int32[P]
+  const int32_t* group_start;    // DEVICE int32[G+1]
+  const int32_t* group_of;       // DEVICE int32[P]
+};
+
+// Inline gradient of the diagonal quadratic inside the update kernel (g never touches memory).
+struct QuadInline {
+  const float* a;      // DEVICE [ld]
+  const float* b;      // DEVICE [ld]
+  const float* noise;  // DEVICE [P*ld] or nullptr
+  float sigma;
+};
+
+// Step coefficients in both precisions: eta, eta*lambda_l, eta*lambda_g, sigma.
+struct Coef {
+  double eta, cl, cg, sigma;
+  float eta_f, cl_f, cg_f, sigma_f;
+};
+
+struct UpdateArgs {
+  float* x;
+  const float* g;           // nullptr => use quad
+  QuadInline quad;
+  uint16_t* x_bf16;         // optional bf16 shadow of x, same [P][ld] layout (nullptr = none)
+  int64_t d, ld;
+  int32_t P, G;
+  GroupTables tab;
+  const int32_t* ll;        // DEVICE int32[G]
+  const int32_t* gl;        // DEVICE int32[1]
+  Coef k;
+  int arith;                // 0 fp64 unfused, 1 fp64 fma, 2 fp32 fma (see update.cu)
+  uint32_t* status;
+  bool pull;
+};
+cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s);
+
+struct ElectArgs {
+  const float* loss_in;     // DEVICE float[P] or nullptr when partials are given
+  const double* partials;   // DEVICE double[P][n_partials] (row sums in fixed order) or nullptr
+  int32_t n_partials;
+  double partial_scale;     // loss_i = partial_scale * sum_b partials[i][b]
+  float* loss_out;          // DEVICE float[P]: the loss vector the election used
+  int32_t P, G;
+  GroupTables tab;
+  int32_t* ll;
+  int32_t* gl;
+  unsigned long long* group_keys;  // DEVICE u64[G] scratch
+  int32_t* count_global;    // DEVICE int32[P]
+  int32_t* count_local;     // DEVICE int32[P]
+};
+cudaError_t launch_elect(const ElectArgs& a, cudaStream_t s);
+
+// Quadratic objective.
+cudaError_t launch_quadratic_grad(const float* x, float* g, const float* a, const float* b,
+                                  const float* noise, float sigma, int32_t P, int64_t d, int64_t ld,
+                                  bool fp64, cudaStream_t s);
+int32_t quadratic_loss_blocks(int64_t d);
+cudaError_t launch_quadratic_loss_partials(const float* x, const float* a, const float* b, int32_t P,
+                                           int64_t d, int64_t ld, double* partials, int32_t n_partials,
+                                           cudaStream_t s);
+
+// Matrix completion objective.
+struct MatcompArgs {
+  lsgd_matcomp_desc m;
+  const float* x;
+  float* g;
+  int64_t ld;
+  int32_t P;
+  uint32_t* status;
+};
+cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, cudaStream_t s);
+int32_t matcomp_loss_blocks(int32_t n_heldout);
+cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials, int32_t n_partials,
+                                         cudaStream_t s);
+
+}  // namespace lsgd
+
+struct lsgd_ctx {
+  lsgd_config cfg;
+  lsgd_quadratic_desc quad;
+  lsgd_matcomp_desc mc;
+  lsgd_mlp_desc mlp;
+  cudaStream_t stream;
+  int device;
+  std::vector<int32_t> group_of;
+  // one device slab holding all small state
+  void* slab;
+  int32_t *d_rows_by_group, *d_group_start, *d_group_of, *d_ll, *d_gl, *d_count_g, *d_count_l;
+  uint32_t* d_status;
+  float* d_loss;
+  unsigned long long* d_group_keys;
+  double* d_partials;
+  int32_t n_partials;
+  int64_t t;
+  int64_t n_elections;
+  bool grad_ready;
+  const float* armed_noise;  // QUADRATIC with g == NULL: noise pointer for the next step
+  void* mlp_state;           // opaque MLP pipeline state
+};

@@ -1,0 +1,364 @@
+// Host side of the C ABI: validation, group tables, device state, and the dispatch of each entry
+// point to its kernels.  See include/lsgd.h for the contract of every function.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+#include "mlp.h"
+
+using namespace lsgd;
+
+namespace {
+
+constexpr int32_t kMaxWorkers = 4096;  // group tables live in shared memory of the update kernel
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t up256(size_t n) { return (n + 255) & ~size_t(255); }
+
+#define LSGD_CUDA(expr)                          \
+  do {                                           \
+    cudaError_t e__ = (expr);                    \
+    if (e__ != cudaSuccess) return LSGD_ERR_CUDA; \
+  } while (0)
+
+lsgd_status validate(const lsgd_config* c) {
+  if (!c) return LSGD_ERR_INVALID_ARG;
+  if (c->struct_size != sizeof(lsgd_config)) return LSGD_ERR_INVALID_ARG;
+  if (c->P < 1 || c->d < 1 || c->ld < c->d || c->tau < 1) return LSGD_ERR_INVALID_ARG;
+  if (!std::isfinite(c->eta) || !std::isfinite(c->lambda_l) || !std::isfinite(c->lambda_g)) return LSGD_ERR_INVALID_ARG;
+  if (c->G < 1 || c->G > c->P) return LSGD_ERR_BAD_GROUPS;
+  if (!c->group_of) return LSGD_ERR_INVALID_ARG;
+  {
+    std::vector<int32_t> cnt(c->G, 0);
+    for (int i = 0; i < c->P; ++i) {
+      if (c->group_of[i] < 0 || c->group_of[i] >= c->G) return LSGD_ERR_BAD_GROUPS;
+      cnt[c->group_of[i]]++;
+    }
+    for (int j = 0; j < c->G; ++j)
+      if (cnt[j] == 0) return LSGD_ERR_BAD_GROUPS;
+  }
+  if (c->arithmetic < LSGD_ARITH_FP64 || c->arithmetic > LSGD_ARITH_FP32) return LSGD_ERR_INVALID_ARG;
+  if (c->P > kMaxWorkers) return LSGD_ERR_UNSUPPORTED;
+  if (c->ld % 32 != 0) return LSGD_ERR_ALIGNMENT;
+  if (!c->x) return LSGD_ERR_INVALID_ARG;
+  if (!aligned16(c->x) || !aligned16(c->g)) return LSGD_ERR_ALIGNMENT;
+  switch (c->objective) {
+    case LSGD_OBJ_EXTERNAL:
+      if (!c->g) return LSGD_ERR_INVALID_ARG;
+      break;
+    case LSGD_OBJ_QUADRATIC: {
+      const auto* q = static_cast<const lsgd_quadratic_desc*>(c->objective_desc);
+      if (!q || !q->a || !q->b || !std::isfinite(q->sigma)) return LSGD_ERR_INVALID_ARG;
+      if (!aligned16(q->a) || !aligned16(q->b)) return LSGD_ERR_ALIGNMENT;
+      break;
+    }
+    case LSGD_OBJ_MATCOMP: {
+      const auto* m = static_cast<const lsgd_matcomp_desc*>(c->objective_desc);
+      if (!m || !c->g) return LSGD_ERR_INVALID_ARG;
+      if (m->n_rows < 1 || m->n_cols < 1 || m->rank < 1 || m->n_obs < 1 || m->batch < 1 || m->n_heldout < 1)
+        return LSGD_ERR_INVALID_ARG;
+      if (!m->obs_r || !m->obs_c || !m->obs_v || !m->heldout_pos) return LSGD_ERR_INVALID_ARG;
+      if ((int64_t)(m->n_rows + (int64_t)m->n_cols) * m->rank != c->d) return LSGD_ERR_INVALID_ARG;
+      if (m->rank > 32) return LSGD_ERR_UNSUPPORTED;
+      break;
+    }
+    case LSGD_OBJ_MLP: {
+      const auto* m = static_cast<const lsgd_mlp_desc*>(c->objective_desc);
+      if (!m || !c->g) return LSGD_ERR_INVALID_ARG;
+      lsgd_status st = mlp_validate(*c, *m);
+      if (st != LSGD_OK) return st;
+      break;
+    }
+    default:
+      return LSGD_ERR_INVALID_ARG;
+  }
+  return LSGD_OK;
+}
+
+GroupTables tables(const lsgd_ctx* h) { return GroupTables{h->d_rows_by_group, h->d_group_start, h->d_group_of}; }
+
+}  // namespace
+
+extern "C" {
+
+lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
+  if (out) *out = nullptr;
+  if (!out) return LSGD_ERR_INVALID_ARG;
+  lsgd_status st = validate(cfg);
+  if (st != LSGD_OK) return st;
+
+  lsgd_ctx* h = new (std::nothrow) lsgd_ctx();
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  h->cfg = *cfg;
+  h->group_of.assign(cfg->group_of, cfg->group_of + cfg->P);
+  h->cfg.group_of = h->group_of.data();
+  h->stream = static_cast<cudaStream_t>(cfg->stream);
+  h->t = 0;
+  h->n_elections = 0;
+  h->grad_ready = false;
+  h->armed_noise = nullptr;
+  h->slab = nullptr;
+  h->mlp_state = nullptr;
+  std::memset(&h->quad, 0, sizeof(h->quad));
+  std::memset(&h->mc, 0, sizeof(h->mc));
+  std::memset(&h->mlp, 0, sizeof(h->mlp));
+  h->n_partials = 0;
+  if (cfg->objective == LSGD_OBJ_QUADRATIC) {
+    h->quad = *static_cast<const lsgd_quadratic_desc*>(cfg->objective_desc);
+    h->n_partials = quadratic_loss_blocks(cfg->d);
+  } else if (cfg->objective == LSGD_OBJ_MATCOMP) {
+    h->mc = *static_cast<const lsgd_matcomp_desc*>(cfg->objective_desc);
+    h->n_partials = matcomp_loss_blocks(h->mc.n_heldout);
+  } else if (cfg->objective == LSGD_OBJ_MLP) {
+    h->mlp = *static_cast<const lsgd_mlp_desc*>(cfg->objective_desc);
+  }
+  h->cfg.objective_desc = nullptr;
+
+  if (cudaGetDevice(&h->device) != cudaSuccess) {
+    delete h;
+    return LSGD_ERR_CUDA;
+  }
+
+  // Workers sorted by group (counting sort keeps index order inside a group).
+  const int P = cfg->P, G = cfg->G;
+  std::vector<int32_t> start(G + 1, 0), rows(P);
+  for (int i = 0; i < P; ++i) start[h->group_of[i] + 1]++;
+  for (int j = 0; j < G; ++j) start[j + 1] += start[j];
+  {
+    std::vector<int32_t> fill(start.begin(), start.end() - 1);
+    for (int i = 0; i < P; ++i) rows[fill[h->group_of[i]]++] = i;
+  }
+
+  // One slab: rows_by_group[P] group_start[G+1] group_of[P] ll[G] gl[1] count_g[P] count_l[P]
+  //           status[1] loss[P] group_keys[G] partials[P*n_partials]
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += up256(bytes); return o; };
+  const size_t o_rows = take(sizeof(int32_t) * P), o_start = take(sizeof(int32_t) * (G + 1));
+  const size_t o_gof = take(sizeof(int32_t) * P), o_ll = take(sizeof(int32_t) * G), o_gl = take(sizeof(int32_t));
+  const size_t o_cg = take(sizeof(int32_t) * P), o_cl = take(sizeof(int32_t) * P), o_status = take(sizeof(uint32_t));
+  const size_t o_loss = take(sizeof(float) * P), o_keys = take(sizeof(unsigned long long) * G);
+  const size_t o_part = take(sizeof(double) * (size_t)P * (size_t)(h->n_partials > 0 ? h->n_partials : 1));
+  if (cudaMalloc(&h->slab, off) != cudaSuccess) {
+    delete h;
+    return LSGD_ERR_CUDA;
+  }
+  char* base = static_cast<char*>(h->slab);
+  h->d_rows_by_group = reinterpret_cast<int32_t*>(base + o_rows);
+  h->d_group_start = reinterpret_cast<int32_t*>(base + o_start);
+  h->d_group_of = reinterpret_cast<int32_t*>(base + o_gof);
+  h->d_ll = reinterpret_cast<int32_t*>(base + o_ll);
+  h->d_gl = reinterpret_cast<int32_t*>(base + o_gl);
+  h->d_count_g = reinterpret_cast<int32_t*>(base + o_cg);
+  h->d_count_l = reinterpret_cast<int32_t*>(base + o_cl);
+  h->d_status = reinterpret_cast<uint32_t*>(base + o_status);
+  h->d_loss = reinterpret_cast<float*>(base + o_loss);
+  h->d_group_keys = reinterpret_cast<unsigned long long*>(base + o_keys);
+  h->d_partials = reinterpret_cast<double*>(base + o_part);
+
+  bool ok = cudaMemsetAsync(h->slab, 0, off, h->stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(h->d_rows_by_group, rows.data(), sizeof(int32_t) * P, cudaMemcpyHostToDevice, h->stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(h->d_group_start, start.data(), sizeof(int32_t) * (G + 1), cudaMemcpyHostToDevice, h->stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(h->d_group_of, h->group_of.data(), sizeof(int32_t) * P, cudaMemcpyHostToDevice, h->stream) == cudaSuccess;
+  // the host vectors die at return: drain the copies now (creation is not on the hot path)
+  ok = ok && cudaStreamSynchronize(h->stream) == cudaSuccess;
+  if (ok && cfg->objective == LSGD_OBJ_MLP) ok = (mlp_create(h) == LSGD_OK);
+  if (!ok) {
+    cudaFree(h->slab);
+    delete h;
+    return LSGD_ERR_CUDA;
+  }
+  *out = h;
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  const lsgd_config& c = h->cfg;
+  switch (c.objective) {
+    case LSGD_OBJ_EXTERNAL:
+      break;
+    case LSGD_OBJ_QUADRATIC:
+      if (batch && !aligned16(batch)) return LSGD_ERR_ALIGNMENT;
+      if (c.g) {
+        LSGD_CUDA(launch_quadratic_grad(c.x, c.g, h->quad.a, h->quad.b, static_cast<const float*>(batch),
+                                        h->quad.sigma, c.P, c.d, c.ld, c.arithmetic != LSGD_ARITH_FP32,
+                                        h->stream));
+      } else {
+        h->armed_noise = static_cast<const float*>(batch);
+      }
+      break;
+    case LSGD_OBJ_MATCOMP: {
+      if (!batch) return LSGD_ERR_INVALID_ARG;
+      MatcompArgs a{h->mc, c.x, c.g, c.ld, c.P, h->d_status};
+      LSGD_CUDA(launch_matcomp_grad(a, static_cast<const int32_t*>(batch), h->stream));
+      break;
+    }
+    case LSGD_OBJ_MLP: {
+      if (!batch) return LSGD_ERR_INVALID_ARG;
+      lsgd_status st = mlp_grad(h, static_cast<const int32_t*>(batch));
+      if (st != LSGD_OK) return st;
+      break;
+    }
+    default:
+      return LSGD_ERR_INVALID_ARG;
+  }
+  h->grad_ready = true;
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  const lsgd_config& c = h->cfg;
+  ElectArgs e{};
+  e.loss_in = loss;
+  e.partials = nullptr;
+  e.n_partials = 0;
+  e.partial_scale = 1.0;
+  e.loss_out = h->d_loss;
+  e.P = c.P;
+  e.G = c.G;
+  e.tab = tables(h);
+  e.ll = h->d_ll;
+  e.gl = h->d_gl;
+  e.group_keys = h->d_group_keys;
+  e.count_global = h->d_count_g;
+  e.count_local = h->d_count_l;
+  if (!loss) {
+    switch (c.objective) {
+      case LSGD_OBJ_QUADRATIC:
+        LSGD_CUDA(launch_quadratic_loss_partials(c.x, h->quad.a, h->quad.b, c.P, c.d, c.ld, h->d_partials,
+                                                 h->n_partials, h->stream));
+        e.partials = h->d_partials;
+        e.n_partials = h->n_partials;
+        e.partial_scale = 0.5;
+        break;
+      case LSGD_OBJ_MATCOMP: {
+        MatcompArgs a{h->mc, c.x, c.g, c.ld, c.P, h->d_status};
+        LSGD_CUDA(launch_matcomp_loss_partials(a, h->d_partials, h->n_partials, h->stream));
+        e.partials = h->d_partials;
+        e.n_partials = h->n_partials;
+        e.partial_scale = 1.0 / (double)h->mc.n_heldout;
+        break;
+      }
+      case LSGD_OBJ_MLP: {
+        lsgd_status st = mlp_heldout_loss(h, h->d_loss);
+        if (st != LSGD_OK) return st;
+        e.loss_in = h->d_loss;
+        break;
+      }
+      default:
+        return LSGD_ERR_INVALID_ARG;  // EXTERNAL has no loss of its own
+    }
+  }
+  LSGD_CUDA(launch_elect(e, h->stream));
+  h->n_elections++;
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_step(lsgd_handle h) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  const lsgd_config& c = h->cfg;
+  const bool pull = (h->t % c.tau) == 0;
+  if (pull && h->n_elections == 0) return LSGD_ERR_STATE;
+  if (c.objective != LSGD_OBJ_EXTERNAL && !h->grad_ready) return LSGD_ERR_STATE;
+  UpdateArgs a{};
+  a.x = c.x;
+  a.g = c.g;
+  a.quad = QuadInline{h->quad.a, h->quad.b, h->armed_noise, h->quad.sigma};
+  a.x_bf16 = (c.objective == LSGD_OBJ_MLP) ? mlp_weight_shadow(h) : nullptr;
+  a.d = c.d;
+  a.ld = c.ld;
+  a.P = c.P;
+  a.G = c.G;
+  a.tab = tables(h);
+  a.ll = h->d_ll;
+  a.gl = h->d_gl;
+  a.k.eta = (double)c.eta;
+  a.k.cl = (double)c.eta * (double)c.lambda_l;
+  a.k.cg = (double)c.eta * (double)c.lambda_g;
+  a.k.sigma = (double)h->quad.sigma;
+  a.k.eta_f = c.eta;
+  a.k.cl_f = (float)a.k.cl;
+  a.k.cg_f = (float)a.k.cg;
+  a.k.sigma_f = h->quad.sigma;
+  a.arith = c.arithmetic;
+  a.status = h->d_status;
+  a.pull = pull;
+  LSGD_CUDA(launch_update(a, h->stream));
+  h->t++;
+  h->grad_ready = false;
+  h->armed_noise = nullptr;
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_destroy(lsgd_handle h) {
+  if (!h) return LSGD_OK;
+  cudaStreamSynchronize(h->stream);
+  if (h->mlp_state) mlp_destroy(h);
+  cudaError_t e = cudaFree(h->slab);
+  delete h;
+  return e == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
+}
+
+lsgd_status lsgd_get_leaders(lsgd_handle h, int32_t* local_leaders, int32_t* global_leader) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  if (h->n_elections == 0) return LSGD_ERR_STATE;
+  LSGD_CUDA(cudaStreamSynchronize(h->stream));
+  if (local_leaders) LSGD_CUDA(cudaMemcpy(local_leaders, h->d_ll, sizeof(int32_t) * h->cfg.G, cudaMemcpyDeviceToHost));
+  if (global_leader) LSGD_CUDA(cudaMemcpy(global_leader, h->d_gl, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_get_loss(lsgd_handle h, float* loss) {
+  if (!h || !loss) return LSGD_ERR_INVALID_ARG;
+  LSGD_CUDA(cudaStreamSynchronize(h->stream));
+  LSGD_CUDA(cudaMemcpy(loss, h->d_loss, sizeof(float) * h->cfg.P, cudaMemcpyDeviceToHost));
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_get_step(lsgd_handle h, int64_t* t) {
+  if (!h || !t) return LSGD_ERR_INVALID_ARG;
+  *t = h->t;
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_get_leader_counts(lsgd_handle h, int32_t* global_counts, int32_t* local_counts) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  LSGD_CUDA(cudaStreamSynchronize(h->stream));
+  if (global_counts) LSGD_CUDA(cudaMemcpy(global_counts, h->d_count_g, sizeof(int32_t) * h->cfg.P, cudaMemcpyDeviceToHost));
+  if (local_counts) LSGD_CUDA(cudaMemcpy(local_counts, h->d_count_l, sizeof(int32_t) * h->cfg.P, cudaMemcpyDeviceToHost));
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  uint32_t f = 0;
+  LSGD_CUDA(cudaStreamSynchronize(h->stream));
+  LSGD_CUDA(cudaMemcpy(&f, h->d_status, sizeof(f), cudaMemcpyDeviceToHost));
+  if (f) LSGD_CUDA(cudaMemset(h->d_status, 0, sizeof(f)));
+  if (flag_out) *flag_out = f;
+  return f ? LSGD_ERR_DEVICE_FLAG : LSGD_OK;
+}
+
+lsgd_status lsgd_set_eta(lsgd_handle h, float eta) {
+  if (!h || !std::isfinite(eta)) return LSGD_ERR_INVALID_ARG;
+  h->cfg.eta = eta;
+  return LSGD_OK;
+}
+
+const char* lsgd_status_string(lsgd_status s) {
+  switch (s) {
+    case LSGD_OK: return "ok";
+    case LSGD_ERR_INVALID_ARG: return "invalid argument";
+    case LSGD_ERR_BAD_GROUPS: return "bad group assignment";
+    case LSGD_ERR_ALIGNMENT: return "misaligned pointer or row stride";
+    case LSGD_ERR_STATE: return "call order violates the step protocol";
+    case LSGD_ERR_CUDA: return "CUDA runtime error";
+    case LSGD_ERR_UNSUPPORTED: return "unsupported configuration";
+    case LSGD_ERR_DEVICE_FLAG: return "a kernel reported a device-side failure";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

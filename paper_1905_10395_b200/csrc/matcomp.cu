@@ -1,0 +1,122 @@
+// Factorised matrix completion on observed entries (low-rank completion is the paper's motivating
+// example, Section 2.1; here with two factors and a sampled set of observed cells).
+// Worker row = [X (n_rows x rank) | Y (n_cols x rank)], both row-major.
+//
+//   gradient of (1/(2B)) sum_{(r,c,v) in batch} (<X_r, Y_c> - v)^2 :
+//     dX_r += e Y_c / B,  dY_c += e X_r / B,  e = <X_r, Y_c> - v     (duplicates in a batch add up)
+//   election loss: (1/N) sum over the held-out list of e^2, fp64 partial sums in a fixed order.
+//
+// The whole state of this workload (a few MB per worker) lives in L2; the kernels are gather /
+// scatter bound, not HBM bound.  The gradient buffer is cleared and then accumulated with fp32
+// reductions in L2; rows hit once or twice in a batch are order-independent (fp addition commutes),
+// rows hit three or more times may differ in the last bit from run to run.
+#include "internal.h"
+
+namespace lsgd {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxRank = 32;
+constexpr int kLossPerThread = 4;
+
+__global__ void __launch_bounds__(kThreads)
+matcomp_grad_kernel(MatcompArgs a, const int32_t* __restrict__ pos) {
+  const int i = blockIdx.y;
+  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= a.m.batch) return;
+  const int q = pos[(int64_t)i * a.m.batch + p];
+  if (q < 0 || q >= a.m.n_obs) {
+    atomicOr(a.status, FLAG_BAD_INDEX);
+    return;
+  }
+  const int r = a.m.obs_r[q], c = a.m.obs_c[q];
+  if (r < 0 || r >= a.m.n_rows || c < 0 || c >= a.m.n_cols) {
+    atomicOr(a.status, FLAG_BAD_INDEX);
+    return;
+  }
+  const int rank = a.m.rank;
+  const int64_t xo = (int64_t)i * a.ld + (int64_t)r * rank;
+  const int64_t yo = (int64_t)i * a.ld + ((int64_t)a.m.n_rows + c) * rank;
+  float xr[kMaxRank], yc[kMaxRank];
+  float dot = 0.f;
+#pragma unroll
+  for (int k = 0; k < kMaxRank; ++k) {
+    if (k < rank) {
+      xr[k] = a.x[xo + k];
+      yc[k] = a.x[yo + k];
+      dot = fmaf(xr[k], yc[k], dot);
+    }
+  }
+  const float e = (dot - a.m.obs_v[q]) / (float)a.m.batch;
+#pragma unroll
+  for (int k = 0; k < kMaxRank; ++k) {
+    if (k < rank) {
+      atomicAdd(a.g + xo + k, e * yc[k]);
+      atomicAdd(a.g + yo + k, e * xr[k]);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+matcomp_loss_kernel(MatcompArgs a, double* __restrict__ partials, int32_t n_partials) {
+  const int i = blockIdx.y;
+  const int rank = a.m.rank;
+  const float* xi = a.x + (int64_t)i * a.ld;
+  double acc = 0.0;
+#pragma unroll
+  for (int u = 0; u < kLossPerThread; ++u) {
+    const int p = (blockIdx.x * kLossPerThread + u) * kThreads + threadIdx.x;
+    if (p < a.m.n_heldout) {
+      const int q = a.m.heldout_pos[p];
+      if (q < 0 || q >= a.m.n_obs) {
+        atomicOr(a.status, FLAG_BAD_INDEX);
+        continue;
+      }
+      const int r = a.m.obs_r[q], c = a.m.obs_c[q];
+      if (r < 0 || r >= a.m.n_rows || c < 0 || c >= a.m.n_cols) {
+        atomicOr(a.status, FLAG_BAD_INDEX);
+        continue;
+      }
+      const float* xr = xi + (int64_t)r * rank;
+      const float* yc = xi + ((int64_t)a.m.n_rows + c) * rank;
+      double dot = 0.0;
+      for (int k = 0; k < rank; ++k) dot += (double)xr[k] * (double)yc[k];
+      const double e = dot - (double)a.m.obs_v[q];
+      acc += e * e;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+  __shared__ double s_w[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) t += s_w[w];
+    partials[(int64_t)i * n_partials + blockIdx.x] = t;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, cudaStream_t s) {
+  cudaError_t e = cudaMemsetAsync(a.g, 0, sizeof(float) * (size_t)a.P * (size_t)a.ld, s);
+  if (e != cudaSuccess) return e;
+  dim3 grid((unsigned)((a.m.batch + kThreads - 1) / kThreads), (unsigned)a.P);
+  matcomp_grad_kernel<<<grid, kThreads, 0, s>>>(a, pos);
+  return cudaGetLastError();
+}
+
+int32_t matcomp_loss_blocks(int32_t n_heldout) {
+  const int per = kThreads * kLossPerThread;
+  return (n_heldout + per - 1) / per;
+}
+
+cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials, int32_t n_partials, cudaStream_t s) {
+  dim3 grid((unsigned)n_partials, (unsigned)a.P);
+  matcomp_loss_kernel<<<grid, kThreads, 0, s>>>(a, partials, n_partials);
+  return cudaGetLastError();
+}
+
+}  // namespace lsgd

@@ -1,0 +1,259 @@
+// Fused LSGD update (Eq. (1) with eta-scaled pulls, Section 3.1.1) and the plain (S)GD step used
+// between communications (Section 3.1.2).
+//
+// Pull form.  A thread owns one 16-byte column (4 consecutive parameters) for ALL P workers.  It
+// reads the global leader's 4 values once, then walks the workers group by group: the group's local
+// leader is read once into registers, after which each member row is read, updated and written.
+// A leader row is taken from the registers it was staged in instead of being read again, so every
+// byte of x and g is read exactly once and every byte of x written exactly once (12 B per
+// worker-parameter, leaders cost nothing extra).  Because the same thread reads a leader's column
+// before it (or anyone) writes it, all right-hand sides are x at time t although x is updated in
+// place -- the simultaneous update the paper describes ("all workers are updated at the same
+// time", Section 2.2).
+//
+// A leader's own pull term is (x - x) = 0 exactly, and fmaf(-c, 0, acc) == acc, so the leader's
+// step is bit-identical to the plain step without a branch (supplement, "Definitions and Notation":
+// the update reduces to an (S)GD step for the leader).
+#include <cuda_bf16.h>
+
+#include "internal.h"
+
+namespace lsgd {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRowsInFlight = 4;  // rows whose loads are issued before the first is consumed
+
+__device__ __forceinline__ float4 ld4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 ld4_cached(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ void st4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+
+__device__ __forceinline__ void st4_bf16(uint16_t* p, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t*>(&lo);
+  u.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+
+// Arithmetic modes (UpdateArgs::arith).  The stored types are always fp32.
+//   0: fp64 evaluation, one IEEE operation per printed operation (no contraction), one rounding to
+//      fp32 at the end -- the same value a plain double-precision restatement of Eq. (1) produces;
+//   1: fp64 evaluation with fused multiply-adds;
+//   2: fp32 fused multiply-adds.
+template <int MODE>
+__device__ __forceinline__ float quad_g(float x, float a, float b, float n, const Coef& k, bool noise) {
+  if (MODE == 0) {
+    double r = __dmul_rn((double)a, __dsub_rn((double)x, (double)b));
+    if (noise) r = __dadd_rn(r, __dmul_rn(k.sigma, (double)n));
+    return (float)r;
+  } else if (MODE == 1) {
+    double r = (double)a * ((double)x - (double)b);
+    if (noise) r = fma(k.sigma, (double)n, r);
+    return (float)r;
+  } else {
+    return fmaf(a, x - b, noise ? k.sigma_f * n : 0.f);
+  }
+}
+
+template <int MODE>
+__device__ __forceinline__ float plain1(float x, float g, const Coef& k) {
+  if (MODE == 0) return (float)__dsub_rn((double)x, __dmul_rn(k.eta, (double)g));
+  if (MODE == 1) return (float)fma(-k.eta, (double)g, (double)x);
+  return fmaf(-k.eta_f, g, x);
+}
+
+template <int MODE>
+__device__ __forceinline__ float pull1(float x, float g, float xl, float xg, const Coef& k) {
+  if (MODE == 0) {
+    const double X = (double)x;
+    double acc = __dsub_rn(X, __dmul_rn(k.eta, (double)g));
+    acc = __dsub_rn(acc, __dmul_rn(k.cl, __dsub_rn(X, (double)xl)));
+    acc = __dsub_rn(acc, __dmul_rn(k.cg, __dsub_rn(X, (double)xg)));
+    return (float)acc;
+  } else if (MODE == 1) {
+    const double X = (double)x;
+    double acc = fma(-k.eta, (double)g, X);
+    acc = fma(-k.cl, X - (double)xl, acc);
+    acc = fma(-k.cg, X - (double)xg, acc);
+    return (float)acc;
+  } else {
+    float acc = fmaf(-k.eta_f, g, x);
+    acc = fmaf(-k.cl_f, x - xl, acc);
+    acc = fmaf(-k.cg_f, x - xg, acc);
+    return acc;
+  }
+}
+
+template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
+__global__ void __launch_bounds__(kThreads)
+pull_update_kernel(UpdateArgs p, int64_t n4) {
+  extern __shared__ int32_t s_tab[];
+  int32_t* s_ll = s_tab;                 // [G]
+  int32_t* s_start = s_ll + p.G;         // [G+1]
+  int32_t* s_rows = s_start + p.G + 1;   // [P]
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  for (int k = threadIdx.x; k < p.G; k += blockDim.x) {
+    int l = p.ll[k];
+    if (l < 0 || l >= p.P) s_bad = 1;
+    s_ll[k] = l;
+  }
+  for (int k = threadIdx.x; k <= p.G; k += blockDim.x) s_start[k] = p.tab.group_start[k];
+  for (int k = threadIdx.x; k < p.P; k += blockDim.x) s_rows[k] = p.tab.rows_by_group[k];
+  const int gl = *p.gl;
+  if (threadIdx.x == 0 && (gl < 0 || gl >= p.P)) s_bad = 1;
+  __syncthreads();
+  if (s_bad) {  // never dereference a leader index that is out of range
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(p.status, FLAG_BAD_LEADER);
+    return;
+  }
+  const Coef k = p.k;
+  const int64_t ld = p.ld;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < n4; c += stride) {
+    const int64_t col = c * 4;
+    float* xc = p.x + col;
+    const float* gc = (QUAD ? p.quad.noise : p.g) + col;
+    const float4 xg = ld4(xc + (int64_t)gl * ld);
+    float4 av, bv;
+    if (QUAD) {
+      av = ld4_cached(p.quad.a + col);
+      bv = ld4_cached(p.quad.b + col);
+    }
+    for (int j = 0; j < p.G; ++j) {
+      const int l = s_ll[j];
+      const float4 xl = (l == gl) ? xg : ld4(xc + (int64_t)l * ld);
+      const int m1 = s_start[j + 1];
+      for (int m = s_start[j]; m < m1; m += kRowsInFlight) {
+        float4 xs[kRowsInFlight], gs[kRowsInFlight];
+        int rows[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+          if (m + u < m1) {
+            const int i = s_rows[m + u];
+            rows[u] = i;
+            xs[u] = (i == l) ? xl : ld4(xc + (int64_t)i * ld);
+            if (!QUAD || NOISE) gs[u] = ld4(gc + (int64_t)i * ld);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+          if (m + u < m1) {
+            float4 x = xs[u], g = gs[u];
+            if (QUAD) {
+              g.x = quad_g<MODE>(x.x, av.x, bv.x, g.x, k, NOISE);
+              g.y = quad_g<MODE>(x.y, av.y, bv.y, g.y, k, NOISE);
+              g.z = quad_g<MODE>(x.z, av.z, bv.z, g.z, k, NOISE);
+              g.w = quad_g<MODE>(x.w, av.w, bv.w, g.w, k, NOISE);
+            }
+            float4 r;
+            r.x = pull1<MODE>(x.x, g.x, xl.x, xg.x, k);
+            r.y = pull1<MODE>(x.y, g.y, xl.y, xg.y, k);
+            r.z = pull1<MODE>(x.z, g.z, xl.z, xg.z, k);
+            r.w = pull1<MODE>(x.w, g.w, xl.w, xg.w, k);
+            st4(xc + (int64_t)rows[u] * ld, r);
+            if (SHADOW) st4_bf16(p.x_bf16 + col + (int64_t)rows[u] * ld, r);
+          }
+        }
+      }
+    }
+  }
+}
+
+// Plain step x <- x - eta g over the whole [P][n4] grid of 16-byte columns.
+template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
+__global__ void __launch_bounds__(kThreads)
+plain_update_kernel(UpdateArgs p, int64_t n4) {
+  const int64_t total = (int64_t)p.P * n4;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const Coef k = p.k;
+  for (int64_t e0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e0 < total; e0 += stride * kRowsInFlight) {
+    float4 xs[kRowsInFlight], gs[kRowsInFlight];
+    int64_t off[kRowsInFlight], cols[kRowsInFlight];
+#pragma unroll
+    for (int u = 0; u < kRowsInFlight; ++u) {
+      const int64_t e = e0 + u * stride;
+      if (e < total) {
+        const int64_t row = e / n4, c = e - row * n4;
+        cols[u] = c * 4;
+        off[u] = row * p.ld + c * 4;
+        xs[u] = ld4(p.x + off[u]);
+        if (!QUAD || NOISE) gs[u] = ld4((QUAD ? p.quad.noise : p.g) + off[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kRowsInFlight; ++u) {
+      const int64_t e = e0 + u * stride;
+      if (e < total) {
+        float4 x = xs[u], g = gs[u];
+        if (QUAD) {
+          const float4 av = ld4_cached(p.quad.a + cols[u]);
+          const float4 bv = ld4_cached(p.quad.b + cols[u]);
+          g.x = quad_g<MODE>(x.x, av.x, bv.x, g.x, k, NOISE);
+          g.y = quad_g<MODE>(x.y, av.y, bv.y, g.y, k, NOISE);
+          g.z = quad_g<MODE>(x.z, av.z, bv.z, g.z, k, NOISE);
+          g.w = quad_g<MODE>(x.w, av.w, bv.w, g.w, k, NOISE);
+        }
+        float4 r;
+        r.x = plain1<MODE>(x.x, g.x, k);
+        r.y = plain1<MODE>(x.y, g.y, k);
+        r.z = plain1<MODE>(x.z, g.z, k);
+        r.w = plain1<MODE>(x.w, g.w, k);
+        st4(p.x + off[u], r);
+        if (SHADOW) st4_bf16(p.x_bf16 + off[u], r);
+      }
+    }
+  }
+}
+
+template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
+cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
+  }
+  const int64_t n4 = (a.d + 3) / 4;
+  const int64_t cap = (int64_t)sms * 8;
+  if (a.pull) {
+    int64_t blocks = (n4 + kThreads - 1) / kThreads;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    const size_t smem = sizeof(int32_t) * (size_t)(a.P + 2 * a.G + 1);
+    pull_update_kernel<MODE, QUAD, NOISE, SHADOW><<<(unsigned)blocks, kThreads, smem, s>>>(a, n4);
+  } else {
+    const int64_t total = (int64_t)a.P * n4;
+    int64_t blocks = (total + (int64_t)kThreads * kRowsInFlight - 1) / ((int64_t)kThreads * kRowsInFlight);
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    plain_update_kernel<MODE, QUAD, NOISE, SHADOW><<<(unsigned)blocks, kThreads, 0, s>>>(a, n4);
+  }
+  return cudaGetLastError();
+}
+
+template <int MODE>
+cudaError_t launch_m(const UpdateArgs& a, cudaStream_t s) {
+  const bool quad = (a.g == nullptr);
+  const bool noise = quad && a.quad.noise != nullptr;
+  const bool shadow = a.x_bf16 != nullptr;
+  if (!quad) return shadow ? launch_t<MODE, false, false, true>(a, s) : launch_t<MODE, false, false, false>(a, s);
+  if (shadow) return cudaErrorNotSupported;
+  return noise ? launch_t<MODE, true, true, false>(a, s) : launch_t<MODE, true, false, false>(a, s);
+}
+
+}  // namespace
+
+cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s) {
+  switch (a.arith) {
+    case 0: return launch_m<0>(a, s);
+    case 1: return launch_m<1>(a, s);
+    default: return launch_m<2>(a, s);
+  }
+}
+
+}  // namespace lsgd

@@ -1,0 +1,115 @@
+"""Drives the C ABI over a `inputs.Workload`: uploads the arrays with torch, creates the handle and
+issues grad / elect / step in the order of one synchronous LSGD step.  Marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import api
+from .inputs import Workload
+
+
+class Population:
+    def __init__(self, w: Workload, *, fused_quadratic: bool = False, arithmetic: int = api.ARITH_FP64,
+                 device: str = "cuda:0", x: Optional[torch.Tensor] = None, g: Optional[torch.Tensor] = None,
+                 upload_noise: bool = True):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (there is no CPU path)")
+        self.w = w
+        self.dev = torch.device(device)
+        torch.cuda.set_device(self.dev)
+        self.stream = torch.cuda.current_stream(self.dev)
+        dev = self.dev
+        self.x = x if x is not None else torch.from_numpy(w.x0).to(dev)
+        self.g = g
+        self.batches: List[Optional[torch.Tensor]] = []
+        self.loss_ring: Optional[torch.Tensor] = None
+        self._keep = []
+        desc = None
+        A = w.arrays
+        if w.objective == "external":
+            obj = api.OBJ_EXTERNAL
+            if self.g is None:
+                self.g = torch.from_numpy(A["g"]).to(dev)
+            self.loss_ring = torch.from_numpy(A["loss_ring"]).to(dev)
+        elif w.objective == "quadratic":
+            obj = api.OBJ_QUADRATIC
+            self.a = torch.from_numpy(A["a"]).to(dev)
+            self.b = torch.from_numpy(A["b"]).to(dev)
+            desc = api.QuadraticDesc(self.a.data_ptr(), self.b.data_ptr(), float(w.meta["sigma"]))
+            if upload_noise and A.get("noise") is not None:
+                self.batches = [torch.from_numpy(n).to(dev) for n in A["noise"]]
+            if not fused_quadratic and self.g is None:
+                self.g = torch.empty_like(self.x)
+        elif w.objective == "matcomp":
+            obj = api.OBJ_MATCOMP
+            m = w.meta
+            self.obs_r = torch.from_numpy(A["obs_r"]).to(dev)
+            self.obs_c = torch.from_numpy(A["obs_c"]).to(dev)
+            self.obs_v = torch.from_numpy(A["obs_v"]).to(dev)
+            self.held = torch.from_numpy(A["heldout_pos"]).to(dev)
+            desc = api.MatcompDesc(m["n_rows"], m["n_cols"], m["rank"], len(A["obs_r"]), self.obs_r.data_ptr(),
+                                   self.obs_c.data_ptr(), self.obs_v.data_ptr(), m["batch"], len(A["heldout_pos"]),
+                                   self.held.data_ptr())
+            self.batches = [torch.from_numpy(np.ascontiguousarray(p)).to(dev) for p in A["batch_pos"]]
+            if self.g is None:
+                self.g = torch.empty_like(self.x)
+        elif w.objective == "mlp":
+            obj = api.OBJ_MLP
+            m = w.meta
+            self.pool_x = torch.from_numpy(A["pool_x"]).to(dev)
+            self.pool_y = torch.from_numpy(A["pool_y"]).to(dev)
+            self.held_x = torch.from_numpy(A["held_x"]).to(dev)
+            self.held_y = torch.from_numpy(A["held_y"]).to(dev)
+            nbytes = api.mlp_scratch_bytes(m["dims"], w.P, m["batch"], len(A["held_y"]))
+            self.scratch = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+            sp = (self.scratch.data_ptr() + 1023) // 1024 * 1024
+            desc = api.MlpDesc((C.c_int32 * 4)(*m["dims"]), m["batch"], len(A["pool_y"]), self.pool_x.data_ptr(),
+                               self.pool_y.data_ptr(), len(A["held_y"]), self.held_x.data_ptr(),
+                               self.held_y.data_ptr(), sp, nbytes)
+            self.batches = [torch.from_numpy(np.ascontiguousarray(p)).to(dev) for p in A["batch_idx"]]
+            if self.g is None:
+                self.g = torch.empty_like(self.x)
+        else:
+            raise ValueError(w.objective)
+        cfg, keep = api.make_config(P=w.P, G=w.G, group_of=w.group_of, d=w.d, ld=w.ld, eta=w.eta,
+                                    lambda_l=w.lambda_l, lambda_g=w.lambda_g, tau=w.tau, objective=obj, desc=desc,
+                                    x=self.x, g=self.g, stream=self.stream.cuda_stream, arithmetic=arithmetic)
+        self._keep.append(keep)
+        self.lsgd = api.Lsgd(cfg, keep)
+        self.t = 0
+        self.n_elections = 0
+        self.history: List[dict] = []
+
+    # one synchronous step, in the order gradient -> (election loss, election) -> update
+    def step(self, forced_loss: Optional[torch.Tensor] = None, record: bool = False) -> None:
+        w = self.w
+        batch = self.batches[self.t % len(self.batches)] if self.batches else None
+        self.lsgd.grad(batch)
+        if self.t % w.tau == 0:
+            if forced_loss is not None:
+                self.lsgd.elect(forced_loss)
+            elif self.loss_ring is not None:
+                self.lsgd.elect(self.loss_ring[self.n_elections % self.loss_ring.shape[0]])
+            else:
+                self.lsgd.elect(None)
+            self.n_elections += 1
+            if record:
+                ll, gl = self.lsgd.leaders()
+                self.history.append({"t": self.t, "ll": ll, "gl": gl, "loss": self.lsgd.loss()})
+        self.lsgd.step()
+        self.t += 1
+
+    def run(self, steps: int, record: bool = False) -> None:
+        for _ in range(steps):
+            self.step(record=record)
+
+    def x_host(self) -> np.ndarray:
+        torch.cuda.synchronize(self.dev)
+        return self.x.cpu().numpy()
+
+    def close(self) -> None:
+        self.lsgd.destroy()
