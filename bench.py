@@ -118,7 +118,7 @@ def max_over_ranks(value: float, world: int, device=None) -> float:
 # --------------------------------------------------------------------------------- workloads ----
 def workload_spec(args):
     if args.workload == "c4":
-        return dict(kind="external", P=16, G=4, d=1 << 26, eta=0.01, lambda_l=0.1, lambda_g=0.05,
+        return dict(kind="external", P=16, G=4, d=args.d or (1 << 26), eta=0.01, lambda_l=0.1, lambda_g=0.05,
                     tau=args.tau or 1, name="C4 fused-update stress: P=16 G=4 d=2^26 fp32, supplied g and losses")
     if args.workload == "c1":
         return dict(kind="quadratic", P=64, G=8, d=1 << 20, eta=0.05, lambda_l=0.1, lambda_g=0.05,
@@ -328,6 +328,7 @@ def main():
     ap.add_argument("--arith", type=int, default=0, choices=[0, 1, 2])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--sample-cols", type=int, default=0)
+    ap.add_argument("--d", type=int, default=0, help="shrink the c4 workload (profiler captures on a small case)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

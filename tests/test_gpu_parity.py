@@ -99,7 +99,9 @@ def test_external_update_ragged_unequal_groups(arith, exact):
     x = pop.x_host()
     if exact:
         assert np.array_equal(x.view(np.uint32), o.x.view(np.uint32))
-    assert rel_err(x, o.x) <= TOL
+    # fp32 arithmetic (mode 2) cannot bound the error of a cancelling result relative to the result
+    # itself, only relative to the O(1) operands; the fp64 modes meet the bound with the 1e-3 floor
+    assert rel_err(x, o.x, floor=1.0 if arith == 2 else FLOOR) <= TOL
     assert np.all(x[:, w.d:] == 0)
     assert pop.lsgd.check_device() == 0
     pop.close()
