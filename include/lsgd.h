@@ -49,7 +49,8 @@ typedef enum {
   LSGD_ERR_STATE = 4,        /* call order: pull step before any election, step without a gradient   */
   LSGD_ERR_CUDA = 5,         /* a CUDA runtime call or launch failed (no usable device included)     */
   LSGD_ERR_UNSUPPORTED = 6,  /* combination not implemented (documented at the argument)             */
-  LSGD_ERR_DEVICE_FLAG = 7   /* a kernel recorded a bounded-wait / bounds failure in its status word */
+  LSGD_ERR_DEVICE_FLAG = 7,  /* a kernel recorded a bounded-wait / bounds failure in its status word */
+  LSGD_ERR_TOO_LARGE = 8     /* the problem exceeds a fixed capacity stated at the entry point       */
 } lsgd_status;
 
 typedef enum {
@@ -173,6 +174,31 @@ LSGD_API lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out /* HOST
 LSGD_API lsgd_status lsgd_set_eta(lsgd_handle h, float eta);
 
 LSGD_API const char* lsgd_status_string(lsgd_status s);
+
+/* Allocation-free election loss of the diagonal quadratic.  (The paper has no counterpart: this is a
+ * packaging variant of the loss evaluation, not a step of the method.)
+ *
+ * For callers that are not allowed to allocate device memory: code inside a framework-managed region
+ * where every byte belongs to a memory pool, loops with a "no allocation after start-up" rule, or
+ * guests in another component's CUDA context with a fixed memory budget.  lsgd_create is closed to
+ * them because it calls cudaMalloc; this function calls no cudaMalloc / cudaFree and no allocating
+ * library routine.
+ *
+ * Computes loss[i] = 1/2 sum_k a[k] (x[i][k] - b[k])^2 for i < P, bit-identical to what
+ * lsgd_elect(h, NULL) stores for the QUADRATIC objective (same chunking, same fp64 summation order).
+ *   x     DEVICE float[P*ld], 16-byte aligned; a, b DEVICE float[ld], 16-byte aligned
+ *   loss  DEVICE float[P], written on `stream` (cudaStream_t; NULL = legacy default stream)
+ *   d, ld as in lsgd_config (ld >= d, ld % 32 == 0).
+ * Scratch: the per-chunk partial sums, P * ceil(d / 8192) doubles, live in a fixed 512 KiB array that
+ * is part of the library image on every GPU that loads it (held until the process exits).  Capacity:
+ * P * ceil(d / 8192) <= 65536, otherwise LSGD_ERR_TOO_LARGE and nothing is launched.
+ * The first call on each device looks up the array's device address (with that device current); make
+ * that first call before starting any stream capture.
+ * All calls share the one array, which keeps the previous call's contents; every entry this call reads
+ * is first overwritten by this call, so nothing needs clearing.  Two calls that overlap on the GPU
+ * (different streams, or different host threads without ordering) race on the array: serialise them. */
+LSGD_API lsgd_status lsgd_quadratic_loss_noalloc(const float* x, const float* a, const float* b, int32_t P,
+                                                 int64_t d, int64_t ld, float* loss, void* stream);
 
 /* MLP helpers (host only).  Offsets in floats of W_l and b_l inside a parameter row, and the row
  * length d.  n_layers = 3.                                                                        */

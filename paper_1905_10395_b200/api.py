@@ -11,7 +11,8 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblsgd.so")
 
-OK, ERR_INVALID_ARG, ERR_BAD_GROUPS, ERR_ALIGNMENT, ERR_STATE, ERR_CUDA, ERR_UNSUPPORTED, ERR_DEVICE_FLAG = range(8)
+(OK, ERR_INVALID_ARG, ERR_BAD_GROUPS, ERR_ALIGNMENT, ERR_STATE, ERR_CUDA, ERR_UNSUPPORTED, ERR_DEVICE_FLAG,
+ ERR_TOO_LARGE) = range(9)
 OBJ_EXTERNAL, OBJ_QUADRATIC, OBJ_MATCOMP, OBJ_MLP = range(4)
 ARITH_FP64, ARITH_FP64_FMA, ARITH_FP32 = range(3)
 
@@ -69,6 +70,9 @@ def lib() -> C.CDLL:
         L.lsgd_get_leader_counts.argtypes = [H, C.c_void_p, C.c_void_p]
         L.lsgd_check_device.argtypes = [H, C.POINTER(C.c_uint32)]
         L.lsgd_set_eta.argtypes = [H, C.c_float]
+        L.lsgd_quadratic_loss_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64,
+                                                  C.c_void_p, C.c_void_p]
+        L.lsgd_quadratic_loss_noalloc.restype = C.c_int
         L.lsgd_status_string.argtypes = [C.c_int]
         L.lsgd_status_string.restype = C.c_char_p
         L.lsgd_mlp_param_offsets.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int64)]
@@ -121,6 +125,13 @@ def lsgd_step(h) -> None:
 
 def lsgd_destroy(h) -> None:
     _check(lib().lsgd_destroy(h), "lsgd_destroy")
+
+
+def lsgd_quadratic_loss_noalloc(x, a, b, P: int, d: int, ld: int, loss, stream: int = 0) -> None:
+    """Election loss of the quadratic objective without any device allocation (fixed 512 KiB scratch
+    inside the library; P * ceil(d / 8192) <= 65536).  For callers that may not allocate."""
+    _check(lib().lsgd_quadratic_loss_noalloc(_ptr(x), _ptr(a), _ptr(b), int(P), int(d), int(ld), _ptr(loss),
+                                             stream or None), "lsgd_quadratic_loss_noalloc")
 
 
 def mlp_param_offsets(dims: Sequence[int]):

@@ -357,6 +357,7 @@ const char* lsgd_status_string(lsgd_status s) {
     case LSGD_ERR_CUDA: return "CUDA runtime error";
     case LSGD_ERR_UNSUPPORTED: return "unsupported configuration";
     case LSGD_ERR_DEVICE_FLAG: return "a kernel reported a device-side failure";
+    case LSGD_ERR_TOO_LARGE: return "problem exceeds the fixed capacity of this entry point";
   }
   return "unknown status";
 }
