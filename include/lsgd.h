@@ -206,6 +206,33 @@ LSGD_API lsgd_status lsgd_mlp_param_offsets(const int32_t* dims /* HOST int32[4]
                                    int64_t* b_off /* [3] */, int64_t* d_out);
 LSGD_API uint64_t lsgd_mlp_scratch_bytes(const int32_t* dims, int32_t P, int32_t batch, int32_t n_heldout);
 
+/* Batched bf16 x bf16 -> fp32-accumulate matrix product on the tensor cores: C[z] = A[z] . B[z] for
+ * z < batch, C is M x N, contraction length K.  This is the product the MLP objective is built from
+ * (its forward, back-propagation and weight-gradient products), exposed so that it can be checked
+ * against a library matmul on its own.  All pointers DEVICE.
+ *   a_mn_major = 0: A is stored [M][lda] (K contiguous);  1: A is stored [K][lda] (M contiguous).
+ *   b_mn_major = 0: B is stored [N][ldb] (K contiguous);  1: B is stored [K][ldb] (N contiguous).
+ *   lda, ldb, ldc: row pitch in elements; lda, ldb multiples of 8.  stride_*: elements between batch
+ *   entries (stride_a / stride_b = 0 shares the operand across the batch; multiples of 8 otherwise).
+ *   a, b 16-byte aligned.  epilogue: 0 C fp32 = acc; 1 C bf16 = relu(acc + bias[z][n]);
+ *   2 C bf16 = (mask[z][m][n] > 0 ? acc : 0), mask bf16; 3 C bf16 = acc.
+ * Enqueues on `stream` and returns.  LSGD_ERR_ALIGNMENT if an operand breaks the rules above.      */
+typedef struct {
+  const void* a;
+  const void* b;
+  void* c;
+  int32_t M, N, K, batch;
+  int32_t a_mn_major, b_mn_major;
+  int64_t lda, ldb, ldc;
+  int64_t stride_a, stride_b, stride_c;
+  int32_t epilogue;
+  const float* bias;
+  int64_t stride_bias;
+  const void* mask;
+  int64_t ld_mask, stride_mask;
+} lsgd_bgemm_desc;
+LSGD_API lsgd_status lsgd_bgemm_bf16(const lsgd_bgemm_desc* desc, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

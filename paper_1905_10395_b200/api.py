@@ -39,6 +39,14 @@ class MlpDesc(C.Structure):
                 ("scratch", C.c_void_p), ("scratch_bytes", C.c_uint64)]
 
 
+class BgemmDesc(C.Structure):
+    _fields_ = [("a", C.c_void_p), ("b", C.c_void_p), ("c", C.c_void_p), ("M", C.c_int32), ("N", C.c_int32),
+                ("K", C.c_int32), ("batch", C.c_int32), ("a_mn_major", C.c_int32), ("b_mn_major", C.c_int32),
+                ("lda", C.c_int64), ("ldb", C.c_int64), ("ldc", C.c_int64), ("stride_a", C.c_int64),
+                ("stride_b", C.c_int64), ("stride_c", C.c_int64), ("epilogue", C.c_int32), ("bias", C.c_void_p),
+                ("stride_bias", C.c_int64), ("mask", C.c_void_p), ("ld_mask", C.c_int64), ("stride_mask", C.c_int64)]
+
+
 class Config(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("P", C.c_int32), ("G", C.c_int32), ("group_of", C.c_void_p),
                 ("d", C.c_int64), ("ld", C.c_int64), ("eta", C.c_float), ("lambda_l", C.c_float),
@@ -73,6 +81,8 @@ def lib() -> C.CDLL:
         L.lsgd_quadratic_loss_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64,
                                                   C.c_void_p, C.c_void_p]
         L.lsgd_quadratic_loss_noalloc.restype = C.c_int
+        L.lsgd_bgemm_bf16.argtypes = [C.POINTER(BgemmDesc), C.c_void_p]
+        L.lsgd_bgemm_bf16.restype = C.c_int
         L.lsgd_status_string.argtypes = [C.c_int]
         L.lsgd_status_string.restype = C.c_char_p
         L.lsgd_mlp_param_offsets.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int64)]
@@ -132,6 +142,10 @@ def lsgd_quadratic_loss_noalloc(x, a, b, P: int, d: int, ld: int, loss, stream: 
     inside the library; P * ceil(d / 8192) <= 65536).  For callers that may not allocate."""
     _check(lib().lsgd_quadratic_loss_noalloc(_ptr(x), _ptr(a), _ptr(b), int(P), int(d), int(ld), _ptr(loss),
                                              stream or None), "lsgd_quadratic_loss_noalloc")
+
+
+def lsgd_bgemm_bf16(desc: BgemmDesc, stream: int = 0) -> None:
+    _check(lib().lsgd_bgemm_bf16(C.byref(desc), stream or None), "lsgd_bgemm_bf16")
 
 
 def mlp_param_offsets(dims: Sequence[int]):

@@ -65,7 +65,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             if verbose and log:
                 print(log)
     if jobs or force or _stale(LIB, objs):
-        run([nvcc, "-shared", "-o", LIB] + objs + ["-lcudart", "-lcuda"])
+        run([nvcc, "-shared", "-o", LIB] + objs + ["-lcudart"])
     return LIB
 
 

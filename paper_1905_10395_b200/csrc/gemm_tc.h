@@ -1,0 +1,38 @@
+// Batched bf16 tensor-core matrix product: launcher interface (see gemm_tc.cu).
+#pragma once
+#include <cuda.h>
+
+#include "internal.h"
+
+namespace lsgd {
+
+enum GemmEpilogue : int {
+  GEMM_EPI_F32 = 0,             // C fp32 = acc
+  GEMM_EPI_BIAS_RELU_BF16 = 1,  // C bf16 = relu(acc + bias[n])
+  GEMM_EPI_MASK_BF16 = 2,       // C bf16 = mask[m][n] > 0 ? acc : 0
+  GEMM_EPI_BF16 = 3,            // C bf16 = acc
+};
+
+struct GemmShape {
+  int M, N, K, batch;
+  int a_mn, b_mn;               // 1: the M (resp. N) index is contiguous in memory, 0: the K index is
+  int a_batched, b_batched;     // 0: every batch entry reads batch 0 of that operand
+  int epilogue;
+  int vec_ok;                   // set by the launcher: C rows allow 16-byte stores
+  void* c;                      // [batch][M][ldc]
+  int64_t ldc, stride_c;        // in elements of C
+  const float* bias;            // [batch][N] fp32 (stride_bias apart)
+  int64_t stride_bias;
+  const void* mask;             // bf16 [batch][M][ld_mask]
+  int64_t ld_mask, stride_mask;
+  uint32_t* status;             // device status word (bounded-wait failures)
+};
+
+// 3-D tensor map {inner (contiguous), outer, batch} of bf16 with a 64 x 64 x 1 box and 128-byte swizzle.
+// K-major operand: inner = K, outer = M or N.  MN-major operand: inner = M or N, outer = K.
+bool make_operand_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t pitch_elems,
+                      int64_t batch, int64_t batch_stride_elems);
+
+cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmShape& p, cudaStream_t s);
+
+}  // namespace lsgd

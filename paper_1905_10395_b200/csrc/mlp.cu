@@ -1,16 +1,394 @@
-// MLP population objective: host orchestration.
+// MLP population objective: a population of P three-layer ReLU classifiers trained with mean softmax
+// cross-entropy, each worker on its own minibatch (the paper's deep-network setting, Section 4: every
+// worker runs its own SGD on its own batches; here the networks are small dense MLPs).
+//
+// Parameter row = [W1 | b1 | W2 | b2 | W3 | b3], W_l stored [n_out][n_in].  All matrix products take
+// bf16 operands and accumulate in fp32:
+//   forward   H1 = relu(X W1^T + b1), H2 = relu(H1 W2^T + b2)            tensor cores (gemm_tc.cu)
+//   head      Z = H2 W3^T + b3, loss, dZ, dW3, db3, dH2, db2             CUDA cores (n_classes is tiny)
+//   backward  dH1 = (dH2 W2) * [H1 > 0], dW2 = dH2^T H1, dW1 = dH1^T X   tensor cores
+// Stored activations and back-propagated deltas are rounded to bf16 once, when they are written.
+// The bf16 copy of the weights is refreshed by the update kernel itself when it writes x.
+#include <cuda_bf16.h>
+
+#include <cmath>
+#include <new>
+
+#include "gemm_tc.h"
 #include "mlp.h"
 
 namespace lsgd {
+namespace {
 
-static inline int64_t up32(int64_t n) { return (n + 31) / 32 * 32; }
+constexpr int kMaxClasses = 16;
 
-lsgd_status mlp_validate(const lsgd_config&, const lsgd_mlp_desc&) { return LSGD_ERR_UNSUPPORTED; }
-lsgd_status mlp_create(lsgd_ctx*) { return LSGD_ERR_UNSUPPORTED; }
-lsgd_status mlp_grad(lsgd_ctx*, const int32_t*) { return LSGD_ERR_UNSUPPORTED; }
-lsgd_status mlp_heldout_loss(lsgd_ctx*, float*) { return LSGD_ERR_UNSUPPORTED; }
-uint16_t* mlp_weight_shadow(lsgd_ctx*) { return nullptr; }
-void mlp_destroy(lsgd_ctx*) {}
+inline int64_t up32(int64_t n) { return (n + 31) / 32 * 32; }
+inline size_t up1k(size_t n) { return (n + 1023) & ~size_t(1023); }
+
+struct Layout {
+  int64_t w[3], b[3], d;
+};
+Layout param_layout(const int32_t* dims) {
+  Layout L{};
+  int64_t off = 0;
+  for (int l = 0; l < 3; ++l) {
+    L.w[l] = off;
+    off = up32(off + (int64_t)dims[l] * dims[l + 1]);
+    L.b[l] = off;
+    off = up32(off + dims[l + 1]);
+  }
+  L.d = off;
+  return L;
+}
+
+struct Scratch {
+  size_t wb, xb, h1, h2, dh2, dh1, dz, loss_b, xh, hh1, hh2, loss_h, total;
+};
+Scratch scratch_layout(const int32_t* dims, int64_t ld, int32_t P, int32_t B, int32_t nH) {
+  Scratch s{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += up1k(bytes); return o; };
+  s.wb = take((size_t)P * ld * 2);
+  s.xb = take((size_t)P * B * dims[0] * 2);
+  s.h1 = take((size_t)P * B * dims[1] * 2);
+  s.h2 = take((size_t)P * B * dims[2] * 2);
+  s.dh2 = take((size_t)P * B * dims[2] * 2);
+  s.dh1 = take((size_t)P * B * dims[1] * 2);
+  s.dz = take((size_t)P * B * dims[3] * 4);
+  s.loss_b = take((size_t)P * B * 4);
+  s.xh = take((size_t)nH * dims[0] * 2);
+  s.hh1 = take((size_t)P * nH * dims[1] * 2);
+  s.hh2 = take((size_t)P * nH * dims[2] * 2);
+  s.loss_h = take((size_t)P * nH * 4);
+  s.total = off;
+  return s;
+}
+
+struct MlpState {
+  Layout L;
+  Scratch S;
+  int32_t dims[4];
+  int32_t B, nH, P;
+  int64_t ld;
+  __nv_bfloat16 *wb, *xb, *h1, *h2, *dh2, *dh1, *xh, *hh1, *hh2;
+  float *dz, *loss_b, *loss_h;
+  CUtensorMap m_xb, m_w1, m_w2, m_h1, m_dh2, m_dh1, m_xh, m_hh1;
+};
+
+// ------------------------------------------------------------------------------------ small kernels
+__global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t n) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+// xb[row][:] = bf16(pool[idx[row]][:])
+__global__ void gather_rows_kernel(const float* __restrict__ pool, const int32_t* __restrict__ idx, __nv_bfloat16* __restrict__ xb,
+                                   int32_t rows_total, int32_t d0, int32_t pool_rows, uint32_t* status) {
+  const int row = blockIdx.x;
+  if (row >= rows_total) return;
+  const int src = idx[row];
+  if (src < 0 || src >= pool_rows) {
+    if (threadIdx.x == 0) atomicOr(status, FLAG_BAD_INDEX);
+    for (int k = threadIdx.x; k < d0; k += blockDim.x) xb[(int64_t)row * d0 + k] = __float2bfloat16_rn(0.f);
+    return;
+  }
+  const float* s = pool + (int64_t)src * d0;
+  for (int k = threadIdx.x; k < d0; k += blockDim.x) xb[(int64_t)row * d0 + k] = __float2bfloat16_rn(s[k]);
+}
+
+// One warp per sample: logits, softmax cross-entropy, and (training) dZ = (p - onehot) / n rounded to bf16.
+__global__ void __launch_bounds__(256)
+head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ x,
+                    const int32_t* __restrict__ labels, const int32_t* __restrict__ label_idx, float* __restrict__ dz,
+                    float* __restrict__ loss_b, int32_t n, int32_t d2, int32_t C, int64_t ld, int64_t w3_off, int64_t b3_off,
+                    int32_t label_rows, uint32_t* status) {
+  const int i = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x * (blockDim.x >> 5) + warp;
+  if (b >= n) return;
+  const __nv_bfloat16* h = h2 + ((int64_t)i * n + b) * d2;
+  const __nv_bfloat16* w3 = wb + (int64_t)i * ld + w3_off;
+  float acc[kMaxClasses];
+#pragma unroll
+  for (int c = 0; c < kMaxClasses; ++c) acc[c] = 0.f;
+  for (int k = lane; k < d2; k += 32) {
+    const float hv = __bfloat162float(h[k]);
+#pragma unroll
+    for (int c = 0; c < kMaxClasses; ++c)
+      if (c < C) acc[c] = fmaf(hv, __bfloat162float(w3[(int64_t)c * d2 + k]), acc[c]);
+  }
+#pragma unroll
+  for (int c = 0; c < kMaxClasses; ++c)
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xFFFFFFFFu, acc[c], o);
+  if (lane == 0) {
+    int y = label_idx ? label_idx[(int64_t)i * n + b] : b;   // training: pool row of this sample
+    if (y < 0 || y >= label_rows) {
+      atomicOr(status, FLAG_BAD_INDEX);
+      y = 0;
+    }
+    int cls = labels[y];
+    if (cls < 0 || cls >= C) {
+      atomicOr(status, FLAG_BAD_INDEX);
+      cls = 0;
+    }
+    const float* b3 = x + (int64_t)i * ld + b3_off;
+    float zmax = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < kMaxClasses; ++c)
+      if (c < C) {
+        acc[c] += b3[c];
+        zmax = fmaxf(zmax, acc[c]);
+      }
+    float sum = 0.f, zy = 0.f;
+#pragma unroll
+    for (int c = 0; c < kMaxClasses; ++c)
+      if (c < C) {
+        sum += expf(acc[c] - zmax);
+        if (c == cls) zy = acc[c];
+      }
+    const float lse = zmax + logf(sum);
+    loss_b[(int64_t)i * n + b] = lse - zy;
+    if (dz) {
+      const float inv_n = 1.f / (float)n;
+#pragma unroll
+      for (int c = 0; c < kMaxClasses; ++c)
+        if (c < C) {
+          const float pc = expf(acc[c] - lse);
+          const float v = (pc - (c == cls ? 1.f : 0.f)) * inv_n;
+          dz[((int64_t)i * n + b) * C + c] = __bfloat162float(__float2bfloat16_rn(v));
+        }
+    }
+  }
+}
+
+// One thread per hidden unit k of the last hidden layer: dW3[:, k], dH2[:, k] (masked, rounded), db2[k];
+// block 0 of each worker also writes db3.
+__global__ void __launch_bounds__(128)
+head_backward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ dz,
+                     __nv_bfloat16* __restrict__ dh2, float* __restrict__ g, int32_t n, int32_t d2, int32_t C, int64_t ld,
+                     int64_t w3_off, int64_t b3_off, int64_t b2_off) {
+  extern __shared__ float s_dz[];   // [n][C]
+  const int i = blockIdx.y;
+  const float* dzi = dz + (int64_t)i * n * C;
+  for (int t = threadIdx.x; t < n * C; t += blockDim.x) s_dz[t] = dzi[t];
+  __syncthreads();
+  float* gi = g + (int64_t)i * ld;
+  if (blockIdx.x == 0 && threadIdx.x < C) {
+    float s = 0.f;
+    for (int b = 0; b < n; ++b) s += s_dz[b * C + threadIdx.x];
+    gi[b3_off + threadIdx.x] = s;
+  }
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= d2) return;
+  const __nv_bfloat16* w3 = wb + (int64_t)i * ld + w3_off;
+  float w[kMaxClasses], aw[kMaxClasses];
+#pragma unroll
+  for (int c = 0; c < kMaxClasses; ++c) {
+    w[c] = c < C ? __bfloat162float(w3[(int64_t)c * d2 + k]) : 0.f;
+    aw[c] = 0.f;
+  }
+  float ab = 0.f;
+  const __nv_bfloat16* hcol = h2 + (int64_t)i * n * d2 + k;
+  __nv_bfloat16* dcol = dh2 + (int64_t)i * n * d2 + k;
+  for (int b = 0; b < n; ++b) {
+    const float hv = __bfloat162float(hcol[(int64_t)b * d2]);
+    float dh = 0.f;
+#pragma unroll
+    for (int c = 0; c < kMaxClasses; ++c)
+      if (c < C) {
+        const float z = s_dz[b * C + c];
+        aw[c] = fmaf(z, hv, aw[c]);
+        dh = fmaf(z, w[c], dh);
+      }
+    const __nv_bfloat16 r = __float2bfloat16_rn(hv > 0.f ? dh : 0.f);
+    dcol[(int64_t)b * d2] = r;
+    ab += __bfloat162float(r);
+  }
+#pragma unroll
+  for (int c = 0; c < kMaxClasses; ++c)
+    if (c < C) gi[w3_off + (int64_t)c * d2 + k] = aw[c];
+  gi[b2_off + k] = ab;
+}
+
+// db[k] = sum_b delta[b][k] for a stored (bf16) delta matrix.
+__global__ void __launch_bounds__(128)
+column_sum_kernel(const __nv_bfloat16* __restrict__ delta, float* __restrict__ g, int32_t n, int32_t dcols, int64_t ld, int64_t off) {
+  const int i = blockIdx.y;
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= dcols) return;
+  const __nv_bfloat16* col = delta + (int64_t)i * n * dcols + k;
+  float s = 0.f;
+  for (int b = 0; b < n; ++b) s += __bfloat162float(col[(int64_t)b * dcols]);
+  g[(int64_t)i * ld + off + k] = s;
+}
+
+// out[i] = mean_b v[i][b], summed in a fixed order by one warp per worker.
+__global__ void __launch_bounds__(32) row_mean_kernel(const float* __restrict__ v, float* __restrict__ out, int32_t n) {
+  const int i = blockIdx.x, lane = threadIdx.x;
+  double acc = 0.0;
+  for (int b = lane; b < n; b += 32) acc += (double)v[(int64_t)i * n + b];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+  if (lane == 0) out[i] = (float)(acc / (double)n);
+}
+
+MlpState* state(lsgd_ctx* h) { return static_cast<MlpState*>(h->mlp_state); }
+
+GemmShape shape(int M, int N, int K, int batch, int a_mn, int b_mn, int a_batched, int epi, void* c, int64_t ldc,
+                int64_t stride_c, uint32_t* status) {
+  GemmShape g{};
+  g.M = M; g.N = N; g.K = K; g.batch = batch;
+  g.a_mn = a_mn; g.b_mn = b_mn; g.a_batched = a_batched; g.b_batched = 1;
+  g.epilogue = epi; g.c = c; g.ldc = ldc; g.stride_c = stride_c; g.status = status;
+  return g;
+}
+
+lsgd_status forward_hidden(lsgd_ctx* h, const CUtensorMap& m_in, int a_batched, int n, __nv_bfloat16* o1, const CUtensorMap& m_o1,
+                           __nv_bfloat16* o2) {
+  MlpState* st = state(h);
+  const lsgd_config& c = h->cfg;
+  const int32_t* d = st->dims;
+  GemmShape g1 = shape(n, d[1], d[0], st->P, 0, 0, a_batched, GEMM_EPI_BIAS_RELU_BF16, o1, d[1], (int64_t)n * d[1], h->d_status);
+  g1.bias = c.x + st->L.b[0];
+  g1.stride_bias = st->ld;
+  if (launch_bgemm(m_in, st->m_w1, g1, h->stream) != cudaSuccess) return LSGD_ERR_CUDA;
+  GemmShape g2 = shape(n, d[2], d[1], st->P, 0, 0, 1, GEMM_EPI_BIAS_RELU_BF16, o2, d[2], (int64_t)n * d[2], h->d_status);
+  g2.bias = c.x + st->L.b[1];
+  g2.stride_bias = st->ld;
+  if (launch_bgemm(m_o1, st->m_w2, g2, h->stream) != cudaSuccess) return LSGD_ERR_CUDA;
+  return LSGD_OK;
+}
+
+}  // namespace
+
+lsgd_status mlp_validate(const lsgd_config& c, const lsgd_mlp_desc& m) {
+  for (int l = 0; l < 4; ++l)
+    if (m.dims[l] < 1) return LSGD_ERR_INVALID_ARG;
+  if (m.batch < 1 || m.pool < 1 || m.n_heldout < 1) return LSGD_ERR_INVALID_ARG;
+  if (!m.pool_x || !m.pool_y || !m.held_x || !m.held_y || !m.scratch) return LSGD_ERR_INVALID_ARG;
+  // TMA rows must be 16-byte multiples (8 bf16); the head kernels keep the class scores in registers
+  if (m.dims[0] % 8 || m.dims[1] % 8 || m.dims[2] % 8 || m.dims[3] > kMaxClasses) return LSGD_ERR_UNSUPPORTED;
+  if (m.batch % 8 || m.n_heldout % 8 || m.batch > 1024) return LSGD_ERR_UNSUPPORTED;
+  const Layout L = param_layout(m.dims);
+  if (L.d != c.d || c.ld != c.d) return LSGD_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(m.scratch) & 1023u) return LSGD_ERR_ALIGNMENT;
+  if (m.scratch_bytes < lsgd_mlp_scratch_bytes(m.dims, c.P, m.batch, m.n_heldout)) return LSGD_ERR_INVALID_ARG;
+  return LSGD_OK;
+}
+
+lsgd_status mlp_create(lsgd_ctx* h) {
+  const lsgd_config& c = h->cfg;
+  const lsgd_mlp_desc& m = h->mlp;
+  MlpState* st = new (std::nothrow) MlpState();
+  if (!st) return LSGD_ERR_INVALID_ARG;
+  h->mlp_state = st;
+  for (int l = 0; l < 4; ++l) st->dims[l] = m.dims[l];
+  st->L = param_layout(m.dims);
+  st->B = m.batch;
+  st->nH = m.n_heldout;
+  st->P = c.P;
+  st->ld = c.ld;
+  st->S = scratch_layout(m.dims, c.ld, c.P, m.batch, m.n_heldout);
+  char* base = static_cast<char*>(m.scratch);
+  st->wb = reinterpret_cast<__nv_bfloat16*>(base + st->S.wb);
+  st->xb = reinterpret_cast<__nv_bfloat16*>(base + st->S.xb);
+  st->h1 = reinterpret_cast<__nv_bfloat16*>(base + st->S.h1);
+  st->h2 = reinterpret_cast<__nv_bfloat16*>(base + st->S.h2);
+  st->dh2 = reinterpret_cast<__nv_bfloat16*>(base + st->S.dh2);
+  st->dh1 = reinterpret_cast<__nv_bfloat16*>(base + st->S.dh1);
+  st->dz = reinterpret_cast<float*>(base + st->S.dz);
+  st->loss_b = reinterpret_cast<float*>(base + st->S.loss_b);
+  st->xh = reinterpret_cast<__nv_bfloat16*>(base + st->S.xh);
+  st->hh1 = reinterpret_cast<__nv_bfloat16*>(base + st->S.hh1);
+  st->hh2 = reinterpret_cast<__nv_bfloat16*>(base + st->S.hh2);
+  st->loss_h = reinterpret_cast<float*>(base + st->S.loss_h);
+
+  const int32_t* d = st->dims;
+  const int64_t B = st->B, nH = st->nH, P = st->P, ld = st->ld;
+  bool ok = true;
+  ok = ok && make_operand_map(&st->m_xb, st->xb, d[0], B, d[0], P, B * d[0]);
+  ok = ok && make_operand_map(&st->m_w1, st->wb + st->L.w[0], d[0], d[1], d[0], P, ld);
+  ok = ok && make_operand_map(&st->m_w2, st->wb + st->L.w[1], d[1], d[2], d[1], P, ld);
+  ok = ok && make_operand_map(&st->m_h1, st->h1, d[1], B, d[1], P, B * d[1]);
+  ok = ok && make_operand_map(&st->m_dh2, st->dh2, d[2], B, d[2], P, B * d[2]);
+  ok = ok && make_operand_map(&st->m_dh1, st->dh1, d[1], B, d[1], P, B * d[1]);
+  ok = ok && make_operand_map(&st->m_xh, st->xh, d[0], nH, d[0], 1, 0);
+  ok = ok && make_operand_map(&st->m_hh1, st->hh1, d[1], nH, d[1], P, nH * d[1]);
+  if (!ok) return LSGD_ERR_CUDA;
+
+  // bf16 copies of the weights and of the held-out inputs; gradient padding cleared once
+  f32_to_bf16_kernel<<<148 * 8, 256, 0, h->stream>>>(c.x, st->wb, (int64_t)P * ld);
+  f32_to_bf16_kernel<<<148 * 2, 256, 0, h->stream>>>(m.held_x, st->xh, (int64_t)nH * d[0]);
+  if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
+  if (cudaMemsetAsync(c.g, 0, sizeof(float) * (size_t)P * (size_t)ld, h->stream) != cudaSuccess) return LSGD_ERR_CUDA;
+  return LSGD_OK;
+}
+
+lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx) {
+  MlpState* st = state(h);
+  const lsgd_config& c = h->cfg;
+  const lsgd_mlp_desc& m = h->mlp;
+  const int32_t* d = st->dims;
+  const int B = st->B, P = st->P;
+  const int64_t ld = st->ld;
+  cudaStream_t s = h->stream;
+
+  gather_rows_kernel<<<P * B, 128, 0, s>>>(m.pool_x, batch_idx, st->xb, P * B, d[0], m.pool, h->d_status);
+  if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
+  lsgd_status fs = forward_hidden(h, st->m_xb, 1, B, st->h1, st->m_h1, st->h2);
+  if (fs != LSGD_OK) return fs;
+
+  head_forward_kernel<<<dim3((B + 7) / 8, P), 256, 0, s>>>(st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2],
+                                                          d[3], ld, st->L.w[2], st->L.b[2], m.pool, h->d_status);
+  head_backward_kernel<<<dim3((d[2] + 127) / 128, P), 128, sizeof(float) * B * d[3], s>>>(
+      st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]);
+  if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
+
+  // dH1 = (dH2 . W2) masked by H1 > 0        [B x d1] = [B x d2] . [d2 x d1]
+  GemmShape gd = shape(B, d[1], d[2], P, 0, 1, 1, GEMM_EPI_MASK_BF16, st->dh1, d[1], (int64_t)B * d[1], h->d_status);
+  gd.mask = st->h1;
+  gd.ld_mask = d[1];
+  gd.stride_mask = (int64_t)B * d[1];
+  if (launch_bgemm(st->m_dh2, st->m_w2, gd, s) != cudaSuccess) return LSGD_ERR_CUDA;
+  // dW2 = dH2^T . H1                          [d2 x d1], contraction over the batch
+  GemmShape g2 = shape(d[2], d[1], B, P, 1, 1, 1, GEMM_EPI_F32, c.g + st->L.w[1], d[1], ld, h->d_status);
+  if (launch_bgemm(st->m_dh2, st->m_h1, g2, s) != cudaSuccess) return LSGD_ERR_CUDA;
+  column_sum_kernel<<<dim3((d[1] + 127) / 128, P), 128, 0, s>>>(st->dh1, c.g, B, d[1], ld, st->L.b[0]);
+  if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
+  // dW1 = dH1^T . X                           [d1 x d0]
+  GemmShape g1 = shape(d[1], d[0], B, P, 1, 1, 1, GEMM_EPI_F32, c.g + st->L.w[0], d[0], ld, h->d_status);
+  if (launch_bgemm(st->m_dh1, st->m_xb, g1, s) != cudaSuccess) return LSGD_ERR_CUDA;
+  return LSGD_OK;
+}
+
+lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss) {
+  MlpState* st = state(h);
+  const lsgd_config& c = h->cfg;
+  const lsgd_mlp_desc& m = h->mlp;
+  const int32_t* d = st->dims;
+  lsgd_status fs = forward_hidden(h, st->m_xh, 0, st->nH, st->hh1, st->m_hh1, st->hh2);
+  if (fs != LSGD_OK) return fs;
+  head_forward_kernel<<<dim3((st->nH + 7) / 8, st->P), 256, 0, h->stream>>>(st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr,
+                                                                          st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2],
+                                                                          st->L.b[2], st->nH, h->d_status);
+  row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_h, loss, st->nH);
+  return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
+}
+
+lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss) {
+  MlpState* st = state(h);
+  if (!st) return LSGD_ERR_STATE;
+  row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_b, loss, st->B);
+  return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
+}
+
+uint16_t* mlp_weight_shadow(lsgd_ctx* h) { return h->mlp_state ? reinterpret_cast<uint16_t*>(state(h)->wb) : nullptr; }
+
+void mlp_destroy(lsgd_ctx* h) {
+  delete state(h);
+  h->mlp_state = nullptr;
+}
 
 }  // namespace lsgd
 
@@ -18,18 +396,51 @@ extern "C" {
 
 lsgd_status lsgd_mlp_param_offsets(const int32_t* dims, int64_t* w_off, int64_t* b_off, int64_t* d_out) {
   if (!dims || !w_off || !b_off || !d_out) return LSGD_ERR_INVALID_ARG;
-  int64_t off = 0;
-  for (int l = 0; l < LSGD_MLP_MAX_LAYERS; ++l) {
-    if (dims[l] < 1 || dims[l + 1] < 1) return LSGD_ERR_INVALID_ARG;
-    w_off[l] = off;
-    off = lsgd::up32(off + (int64_t)dims[l] * dims[l + 1]);
-    b_off[l] = off;
-    off = lsgd::up32(off + dims[l + 1]);
+  for (int l = 0; l < 4; ++l)
+    if (dims[l] < 1) return LSGD_ERR_INVALID_ARG;
+  const lsgd::Layout L = lsgd::param_layout(dims);
+  for (int l = 0; l < 3; ++l) {
+    w_off[l] = L.w[l];
+    b_off[l] = L.b[l];
   }
-  *d_out = off;
+  *d_out = L.d;
   return LSGD_OK;
 }
 
-uint64_t lsgd_mlp_scratch_bytes(const int32_t*, int32_t, int32_t, int32_t) { return 0; }
+uint64_t lsgd_mlp_scratch_bytes(const int32_t* dims, int32_t P, int32_t batch, int32_t n_heldout) {
+  if (!dims || P < 1 || batch < 1 || n_heldout < 1) return 0;
+  for (int l = 0; l < 4; ++l)
+    if (dims[l] < 1) return 0;
+  const lsgd::Layout L = lsgd::param_layout(dims);
+  return lsgd::scratch_layout(dims, L.d, P, batch, n_heldout).total;
+}
+
+lsgd_status lsgd_bgemm_bf16(const lsgd_bgemm_desc* g, void* stream) {
+  using namespace lsgd;
+  if (!g || !g->a || !g->b || !g->c) return LSGD_ERR_INVALID_ARG;
+  if (g->M < 1 || g->N < 1 || g->K < 1 || g->batch < 1 || g->epilogue < 0 || g->epilogue > 3) return LSGD_ERR_INVALID_ARG;
+  if (g->epilogue == GEMM_EPI_BIAS_RELU_BF16 && !g->bias) return LSGD_ERR_INVALID_ARG;
+  if (g->epilogue == GEMM_EPI_MASK_BF16 && !g->mask) return LSGD_ERR_INVALID_ARG;
+  static uint32_t* status = nullptr;   // status word of the stand-alone entry point, allocated on first use
+  if (!status) {
+    if (cudaMalloc(&status, sizeof(uint32_t)) != cudaSuccess) return LSGD_ERR_CUDA;
+    cudaMemset(status, 0, sizeof(uint32_t));
+  }
+  CUtensorMap ma, mb;
+  const int64_t a_inner = g->a_mn_major ? g->M : g->K, a_outer = g->a_mn_major ? g->K : g->M;
+  const int64_t b_inner = g->b_mn_major ? g->N : g->K, b_outer = g->b_mn_major ? g->K : g->N;
+  if (!make_operand_map(&ma, g->a, a_inner, a_outer, g->lda, g->stride_a ? g->batch : 1, g->stride_a)) return LSGD_ERR_ALIGNMENT;
+  if (!make_operand_map(&mb, g->b, b_inner, b_outer, g->ldb, g->stride_b ? g->batch : 1, g->stride_b)) return LSGD_ERR_ALIGNMENT;
+  GemmShape p{};
+  p.M = g->M; p.N = g->N; p.K = g->K; p.batch = g->batch;
+  p.a_mn = g->a_mn_major ? 1 : 0; p.b_mn = g->b_mn_major ? 1 : 0;
+  p.a_batched = g->stride_a ? 1 : 0; p.b_batched = g->stride_b ? 1 : 0;
+  p.epilogue = g->epilogue; p.c = g->c; p.ldc = g->ldc; p.stride_c = g->stride_c;
+  p.bias = g->bias; p.stride_bias = g->stride_bias;
+  p.mask = g->mask; p.ld_mask = g->ld_mask; p.stride_mask = g->stride_mask;
+  p.status = status;
+  if (launch_bgemm(ma, mb, p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return LSGD_ERR_CUDA;
+  return LSGD_OK;
+}
 
 }  // extern "C"

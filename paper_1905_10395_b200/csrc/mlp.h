@@ -8,6 +8,7 @@ lsgd_status mlp_validate(const lsgd_config& c, const lsgd_mlp_desc& m);
 lsgd_status mlp_create(lsgd_ctx* h);
 lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx);
 lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss);
+lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss);   // mean minibatch loss of the last lsgd_grad
 uint16_t* mlp_weight_shadow(lsgd_ctx* h);
 void mlp_destroy(lsgd_ctx* h);
 
