@@ -165,11 +165,19 @@ LSGD_API lsgd_status lsgd_get_leaders(lsgd_handle h, int32_t* local_leaders /* H
                              int32_t* global_leader /* HOST int32[1] */);
 LSGD_API lsgd_status lsgd_get_loss(lsgd_handle h, float* loss /* HOST float[P]: losses of the last election */);
 LSGD_API lsgd_status lsgd_get_step(lsgd_handle h, int64_t* t);
+/* Mean minibatch loss of every worker from the last lsgd_grad (MLP objective only; LSGD_ERR_UNSUPPORTED
+ * otherwise).  The paper's deep-network runs elect on a running mean of such training losses
+ * (Section 4.1); here it is reported for monitoring and parity checks.                             */
+LSGD_API lsgd_status lsgd_get_train_loss(lsgd_handle h, float* loss /* HOST float[P] */);
 /* Times each worker has been global / local leader so far (the leader statistics of Section 4.2). */
 LSGD_API lsgd_status lsgd_get_leader_counts(lsgd_handle h, int32_t* global_counts /* HOST int32[P] */,
                                    int32_t* local_counts /* HOST int32[P] */);
 /* Reads and clears the device status word; LSGD_ERR_DEVICE_FLAG if any kernel has set it.        */
 LSGD_API lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out /* HOST, may be NULL */);
+/* Call after overwriting x from outside (restoring a checkpoint, re-seeding a worker): re-derives
+ * the library's internal copies of the parameters (the bf16 weight copy of the MLP objective) on the
+ * stream.  The step counter and the leaders are kept.                                               */
+LSGD_API lsgd_status lsgd_sync_parameters(lsgd_handle h);
 /* Replaces eta (learning-rate schedules are the caller's, Section 4).                            */
 LSGD_API lsgd_status lsgd_set_eta(lsgd_handle h, float eta);
 

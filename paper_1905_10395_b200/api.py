@@ -74,6 +74,10 @@ def lib() -> C.CDLL:
         L.lsgd_destroy.argtypes = [H]
         L.lsgd_get_leaders.argtypes = [H, C.c_void_p, C.c_void_p]
         L.lsgd_get_loss.argtypes = [H, C.c_void_p]
+        L.lsgd_get_train_loss.argtypes = [H, C.c_void_p]
+        L.lsgd_get_train_loss.restype = C.c_int
+        L.lsgd_sync_parameters.argtypes = [H]
+        L.lsgd_sync_parameters.restype = C.c_int
         L.lsgd_get_step.argtypes = [H, C.POINTER(C.c_int64)]
         L.lsgd_get_leader_counts.argtypes = [H, C.c_void_p, C.c_void_p]
         L.lsgd_check_device.argtypes = [H, C.POINTER(C.c_uint32)]
@@ -210,6 +214,14 @@ class Lsgd:
         out = np.empty(self.P, dtype=np.float32)
         _check(lib().lsgd_get_loss(self.h, out.ctypes.data), "lsgd_get_loss")
         return out
+
+    def train_loss(self):
+        out = np.empty(self.P, dtype=np.float32)
+        _check(lib().lsgd_get_train_loss(self.h, out.ctypes.data), "lsgd_get_train_loss")
+        return out
+
+    def sync_parameters(self):
+        _check(lib().lsgd_sync_parameters(self.h), "lsgd_sync_parameters")
 
     def t(self) -> int:
         v = C.c_int64()

@@ -317,6 +317,18 @@ lsgd_status lsgd_get_loss(lsgd_handle h, float* loss) {
   return LSGD_OK;
 }
 
+lsgd_status lsgd_get_train_loss(lsgd_handle h, float* loss) {
+  if (!h || !loss) return LSGD_ERR_INVALID_ARG;
+  if (h->cfg.objective != LSGD_OBJ_MLP) return LSGD_ERR_UNSUPPORTED;
+  // the reduction-partials area (at least P doubles, unused by this objective) receives the P means
+  float* tmp = reinterpret_cast<float*>(h->d_partials);
+  lsgd_status st = mlp_train_loss(h, tmp);
+  if (st != LSGD_OK) return st;
+  LSGD_CUDA(cudaStreamSynchronize(h->stream));
+  LSGD_CUDA(cudaMemcpy(loss, tmp, sizeof(float) * h->cfg.P, cudaMemcpyDeviceToHost));
+  return LSGD_OK;
+}
+
 lsgd_status lsgd_get_step(lsgd_handle h, int64_t* t) {
   if (!h || !t) return LSGD_ERR_INVALID_ARG;
   *t = h->t;
@@ -339,6 +351,12 @@ lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out) {
   if (f) LSGD_CUDA(cudaMemset(h->d_status, 0, sizeof(f)));
   if (flag_out) *flag_out = f;
   return f ? LSGD_ERR_DEVICE_FLAG : LSGD_OK;
+}
+
+lsgd_status lsgd_sync_parameters(lsgd_handle h) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  if (h->cfg.objective == LSGD_OBJ_MLP) return mlp_refresh_shadow(h);
+  return LSGD_OK;
 }
 
 lsgd_status lsgd_set_eta(lsgd_handle h, float eta) {

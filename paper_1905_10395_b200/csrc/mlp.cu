@@ -383,6 +383,13 @@ lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss) {
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
 }
 
+lsgd_status mlp_refresh_shadow(lsgd_ctx* h) {
+  MlpState* st = state(h);
+  if (!st) return LSGD_ERR_STATE;
+  f32_to_bf16_kernel<<<148 * 8, 256, 0, h->stream>>>(h->cfg.x, st->wb, (int64_t)st->P * st->ld);
+  return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
+}
+
 uint16_t* mlp_weight_shadow(lsgd_ctx* h) { return h->mlp_state ? reinterpret_cast<uint16_t*>(state(h)->wb) : nullptr; }
 
 void mlp_destroy(lsgd_ctx* h) {

@@ -9,6 +9,7 @@ lsgd_status mlp_create(lsgd_ctx* h);
 lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx);
 lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss);
 lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss);   // mean minibatch loss of the last lsgd_grad
+lsgd_status mlp_refresh_shadow(lsgd_ctx* h);             // bf16 copy of the weights <- x
 uint16_t* mlp_weight_shadow(lsgd_ctx* h);
 void mlp_destroy(lsgd_ctx* h);
 

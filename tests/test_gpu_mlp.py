@@ -1,0 +1,153 @@
+"""GPU parity of the MLP population objective (bf16 tensor-core products, fp32 accumulation) against
+the oracle's bf16-emulation mode.  Tolerance from the workload statement: 2e-2 relative on parameters
+and on losses.  Leaders must agree unless the oracle's own margin is a near-tie (< 2e-2 relative), in
+which case the run is repeated with the oracle's loss vectors forced into the election."""
+import numpy as np
+import pytest
+
+from oracle import lsgd_oracle as orc
+from paper_1905_10395_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2
+LOSS_FLOOR = 1.0     # cross-entropy has a natural O(1) scale (chance level ln 10 = 2.3)
+
+
+def loss_close(got, ref):
+    return bool(np.all(np.abs(got.astype(np.float64) - ref) <= TOL * np.maximum(np.abs(ref), LOSS_FLOOR)))
+
+
+def _oracle(w):
+    A = w.arrays
+    segs, _ = inputs.mlp_layout(w.meta["dims"])
+    obj = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="bf16emu")
+    return orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
+
+
+def _run_pair(w, steps):
+    import torch
+    from paper_1905_10395_b200.runner import Population
+    o = _oracle(w)
+    train_ref = []
+    for _ in range(steps):
+        o.step()
+        train_ref.append(o.obj.last_train_loss.copy())
+    pop = Population(w)
+    train_gpu = []
+    for _ in range(steps):
+        pop.step(record=True)
+        train_gpu.append(pop.lsgd.train_loss())
+    same = all(hg["gl"] == ho["gl"] and np.array_equal(hg["ll"], ho["ll"]) for hg, ho in zip(pop.history, o.history))
+    forced = False
+    if not same:
+        for hg, ho in zip(pop.history, o.history):
+            if hg["gl"] != ho["gl"] or not np.array_equal(hg["ll"], ho["ll"]):
+                srt = np.sort(ho["loss"])
+                assert (srt[1] - srt[0]) <= TOL * abs(srt[0]), "leaders differ without a near-tie"
+                break
+        pop.close()
+        pop = Population(w)
+        train_gpu = []
+        for t in range(steps):
+            fl = torch.from_numpy(o.history[t // w.tau]["loss"]).cuda() if t % w.tau == 0 else None
+            pop.step(forced_loss=fl, record=True)
+            train_gpu.append(pop.lsgd.train_loss())
+        forced = True
+    return pop, o, train_gpu, train_ref, forced
+
+
+def _check(pop, o, w, train_gpu, train_ref, forced):
+    x = pop.x_host().astype(np.float64)
+    ref = o.x.astype(np.float64)
+    scale = np.abs(ref).max()
+    assert np.abs(x - ref).max() <= TOL * scale
+    # the discriminating number: error of the parameter change, norm-wise per worker
+    dx, dref = x - w.x0, ref - w.x0
+    for i in range(w.P):
+        assert np.linalg.norm(dx[i] - dref[i]) <= TOL * np.linalg.norm(dref[i]), i
+    # elementwise: all but a few entries (a ReLU whose pre-activation is within accumulation error of
+    # zero switches a whole sample's contribution on or off) within TOL of the largest change
+    assert np.mean(np.abs(dx - dref) > TOL * np.abs(dref).max()) <= 1e-4
+    for tg, tr in zip(train_gpu, train_ref):
+        assert loss_close(tg, tr)
+    if not forced:
+        for hg, ho in zip(pop.history, o.history):
+            assert loss_close(hg["loss"], ho["loss"])
+    assert np.all(x[:, :][:, _pad_mask(w)] == 0)
+    assert pop.lsgd.check_device() == 0
+
+
+def _pad_mask(w):
+    segs, d = inputs.mlp_layout(w.meta["dims"])
+    m = np.ones(d, dtype=bool)
+    for s in segs:
+        m[s["w"]:s["w"] + s["n_in"] * s["n_out"]] = False
+        m[s["b"]:s["b"] + s["n_out"]] = False
+    return m
+
+
+def test_mlp_small_ragged_population():
+    w = inputs.make_mlp(3, 2, dims=(40, 72, 136, 7), pool=256, heldout=40, batch=24, n_classes=7, steps=6, tau=2,
+                        config_id=80, group_of=np.asarray([0, 1, 1], dtype=np.int32))
+    rng = np.random.default_rng(2)
+    segs, _ = inputs.mlp_layout(w.meta["dims"])
+    for s in segs:                                           # non-zero biases
+        w.x0[:, s["b"]:s["b"] + s["n_out"]] = (0.1 * rng.standard_normal((w.P, s["n_out"]))).astype(np.float32)
+    pop, o, tg, tr, forced = _run_pair(w, 6)
+    _check(pop, o, w, tg, tr, forced)
+    pop.close()
+
+
+def test_mlp_one_step_gradient_matches_oracle():
+    from paper_1905_10395_b200.runner import Population
+    w = inputs.make_mlp(2, 1, pool=512, heldout=128, batch=128, steps=1, tau=1, config_id=81)
+    o = _oracle(w)
+    g_ref = o.obj.grad(w.x0, 0).astype(np.float64)
+    pop = Population(w)
+    pop.lsgd.grad(pop.batches[0])
+    import torch
+    torch.cuda.synchronize()
+    g = pop.g.cpu().numpy().astype(np.float64)
+    segs, _ = inputs.mlp_layout(w.meta["dims"])
+    for s in segs:
+        for lo, n in ((s["w"], s["n_in"] * s["n_out"]), (s["b"], s["n_out"])):
+            a, b = g[:, lo:lo + n], g_ref[:, lo:lo + n]
+            assert np.linalg.norm(a - b) <= TOL * np.linalg.norm(b), (lo, n)
+            assert np.mean(np.abs(a - b) > TOL * np.abs(b).max()) <= 1e-4, (lo, n)
+    assert np.all(g[:, _pad_mask(w)] == 0)
+    pop.close()
+
+
+def test_config3_mlp_population_ten_steps():
+    w = inputs.config(3, steps=10)
+    pop, o, tg, tr, forced = _run_pair(w, 10)
+    _check(pop, o, w, tg, tr, forced)
+    pop.close()
+
+
+def test_config3_single_steps_from_the_oracle_state():
+    """Per-step parity without the amplification of a free-running trajectory: before every step the
+    GPU parameters are set to the oracle's, so each step's losses and parameter change are compared
+    for the same x_t.  Losses here must agree to 2e-2 relative with no floor."""
+    import torch
+    from paper_1905_10395_b200.runner import Population
+    w = inputs.config(3, P=8, G=2, steps=8)
+    o = _oracle(w)
+    pop = Population(w)
+    for t in range(8):
+        x_t = o.x.copy()
+        pop.x.copy_(torch.from_numpy(x_t))
+        pop.lsgd.sync_parameters()
+        o.step()
+        pop.step(record=True)
+        assert np.allclose(pop.lsgd.train_loss(), o.obj.last_train_loss, rtol=TOL, atol=0), t
+        if t % w.tau == 0:
+            hg, ho = pop.history[-1], o.history[-1]
+            assert np.allclose(hg["loss"], ho["loss"], rtol=TOL, atol=0), t
+            assert hg["gl"] == ho["gl"] and np.array_equal(hg["ll"], ho["ll"]), t
+        dx = pop.x_host().astype(np.float64) - x_t
+        dref = o.x.astype(np.float64) - x_t
+        for i in range(w.P):
+            assert np.linalg.norm(dx[i] - dref[i]) <= TOL * np.linalg.norm(dref[i]), (t, i)
+    pop.close()
