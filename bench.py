@@ -93,6 +93,16 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def _threads_used() -> int:
+    """Threads the oracle's NumPy can use: 1 for its element-wise loops; BLAS threads for matmuls."""
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -117,34 +127,72 @@ def max_over_ranks(value: float, world: int, device=None) -> float:
 
 # --------------------------------------------------------------------------------- workloads ----
 def workload_spec(args):
-    if args.workload == "c4":
-        return dict(kind="external", P=16, G=4, d=args.d or (1 << 26), eta=0.01, lambda_l=0.1, lambda_g=0.05,
-                    tau=args.tau or 1, name="C4 fused-update stress: P=16 G=4 d=2^26 fp32, supplied g and losses")
-    if args.workload == "c1":
-        return dict(kind="quadratic", P=64, G=8, d=1 << 20, eta=0.05, lambda_l=0.1, lambda_g=0.05,
-                    tau=args.tau or 4, name="C1 multi-leader quadratic: P=64 G=8 d=2^20 fp32, noise sigma=0.01")
+    wl = args.workload
+    if wl == "c4":
+        return dict(kind="external", cfg=4, P=16, G=4, d=args.d or (1 << 26), eta=0.01, lambda_l=0.1, lambda_g=0.05,
+                    tau=args.tau or 1, name="C4 fused-update stress: P=16 G=4 d=2^26 fp32, supplied g and losses",
+                    launches=(2, 1))
+    if wl == "c1":
+        return dict(kind="quadratic", cfg=1, P=64, G=8, d=1 << 20, eta=0.05, lambda_l=0.1, lambda_g=0.05,
+                    tau=args.tau or 4, name="C1 multi-leader quadratic: P=64 G=8 d=2^20 fp32, noise sigma=0.01, "
+                    "gradient fused into the update", launches=(3, 1))
+    if wl == "c0":
+        return dict(kind="quadratic", cfg=0, P=4, G=1, d=1024, eta=0.1, lambda_l=0.1, lambda_g=0.0, tau=args.tau or 1,
+                    name="C0 single-leader quadratic: P=4 G=1 d=1024", launches=(3, 1))
+    if wl == "c2":
+        return dict(kind="matcomp", cfg=2, P=16, G=4, d=200000, eta=0.01, lambda_l=0.1, lambda_g=0.05,
+                    tau=args.tau or 8, name="C2 matrix completion: P=16 G=4, 10000x10000 rank 10, batch 4096",
+                    launches=(4, 2))
+    if wl == "c3":
+        return dict(kind="mlp", cfg=3, P=32, G=4, d=1863712, eta=0.05, lambda_l=0.1, lambda_g=0.05, tau=args.tau or 4,
+                    name="C3 MLP population: P=32 G=4, 784-1024-1024-10, batch 128, bf16 GEMM fp32 accumulate",
+                    launches=(15, 10))
     raise SystemExit("unknown workload")
 
 
-def bytes_per_worker_param(spec, fused=True):
-    # update: read x + read g (or noise) + write x; quadratic adds a, b once per column
-    return 12.0 + (8.0 / spec["P"] if spec["kind"] == "quadratic" else 0.0)
+def bytes_per_worker_param(spec):
+    # update kernel: read x + read g (or noise) + write x; the fused quadratic adds a, b once per column;
+    # the MLP update also writes the bf16 copy of the weights
+    if spec["kind"] == "quadratic":
+        return 12.0 + 8.0 / spec["P"]
+    if spec["kind"] == "mlp":
+        return 14.0
+    return 12.0
 
 
 # ------------------------------------------------------------------------------ CPU oracle leg ----
 def oracle_sample_run(spec, steps, warmup, sample_cols):
-    """Times the oracle, as it stands, on a column sample of the workload (same P, G, tau)."""
+    """Times the oracle, as it stands, on a bounded sample of the workload: a column sample for the
+    element-wise objectives (same P, G, tau), the full problem for matrix completion, 4 of the
+    workers for the MLP population.  Returns (worker-params/s, seconds, description)."""
     from oracle import lsgd_oracle as orc
     from paper_1905_10395_b200 import inputs
+    P = spec["P"]
     if spec["kind"] == "external":
-        w = inputs.make_external(spec["P"], spec["G"], sample_cols, eta=spec["eta"], lambda_l=spec["lambda_l"],
+        w = inputs.make_external(P, spec["G"], sample_cols, eta=spec["eta"], lambda_l=spec["lambda_l"],
                                  lambda_g=spec["lambda_g"], tau=spec["tau"], steps=steps, config_id=4)
         obj = orc.External(w.arrays["g"], w.arrays["loss_ring"])
-    else:
-        w = inputs.make_quadratic(spec["P"], spec["G"], sample_cols, eta=spec["eta"], lambda_l=spec["lambda_l"],
+        what = f"{P} workers x {sample_cols} of {spec['d']} columns"
+    elif spec["kind"] == "quadratic":
+        cols = min(sample_cols, spec["d"])
+        w = inputs.make_quadratic(P, spec["G"], cols, eta=spec["eta"], lambda_l=spec["lambda_l"],
                                   lambda_g=spec["lambda_g"], tau=spec["tau"], steps=steps, sigma=0.01,
                                   noise_ring=2, config_id=1)
         obj = orc.Quadratic(w.arrays["a"], w.arrays["b"], 0.01, w.arrays["noise"])
+        what = f"{P} workers x {cols} of {spec['d']} columns"
+    elif spec["kind"] == "matcomp":
+        w = inputs.config(2, steps=steps + warmup, tau=spec["tau"])
+        m, A = w.meta, w.arrays
+        obj = orc.MatComp(m["n_rows"], m["n_cols"], m["rank"], A["obs_r"], A["obs_c"], A["obs_v"], A["batch_pos"],
+                          A["heldout_pos"])
+        what = "the full workload"
+    else:
+        P = 4
+        w = inputs.config(3, P=P, G=1, steps=steps + warmup, tau=spec["tau"], pool=8192)
+        A = w.arrays
+        segs, _ = inputs.mlp_layout(w.meta["dims"])
+        obj = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="bf16emu")
+        what = f"{P} of {spec['P']} workers (one group)"
     o = orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
     for _ in range(warmup):
         o.step()
@@ -152,7 +200,7 @@ def oracle_sample_run(spec, steps, warmup, sample_cols):
     for _ in range(steps):
         o.step()
     dt = time.perf_counter() - t0
-    return spec["P"] * sample_cols * steps / dt, dt
+    return P * w.d * steps / dt, dt, what
 
 
 def run_reference(args):
@@ -162,15 +210,15 @@ def run_reference(args):
     spec = workload_spec(args)
     steps, warmup = args.steps, args.warmup
     sample = args.sample_cols or (1 << 22)
-    value, dt = oracle_sample_run(spec, steps, warmup, sample)
+    value, dt, what = oracle_sample_run(spec, steps, warmup, sample)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": spec["name"], "tau": spec["tau"],
-                   "sample": f"each step covers {sample} of the {spec['d']} columns of every worker"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": f"{steps} steps x {spec['P']} workers x {sample} columns"},
+                   "sample": f"each step covers {what}"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _threads_used(), "kind": "oracle",
+                         "sample": f"{steps} steps x {what}"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -195,7 +243,8 @@ def run_ours(args):
     P, G, d = spec["P"], spec["G"], spec["d"]
     steps, warmup = args.steps, max(args.warmup, 3)
 
-    # ---- inputs: generated on the host from the seed, into pinned memory (also used by the e2e leg)
+    # ---- inputs: generated on the host from the seed (C4: into pinned memory, also used by the e2e leg)
+    hx = hg = None
     if spec["kind"] == "external":
         hx = torch.empty((P, d), dtype=torch.float32, pin_memory=True)
         hg = torch.empty((P, d), dtype=torch.float32, pin_memory=True)
@@ -204,12 +253,10 @@ def run_ours(args):
         x = hx.to(dev, non_blocking=True)
         g = hg.to(dev, non_blocking=True)
         pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith)
-        launches_per_step = lambda t: 2 if t % spec["tau"] == 0 else 1
     else:
-        w = inputs.config(1, tau=spec["tau"])
+        w = inputs.config(spec["cfg"], tau=spec["tau"])
         pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith)
-        hx = hg = None
-        launches_per_step = lambda t: 3 if t % spec["tau"] == 0 else 1
+    launches_per_step = lambda t: spec["launches"][0] if t % spec["tau"] == 0 else spec["launches"][1]
     torch.cuda.synchronize(dev)
 
     def barrier():
@@ -262,11 +309,12 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-        "ms_per_step": elapsed_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": elapsed_ms / steps, "steps_per_s": steps * world / (elapsed_ms * 1e-3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": {0: "f64", 1: "f64", 2: "f32"}[args.arith], "data": "synthetic",
         "config": {"workload": spec["name"], "tau": spec["tau"], "storage": "f32",
                    "arithmetic": ["fp64 unfused", "fp64 fma", "fp32 fma"][args.arith],
-                   "l2": "inputs (>= 0.5 GiB per step) exceed the 126 MB L2; no flush between steps",
+                   "l2": ("per-step inputs exceed the 126 MB L2; no flush between steps" if P * d * 8 > 3e8 else
+                          "working set fits in L2; steps run back to back as in training (no flush)"),
                    "multi_gpu": "replicas only"},
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
@@ -307,9 +355,10 @@ def run_ours(args):
     # ---- CPU oracle beside it (rank 0, N = 1 only)
     if rank == 0 and world == 1 and not args.no_cpu:
         sample = args.sample_cols or (1 << 22)
-        v, dt = oracle_sample_run(spec, 3, 1, sample)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"3 steps x {P} workers x {sample} of {d} columns, {dt:.1f} s"}
+        osteps = {"external": 3, "quadratic": 3, "matcomp": 8, "mlp": 4}[spec["kind"]]
+        v, dt, what = oracle_sample_run(spec, osteps, 1, sample)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": _threads_used(), "kind": "oracle",
+                                "sample": f"{osteps} steps x {what}, {dt:.1f} s"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -323,7 +372,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c4", choices=["c4", "c1"])
+    ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4"])
     ap.add_argument("--tau", type=int, default=0)
     ap.add_argument("--arith", type=int, default=0, choices=[0, 1, 2])
     ap.add_argument("--e2e-steps", type=int, default=3)

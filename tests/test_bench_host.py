@@ -1,0 +1,52 @@
+"""Host-side logic of bench.py for N > 1, on CPU with 2 gloo ranks (the data path itself has no
+collective: ranks are independent replicas)."""
+import json
+import os
+import socket
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _torchrun(script_args, n=2, timeout=300):
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
+           "127.0.0.1", "--master-port", str(_free_port())] + script_args
+    return subprocess.run(cmd, capture_output=True, text=True, timeout=timeout, cwd=ROOT)
+
+
+def _json_lines(out):
+    return [json.loads(l) for l in out.splitlines() if l.startswith("{")]
+
+
+def test_two_rank_timing_is_max_and_value_is_whole_job():
+    r = _torchrun([os.path.join(ROOT, "tests", "_gloo_worker.py")])
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = _json_lines(r.stdout)
+    assert len(lines) == 1
+    assert lines[0]["world"] == 2 and lines[0]["slowest_ms"] == 20.0
+    assert abs(lines[0]["value"] - 2 * 1000.0 / 0.020) < 1e-6
+
+
+def test_reference_arm_prints_once_under_two_ranks():
+    r = _torchrun([os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup",
+                   "0", "--sample-cols", "4096"])
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = _json_lines(r.stdout)
+    assert len(lines) == 1
+    l = lines[0]
+    assert l["impl"] == "reference" and l["n_gpus"] == 2 and l["cpu_baseline"]["kind"] == "oracle"
+    assert l["e2e"]["h2d_bytes_per_step"] == 0 and l["value"] > 0
+
+
+def test_single_process_defaults():
+    import bench
+    assert bench.dist_env() == (0, 1, 0) or "RANK" in os.environ
+    assert bench.max_over_ranks(3.5, 1) == 3.5
+    assert bench.aggregate(100.0, 50.0, 4) == 100.0 * 4 / 0.05
