@@ -217,7 +217,8 @@ def run_reference(args):
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": spec["name"], "tau": spec["tau"],
                    "sample": f"each step covers {what}"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _threads_used(), "kind": "oracle",
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _threads_used() if spec["kind"] == "mlp" else 1,
+                         "kind": "oracle",
                          "sample": f"{steps} steps x {what}"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -320,7 +321,9 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
                      "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
-                     "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags))},
+                     "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags)),
+                     "ms_pull": float(np.mean([m for m, f in zip(k_ms, pull_flags) if f])) if any(pull_flags) else None,
+                     "ms_plain": float(np.mean([m for m, f in zip(k_ms, pull_flags) if not f])) if not all(pull_flags) else None},
         "gpu_launches": n_launch,
     }
 
@@ -357,7 +360,8 @@ def run_ours(args):
         sample = args.sample_cols or (1 << 22)
         osteps = {"external": 3, "quadratic": 3, "matcomp": 8, "mlp": 4}[spec["kind"]]
         v, dt, what = oracle_sample_run(spec, osteps, 1, sample)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": _threads_used(), "kind": "oracle",
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": _threads_used() if spec["kind"] == "mlp" else 1,
+                                "kind": "oracle",
                                 "sample": f"{osteps} steps x {what}, {dt:.1f} s"}
     if rank == 0:
         print(json.dumps(line), flush=True)

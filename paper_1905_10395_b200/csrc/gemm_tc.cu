@@ -34,6 +34,8 @@ constexpr int kABytes = BM * BK * 2;                        // 16 KiB
 constexpr int kThreads = 192;                               // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr int kSmemBytes = kStages * kStageBytes + 1024;    // + slack for 1024-byte alignment
 constexpr uint32_t kTmemCols = 128;
+constexpr int kStagePitch = BN + 4;                         // floats; 16-byte accesses stay conflict-free
+static_assert((size_t)BM * kStagePitch * 4 <= (size_t)kStages * kStageBytes, "staging tile must fit in the ring");
 constexpr long long kWaitBudgetCycles = 2000000000LL;       // about one second
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -200,64 +202,67 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     // ---------------------------------------------------------------- epilogue
     if (mbar_wait(&acc_bar, 0, abort_flag, p.status)) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      // All MMAs have completed, so the operand ring is free: it becomes a staging tile through which
+      // the accumulator is transposed from "one row per thread" (tensor-memory order) to "one row per
+      // warp instruction" (512 contiguous bytes per store).  A warp only touches its own 32 rows.
+      float* stage = reinterpret_cast<float*>(smem);
       const int q = warp & 3;                 // TMEM lane quarter this warp may read
-      const int m = m0 + q * 32 + lane;
-      const bool row_ok = m < p.M;
-      const int64_t zc = (int64_t)z * p.stride_c;
+      float* my_row = stage + (size_t)(q * 32 + lane) * kStagePitch;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        const int nb = n0 + c * 32;
-        if (!row_ok || nb >= p.N) continue;
-        const bool full = (nb + 32 <= p.N) && p.vec_ok;
-        if (p.epilogue == GEMM_EPI_F32) {
-          float* out = static_cast<float*>(p.c) + zc + (int64_t)m * p.ldc + nb;
-          if (full) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(out + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                                                __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+        for (int j = 0; j < 32; j += 4)
+          *reinterpret_cast<uint4*>(my_row + c * 32 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+      }
+      __syncwarp();
+      const int n = n0 + lane * 4;            // this lane's 4 columns
+      const int64_t zc = (int64_t)z * p.stride_c;
+      float bias4[4] = {0.f, 0.f, 0.f, 0.f};
+      if (p.epilogue == GEMM_EPI_BIAS_RELU_BF16) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (n + j < p.N) bias4[j] = p.bias[(int64_t)z * p.stride_bias + n + j];
+      }
+      const bool full = (n + 4 <= p.N) && p.vec_ok;
+#pragma unroll 4
+      for (int rr = 0; rr < 32; ++rr) {
+        const int m = m0 + q * 32 + rr;
+        if (m >= p.M || n >= p.N) break;
+        const float4 a4 = *reinterpret_cast<const float4*>(stage + (size_t)(q * 32 + rr) * kStagePitch + lane * 4);
+        float v[4] = {a4.x, a4.y, a4.z, a4.w};
+        if (p.epilogue == GEMM_EPI_F32) {
+          float* out = static_cast<float*>(p.c) + zc + (int64_t)m * p.ldc + n;
+          if (full) {
+            *reinterpret_cast<float4*>(out) = a4;
           } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (nb + j < p.N) out[j] = __uint_as_float(r[j]);
+            for (int j = 0; j < 4; ++j)
+              if (n + j < p.N) out[j] = v[j];
           }
         } else {
-          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.c) + zc + (int64_t)m * p.ldc + nb;
-          const float* bias = p.bias ? p.bias + (int64_t)z * p.stride_bias + nb : nullptr;
-          const __nv_bfloat16* mask =
-              p.mask ? static_cast<const __nv_bfloat16*>(p.mask) + (int64_t)z * p.stride_mask + (int64_t)m * p.ld_mask + nb : nullptr;
-          float v[32];
+          if (p.epilogue == GEMM_EPI_BIAS_RELU_BF16) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            float a = __uint_as_float(r[j]);
-            if (nb + j < p.N) {
-              if (p.epilogue == GEMM_EPI_BIAS_RELU_BF16) {
-                a = fmaxf(a + bias[j], 0.f);
-              } else if (p.epilogue == GEMM_EPI_MASK_BF16) {
-                a = (__bfloat162float(mask[j]) > 0.f) ? a : 0.f;
-              }
-            }
-            v[j] = a;
+            for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j] + bias4[j], 0.f);
+          } else if (p.epilogue == GEMM_EPI_MASK_BF16) {
+            const __nv_bfloat16* mk = static_cast<const __nv_bfloat16*>(p.mask) + (int64_t)z * p.stride_mask + (int64_t)m * p.ld_mask + n;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (n + j < p.N) v[j] = (__bfloat162float(mk[j]) > 0.f) ? v[j] : 0.f;
           }
+          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.c) + zc + (int64_t)m * p.ldc + n;
           if (full) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              __nv_bfloat162 h0 = __floats2bfloat162_rn(v[j], v[j + 1]), h1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]), h3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
-              uint4 u;
-              u.x = *reinterpret_cast<uint32_t*>(&h0);
-              u.y = *reinterpret_cast<uint32_t*>(&h1);
-              u.z = *reinterpret_cast<uint32_t*>(&h2);
-              u.w = *reinterpret_cast<uint32_t*>(&h3);
-              *reinterpret_cast<uint4*>(out + j) = u;
-            }
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
+            uint2 u;
+            u.x = *reinterpret_cast<uint32_t*>(&h0);
+            u.y = *reinterpret_cast<uint32_t*>(&h1);
+            *reinterpret_cast<uint2*>(out) = u;
           } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (nb + j < p.N) out[j] = __float2bfloat16_rn(v[j]);
+            for (int j = 0; j < 4; ++j)
+              if (n + j < p.N) out[j] = __float2bfloat16_rn(v[j]);
           }
         }
       }

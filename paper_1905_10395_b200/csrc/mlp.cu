@@ -96,119 +96,180 @@ __global__ void gather_rows_kernel(const float* __restrict__ pool, const int32_t
   for (int k = threadIdx.x; k < d0; k += blockDim.x) xb[(int64_t)row * d0 + k] = __float2bfloat16_rn(s[k]);
 }
 
-// One warp per sample: logits, softmax cross-entropy, and (training) dZ = (p - onehot) / n rounded to bf16.
-__global__ void __launch_bounds__(256)
+__device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 t = __bfloat1622float2(h[j]);
+    f[2 * j] = t.x;
+    f[2 * j + 1] = t.y;
+  }
+}
+
+constexpr int kHeadWarps = 8;
+constexpr int kHeadSamplesPerWarp = 4;   // a CTA covers 32 samples and stages W3 once in shared memory
+
+// Last layer forward.  One warp per sample: logits Z = H2 W3^T + b3 from 16-byte (8 x bf16) loads, the
+// softmax cross-entropy of the sample, and (training) dZ = (p - onehot) / n rounded to bf16.
+__global__ void __launch_bounds__(kHeadWarps * 32)
 head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ x,
                     const int32_t* __restrict__ labels, const int32_t* __restrict__ label_idx, float* __restrict__ dz,
                     float* __restrict__ loss_b, int32_t n, int32_t d2, int32_t C, int64_t ld, int64_t w3_off, int64_t b3_off,
                     int32_t label_rows, uint32_t* status) {
+  extern __shared__ uint4 s_w3[];   // [C][d2 / 8]
   const int i = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.x * (blockDim.x >> 5) + warp;
-  if (b >= n) return;
-  const __nv_bfloat16* h = h2 + ((int64_t)i * n + b) * d2;
-  const __nv_bfloat16* w3 = wb + (int64_t)i * ld + w3_off;
-  float acc[kMaxClasses];
+  const int chunks = d2 >> 3;
+  const uint4* w3 = reinterpret_cast<const uint4*>(wb + (int64_t)i * ld + w3_off);
+  for (int t = threadIdx.x; t < C * chunks; t += blockDim.x) s_w3[t] = w3[t];
+  __syncthreads();
+  const float* b3 = x + (int64_t)i * ld + b3_off;
+  for (int sidx = 0; sidx < kHeadSamplesPerWarp; ++sidx) {
+    const int b = (blockIdx.x * kHeadWarps + warp) * kHeadSamplesPerWarp + sidx;
+    if (b >= n) break;
+    const uint4* h = reinterpret_cast<const uint4*>(h2 + ((int64_t)i * n + b) * d2);
+    float acc[kMaxClasses];
 #pragma unroll
-  for (int c = 0; c < kMaxClasses; ++c) acc[c] = 0.f;
-  for (int k = lane; k < d2; k += 32) {
-    const float hv = __bfloat162float(h[k]);
-#pragma unroll
-    for (int c = 0; c < kMaxClasses; ++c)
-      if (c < C) acc[c] = fmaf(hv, __bfloat162float(w3[(int64_t)c * d2 + k]), acc[c]);
-  }
-#pragma unroll
-  for (int c = 0; c < kMaxClasses; ++c)
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xFFFFFFFFu, acc[c], o);
-  if (lane == 0) {
-    int y = label_idx ? label_idx[(int64_t)i * n + b] : b;   // training: pool row of this sample
-    if (y < 0 || y >= label_rows) {
-      atomicOr(status, FLAG_BAD_INDEX);
-      y = 0;
-    }
-    int cls = labels[y];
-    if (cls < 0 || cls >= C) {
-      atomicOr(status, FLAG_BAD_INDEX);
-      cls = 0;
-    }
-    const float* b3 = x + (int64_t)i * ld + b3_off;
-    float zmax = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < kMaxClasses; ++c)
-      if (c < C) {
-        acc[c] += b3[c];
-        zmax = fmaxf(zmax, acc[c]);
-      }
-    float sum = 0.f, zy = 0.f;
-#pragma unroll
-    for (int c = 0; c < kMaxClasses; ++c)
-      if (c < C) {
-        sum += expf(acc[c] - zmax);
-        if (c == cls) zy = acc[c];
-      }
-    const float lse = zmax + logf(sum);
-    loss_b[(int64_t)i * n + b] = lse - zy;
-    if (dz) {
-      const float inv_n = 1.f / (float)n;
+    for (int c = 0; c < kMaxClasses; ++c) acc[c] = 0.f;
+    for (int ch = lane; ch < chunks; ch += 32) {
+      float hv[8];
+      unpack8(h[ch], hv);
 #pragma unroll
       for (int c = 0; c < kMaxClasses; ++c)
         if (c < C) {
-          const float pc = expf(acc[c] - lse);
-          const float v = (pc - (c == cls ? 1.f : 0.f)) * inv_n;
-          dz[((int64_t)i * n + b) * C + c] = __bfloat162float(__float2bfloat16_rn(v));
+          float wv[8];
+          unpack8(s_w3[c * chunks + ch], wv);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[c] = fmaf(hv[j], wv[j], acc[c]);
         }
+    }
+#pragma unroll
+    for (int c = 0; c < kMaxClasses; ++c)
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xFFFFFFFFu, acc[c], o);
+    if (lane == 0) {
+      int y = label_idx ? label_idx[(int64_t)i * n + b] : b;   // training: pool row of this sample
+      if (y < 0 || y >= label_rows) {
+        atomicOr(status, FLAG_BAD_INDEX);
+        y = 0;
+      }
+      int cls = labels[y];
+      if (cls < 0 || cls >= C) {
+        atomicOr(status, FLAG_BAD_INDEX);
+        cls = 0;
+      }
+      float zmax = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < kMaxClasses; ++c)
+        if (c < C) {
+          acc[c] += b3[c];
+          zmax = fmaxf(zmax, acc[c]);
+        }
+      float sum = 0.f, zy = 0.f;
+#pragma unroll
+      for (int c = 0; c < kMaxClasses; ++c)
+        if (c < C) {
+          sum += expf(acc[c] - zmax);
+          if (c == cls) zy = acc[c];
+        }
+      const float lse = zmax + logf(sum);
+      loss_b[(int64_t)i * n + b] = lse - zy;
+      if (dz) {
+        const float inv_n = 1.f / (float)n;
+#pragma unroll
+        for (int c = 0; c < kMaxClasses; ++c)
+          if (c < C) {
+            const float pc = expf(acc[c] - lse);
+            const float v = (pc - (c == cls ? 1.f : 0.f)) * inv_n;
+            dz[((int64_t)i * n + b) * C + c] = __bfloat162float(__float2bfloat16_rn(v));
+          }
+      }
     }
   }
 }
 
-// One thread per hidden unit k of the last hidden layer: dW3[:, k], dH2[:, k] (masked, rounded), db2[k];
-// block 0 of each worker also writes db3.
-__global__ void __launch_bounds__(128)
+constexpr int kBwdCols = 128;    // hidden units per CTA
+constexpr int kBwdSlices = 4;    // batch slices per CTA (blockDim.y), combined in a fixed order
+
+// Last layer backward.  Thread (k, s) walks the samples b = s, s + 4, ... of hidden unit k:
+// dH2[b][k] = [H2 > 0] * sum_c dZ[b][c] W3[c][k] (rounded to bf16 and stored), and its share of
+// dW3[:, k] and db2[k]; the 4 slices are added in slice order.  Block 0 of each worker also writes db3.
+__global__ void __launch_bounds__(kBwdCols * kBwdSlices)
 head_backward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ dz,
                      __nv_bfloat16* __restrict__ dh2, float* __restrict__ g, int32_t n, int32_t d2, int32_t C, int64_t ld,
                      int64_t w3_off, int64_t b3_off, int64_t b2_off) {
-  extern __shared__ float s_dz[];   // [n][C]
+  extern __shared__ float s_mem[];
+  float* s_dz = s_mem;                       // [n][C]
+  float* s_red = s_mem + (size_t)n * C;      // [kBwdSlices][C + 1][kBwdCols]
   const int i = blockIdx.y;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const int tid = ty * kBwdCols + tx;
   const float* dzi = dz + (int64_t)i * n * C;
-  for (int t = threadIdx.x; t < n * C; t += blockDim.x) s_dz[t] = dzi[t];
+  for (int t = tid; t < n * C; t += kBwdCols * kBwdSlices) s_dz[t] = dzi[t];
   __syncthreads();
   float* gi = g + (int64_t)i * ld;
-  if (blockIdx.x == 0 && threadIdx.x < C) {
+  if (blockIdx.x == 0 && tid < C) {
     float s = 0.f;
-    for (int b = 0; b < n; ++b) s += s_dz[b * C + threadIdx.x];
-    gi[b3_off + threadIdx.x] = s;
+    for (int b = 0; b < n; ++b) s += s_dz[b * C + tid];
+    gi[b3_off + tid] = s;
   }
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= d2) return;
+  const int k = blockIdx.x * kBwdCols + tx;
+  const bool live = k < d2;
   const __nv_bfloat16* w3 = wb + (int64_t)i * ld + w3_off;
   float w[kMaxClasses], aw[kMaxClasses];
 #pragma unroll
   for (int c = 0; c < kMaxClasses; ++c) {
-    w[c] = c < C ? __bfloat162float(w3[(int64_t)c * d2 + k]) : 0.f;
+    w[c] = (live && c < C) ? __bfloat162float(w3[(int64_t)c * d2 + k]) : 0.f;
     aw[c] = 0.f;
   }
   float ab = 0.f;
-  const __nv_bfloat16* hcol = h2 + (int64_t)i * n * d2 + k;
-  __nv_bfloat16* dcol = dh2 + (int64_t)i * n * d2 + k;
-  for (int b = 0; b < n; ++b) {
-    const float hv = __bfloat162float(hcol[(int64_t)b * d2]);
-    float dh = 0.f;
+  if (live) {
+    const __nv_bfloat16* hcol = h2 + (int64_t)i * n * d2 + k;
+    __nv_bfloat16* dcol = dh2 + (int64_t)i * n * d2 + k;
+    for (int b0 = ty; b0 < n; b0 += 4 * kBwdSlices) {
+      float hv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int b = b0 + u * kBwdSlices;
+        hv[u] = b < n ? __bfloat162float(hcol[(int64_t)b * d2]) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int b = b0 + u * kBwdSlices;
+        if (b < n) {
+          float dh = 0.f;
+#pragma unroll
+          for (int c = 0; c < kMaxClasses; ++c)
+            if (c < C) {
+              const float z = s_dz[b * C + c];
+              aw[c] = fmaf(z, hv[u], aw[c]);
+              dh = fmaf(z, w[c], dh);
+            }
+          const __nv_bfloat16 r = __float2bfloat16_rn(hv[u] > 0.f ? dh : 0.f);
+          dcol[(int64_t)b * d2] = r;
+          ab += __bfloat162float(r);
+        }
+      }
+    }
+  }
+  float* red = s_red + (size_t)ty * (C + 1) * kBwdCols;
+#pragma unroll
+  for (int c = 0; c < kMaxClasses; ++c)
+    if (c < C) red[c * kBwdCols + tx] = aw[c];
+  red[C * kBwdCols + tx] = ab;
+  __syncthreads();
+  if (ty == 0 && live) {
 #pragma unroll
     for (int c = 0; c < kMaxClasses; ++c)
       if (c < C) {
-        const float z = s_dz[b * C + c];
-        aw[c] = fmaf(z, hv, aw[c]);
-        dh = fmaf(z, w[c], dh);
+        float t = 0.f;
+        for (int sl = 0; sl < kBwdSlices; ++sl) t += s_red[((size_t)sl * (C + 1) + c) * kBwdCols + tx];
+        gi[w3_off + (int64_t)c * d2 + k] = t;
       }
-    const __nv_bfloat16 r = __float2bfloat16_rn(hv > 0.f ? dh : 0.f);
-    dcol[(int64_t)b * d2] = r;
-    ab += __bfloat162float(r);
+    float t = 0.f;
+    for (int sl = 0; sl < kBwdSlices; ++sl) t += s_red[((size_t)sl * (C + 1) + C) * kBwdCols + tx];
+    gi[b2_off + k] = t;
   }
-#pragma unroll
-  for (int c = 0; c < kMaxClasses; ++c)
-    if (c < C) gi[w3_off + (int64_t)c * d2 + k] = aw[c];
-  gi[b2_off + k] = ab;
 }
 
 // db[k] = sum_b delta[b][k] for a stored (bf16) delta matrix.
@@ -270,6 +331,10 @@ lsgd_status mlp_validate(const lsgd_config& c, const lsgd_mlp_desc& m) {
   // TMA rows must be 16-byte multiples (8 bf16); the head kernels keep the class scores in registers
   if (m.dims[0] % 8 || m.dims[1] % 8 || m.dims[2] % 8 || m.dims[3] > kMaxClasses) return LSGD_ERR_UNSUPPORTED;
   if (m.batch % 8 || m.n_heldout % 8 || m.batch > 1024) return LSGD_ERR_UNSUPPORTED;
+  // shared-memory budgets of the last-layer kernels (48 KB without opting in)
+  if ((size_t)m.dims[3] * m.dims[2] * 2 > 48 * 1024) return LSGD_ERR_UNSUPPORTED;
+  if (sizeof(float) * ((size_t)m.batch * m.dims[3] + (size_t)kBwdSlices * (m.dims[3] + 1) * kBwdCols) > 48 * 1024)
+    return LSGD_ERR_UNSUPPORTED;
   const Layout L = param_layout(m.dims);
   if (L.d != c.d || c.ld != c.d) return LSGD_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(m.scratch) & 1023u) return LSGD_ERR_ALIGNMENT;
@@ -339,9 +404,12 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx) {
   lsgd_status fs = forward_hidden(h, st->m_xb, 1, B, st->h1, st->m_h1, st->h2);
   if (fs != LSGD_OK) return fs;
 
-  head_forward_kernel<<<dim3((B + 7) / 8, P), 256, 0, s>>>(st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2],
+  const int per_cta = kHeadWarps * kHeadSamplesPerWarp;
+  const size_t w3_smem = (size_t)d[3] * d[2] * 2;
+  head_forward_kernel<<<dim3((B + per_cta - 1) / per_cta, P), kHeadWarps * 32, w3_smem, s>>>(st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2],
                                                           d[3], ld, st->L.w[2], st->L.b[2], m.pool, h->d_status);
-  head_backward_kernel<<<dim3((d[2] + 127) / 128, P), 128, sizeof(float) * B * d[3], s>>>(
+  const size_t bwd_smem = sizeof(float) * ((size_t)B * d[3] + (size_t)kBwdSlices * (d[3] + 1) * kBwdCols);
+  head_backward_kernel<<<dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdCols, kBwdSlices), bwd_smem, s>>>(
       st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]);
   if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
 
@@ -369,7 +437,8 @@ lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss) {
   const int32_t* d = st->dims;
   lsgd_status fs = forward_hidden(h, st->m_xh, 0, st->nH, st->hh1, st->m_hh1, st->hh2);
   if (fs != LSGD_OK) return fs;
-  head_forward_kernel<<<dim3((st->nH + 7) / 8, st->P), 256, 0, h->stream>>>(st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr,
+  const int per_cta = kHeadWarps * kHeadSamplesPerWarp;
+  head_forward_kernel<<<dim3((st->nH + per_cta - 1) / per_cta, st->P), kHeadWarps * 32, (size_t)d[3] * d[2] * 2, h->stream>>>(st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr,
                                                                           st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2],
                                                                           st->L.b[2], st->nH, h->d_status);
   row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_h, loss, st->nH);
