@@ -107,7 +107,7 @@ __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
 }
 
 constexpr int kHeadWarps = 8;
-constexpr int kHeadSamplesPerWarp = 4;   // a CTA covers 32 samples and stages W3 once in shared memory
+constexpr int kHeadSamplesPerWarp = 1;   // a CTA covers 8 samples and stages W3 once in shared memory
 
 // Last layer forward.  One warp per sample: logits Z = H2 W3^T + b3 from 16-byte (8 x bf16) loads, the
 // softmax cross-entropy of the sample, and (training) dZ = (p - onehot) / n rounded to bf16.
@@ -188,12 +188,12 @@ head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* _
   }
 }
 
-constexpr int kBwdCols = 128;    // hidden units per CTA
-constexpr int kBwdSlices = 4;    // batch slices per CTA (blockDim.y), combined in a fixed order
+constexpr int kBwdCols = 64;     // hidden units per CTA
+constexpr int kBwdSlices = 8;    // batch slices per CTA (blockDim.y), combined in a fixed order
 
-// Last layer backward.  Thread (k, s) walks the samples b = s, s + 4, ... of hidden unit k:
+// Last layer backward.  Thread (k, s) walks the samples b = s, s + 8, ... of hidden unit k:
 // dH2[b][k] = [H2 > 0] * sum_c dZ[b][c] W3[c][k] (rounded to bf16 and stored), and its share of
-// dW3[:, k] and db2[k]; the 4 slices are added in slice order.  Block 0 of each worker also writes db3.
+// dW3[:, k] and db2[k]; the slices are added in slice order.  Block 0 of each worker also writes db3.
 __global__ void __launch_bounds__(kBwdCols * kBwdSlices)
 head_backward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ dz,
                      __nv_bfloat16* __restrict__ dh2, float* __restrict__ g, int32_t n, int32_t d2, int32_t C, int64_t ld,

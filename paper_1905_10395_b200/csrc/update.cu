@@ -21,8 +21,31 @@
 namespace lsgd {
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kRowsInFlight = 4;  // rows whose loads are issued before the first is consumed
+// Launch shapes, chosen by timing sweeps on the 16 x 2^26 stress shape (fp64 arithmetic):
+//   pull form : 256 threads, 2 rows of loads in flight, registers capped for 4 CTAs per SM, 8 grid-stride
+//               CTAs per SM (more rows in flight cost occupancy and lose; 5+ CTAs per SM spill);
+//   plain form: 256 threads, 4 elements in flight, one CTA per 1024 columns up to 64 CTAs per SM.
+#ifndef LSGD_K1_THREADS
+#define LSGD_K1_THREADS 256
+#endif
+#ifndef LSGD_K1_PULL_ROWS
+#define LSGD_K1_PULL_ROWS 2
+#endif
+#ifndef LSGD_K1_PULL_MIN_BLOCKS
+#define LSGD_K1_PULL_MIN_BLOCKS 4
+#endif
+#ifndef LSGD_K1_PULL_CTAS_PER_SM
+#define LSGD_K1_PULL_CTAS_PER_SM 8
+#endif
+#ifndef LSGD_K1_PLAIN_ROWS
+#define LSGD_K1_PLAIN_ROWS 4
+#endif
+#ifndef LSGD_K1_PLAIN_CTAS_PER_SM
+#define LSGD_K1_PLAIN_CTAS_PER_SM 64
+#endif
+constexpr int kThreads = LSGD_K1_THREADS;
+constexpr int kPullRows = LSGD_K1_PULL_ROWS;     // rows whose loads are issued before the first is consumed
+constexpr int kPlainRows = LSGD_K1_PLAIN_ROWS;
 
 __device__ __forceinline__ float4 ld4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ float4 ld4_cached(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
@@ -87,7 +110,7 @@ __device__ __forceinline__ float pull1(float x, float g, float xl, float xg, con
 }
 
 template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, LSGD_K1_PULL_MIN_BLOCKS)
 pull_update_kernel(UpdateArgs p, int64_t n4) {
   extern __shared__ int32_t s_tab[];
   int32_t* s_ll = s_tab;                 // [G]
@@ -127,11 +150,11 @@ pull_update_kernel(UpdateArgs p, int64_t n4) {
       const int l = s_ll[j];
       const float4 xl = (l == gl) ? xg : ld4(xc + (int64_t)l * ld);
       const int m1 = s_start[j + 1];
-      for (int m = s_start[j]; m < m1; m += kRowsInFlight) {
-        float4 xs[kRowsInFlight], gs[kRowsInFlight];
-        int rows[kRowsInFlight];
+      for (int m = s_start[j]; m < m1; m += kPullRows) {
+        float4 xs[kPullRows], gs[kPullRows];
+        int rows[kPullRows];
 #pragma unroll
-        for (int u = 0; u < kRowsInFlight; ++u) {
+        for (int u = 0; u < kPullRows; ++u) {
           if (m + u < m1) {
             const int i = s_rows[m + u];
             rows[u] = i;
@@ -140,7 +163,7 @@ pull_update_kernel(UpdateArgs p, int64_t n4) {
           }
         }
 #pragma unroll
-        for (int u = 0; u < kRowsInFlight; ++u) {
+        for (int u = 0; u < kPullRows; ++u) {
           if (m + u < m1) {
             float4 x = xs[u], g = gs[u];
             if (QUAD) {
@@ -170,11 +193,11 @@ plain_update_kernel(UpdateArgs p, int64_t n4) {
   const int64_t total = (int64_t)p.P * n4;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   const Coef k = p.k;
-  for (int64_t e0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e0 < total; e0 += stride * kRowsInFlight) {
-    float4 xs[kRowsInFlight], gs[kRowsInFlight];
-    int64_t off[kRowsInFlight], cols[kRowsInFlight];
+  for (int64_t e0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e0 < total; e0 += stride * kPlainRows) {
+    float4 xs[kPlainRows], gs[kPlainRows];
+    int64_t off[kPlainRows], cols[kPlainRows];
 #pragma unroll
-    for (int u = 0; u < kRowsInFlight; ++u) {
+    for (int u = 0; u < kPlainRows; ++u) {
       const int64_t e = e0 + u * stride;
       if (e < total) {
         const int64_t row = e / n4, c = e - row * n4;
@@ -185,7 +208,7 @@ plain_update_kernel(UpdateArgs p, int64_t n4) {
       }
     }
 #pragma unroll
-    for (int u = 0; u < kRowsInFlight; ++u) {
+    for (int u = 0; u < kPlainRows; ++u) {
       const int64_t e = e0 + u * stride;
       if (e < total) {
         float4 x = xs[u], g = gs[u];
@@ -219,7 +242,7 @@ cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
     if (sms <= 0) sms = 148;
   }
   const int64_t n4 = (a.d + 3) / 4;
-  const int64_t cap = (int64_t)sms * 8;
+  const int64_t cap = (int64_t)sms * (a.pull ? LSGD_K1_PULL_CTAS_PER_SM : LSGD_K1_PLAIN_CTAS_PER_SM);
   if (a.pull) {
     int64_t blocks = (n4 + kThreads - 1) / kThreads;
     if (blocks > cap) blocks = cap;
@@ -228,7 +251,7 @@ cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
     pull_update_kernel<MODE, QUAD, NOISE, SHADOW><<<(unsigned)blocks, kThreads, smem, s>>>(a, n4);
   } else {
     const int64_t total = (int64_t)a.P * n4;
-    int64_t blocks = (total + (int64_t)kThreads * kRowsInFlight - 1) / ((int64_t)kThreads * kRowsInFlight);
+    int64_t blocks = (total + (int64_t)kThreads * kPlainRows - 1) / ((int64_t)kThreads * kPlainRows);
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     plain_update_kernel<MODE, QUAD, NOISE, SHADOW><<<(unsigned)blocks, kThreads, 0, s>>>(a, n4);
