@@ -186,6 +186,45 @@ pull_update_kernel(UpdateArgs p, int64_t n4) {
   }
 }
 
+// Plain step with the quadratic gradient evaluated inline: a thread owns a 16-byte column for all P
+// rows, so a and b (and their conversions to the evaluation precision) are paid once per column.
+template <int MODE, bool NOISE>
+__global__ void __launch_bounds__(kThreads, LSGD_K1_PULL_MIN_BLOCKS)
+quad_plain_column_kernel(UpdateArgs p, int64_t n4) {
+  const Coef k = p.k;
+  const int64_t ld = p.ld;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < n4; c += stride) {
+    const int64_t col = c * 4;
+    float* xc = p.x + col;
+    const float* nc = p.quad.noise + col;
+    const float4 av = ld4_cached(p.quad.a + col);
+    const float4 bv = ld4_cached(p.quad.b + col);
+    for (int m = 0; m < p.P; m += kPullRows) {
+      float4 xs[kPullRows], ns[kPullRows];
+#pragma unroll
+      for (int u = 0; u < kPullRows; ++u) {
+        if (m + u < p.P) {
+          xs[u] = ld4(xc + (int64_t)(m + u) * ld);
+          if (NOISE) ns[u] = ld4(nc + (int64_t)(m + u) * ld);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kPullRows; ++u) {
+        if (m + u < p.P) {
+          const float4 x = xs[u], n = ns[u];
+          float4 r;
+          r.x = plain1<MODE>(x.x, quad_g<MODE>(x.x, av.x, bv.x, n.x, k, NOISE), k);
+          r.y = plain1<MODE>(x.y, quad_g<MODE>(x.y, av.y, bv.y, n.y, k, NOISE), k);
+          r.z = plain1<MODE>(x.z, quad_g<MODE>(x.z, av.z, bv.z, n.z, k, NOISE), k);
+          r.w = plain1<MODE>(x.w, quad_g<MODE>(x.w, av.w, bv.w, n.w, k, NOISE), k);
+          st4(xc + (int64_t)(m + u) * ld, r);
+        }
+      }
+    }
+  }
+}
+
 // Plain step x <- x - eta g over the whole [P][n4] grid of 16-byte columns.
 template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
 __global__ void __launch_bounds__(kThreads)
@@ -249,6 +288,12 @@ cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
     if (blocks < 1) blocks = 1;
     const size_t smem = sizeof(int32_t) * (size_t)(a.P + 2 * a.G + 1);
     pull_update_kernel<MODE, QUAD, NOISE, SHADOW><<<(unsigned)blocks, kThreads, smem, s>>>(a, n4);
+  } else if (QUAD && !SHADOW) {
+    int64_t blocks = (n4 + kThreads - 1) / kThreads;
+    const int64_t qcap = (int64_t)sms * LSGD_K1_PULL_CTAS_PER_SM;
+    if (blocks > qcap) blocks = qcap;
+    if (blocks < 1) blocks = 1;
+    quad_plain_column_kernel<MODE, NOISE><<<(unsigned)blocks, kThreads, 0, s>>>(a, n4);
   } else {
     const int64_t total = (int64_t)a.P * n4;
     int64_t blocks = (total + (int64_t)kThreads * kPlainRows - 1) / ((int64_t)kThreads * kPlainRows);
