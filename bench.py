@@ -150,6 +150,11 @@ def workload_spec(args):
     raise SystemExit("unknown workload")
 
 
+# DRAM bytes per worker-parameter of the update kernels, from the ncu counters of a d = 2^22 capture of
+# the same kernels (profiles/pull_update_kernel_c4.md); traffic is proportional to d.
+MEASURED_TRAFFIC_PER_WORKER_PARAM = {"pull": 11.34, "plain": 11.30}
+
+
 def bytes_per_worker_param(spec):
     # update kernel: read x + read g (or noise) + write x; the fused quadratic adds a, b once per column;
     # the MLP update also writes the bf16 copy of the weights
@@ -305,6 +310,11 @@ def run_ours(args):
     alg_bytes = bytes_per_worker_param(spec) * P * d
     peak, peak_src = read_peaks()
     achieved = alg_bytes / (upd_ms * 1e-3) / 1e9
+    traffic = None
+    if spec["kind"] == "external" and args.arith == 0:
+        n_pull = sum(pull_flags)
+        traffic = P * d * (n_pull * MEASURED_TRAFFIC_PER_WORKER_PARAM["pull"] +
+                           (steps - n_pull) * MEASURED_TRAFFIC_PER_WORKER_PARAM["plain"]) / steps
     if pop.lsgd.check_device() != 0:
         raise SystemExit("device status word set during the bench")
 
@@ -320,7 +330,7 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
                      "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
+                     "traffic": traffic, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
                      "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags)),
                      "ms_pull": float(np.mean([m for m, f in zip(k_ms, pull_flags) if f])) if any(pull_flags) else None,
                      "ms_plain": float(np.mean([m for m, f in zip(k_ms, pull_flags) if not f])) if not all(pull_flags) else None},

@@ -188,10 +188,10 @@ head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* _
   }
 }
 
-constexpr int kBwdCols = 64;     // hidden units per CTA
-constexpr int kBwdSlices = 8;    // batch slices per CTA (blockDim.y), combined in a fixed order
+constexpr int kBwdCols = 128;    // hidden units per CTA
+constexpr int kBwdSlices = 4;    // batch slices per CTA (blockDim.y), combined in a fixed order
 
-// Last layer backward.  Thread (k, s) walks the samples b = s, s + 8, ... of hidden unit k:
+// Last layer backward.  Thread (k, s) walks the samples b = s, s + 4, ... of hidden unit k:
 // dH2[b][k] = [H2 > 0] * sum_c dZ[b][c] W3[c][k] (rounded to bf16 and stored), and its share of
 // dW3[:, k] and db2[k]; the slices are added in slice order.  Block 0 of each worker also writes db3.
 __global__ void __launch_bounds__(kBwdCols * kBwdSlices)
