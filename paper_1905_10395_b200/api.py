@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "liblsgd.so")
  ERR_TOO_LARGE) = range(9)
 OBJ_EXTERNAL, OBJ_QUADRATIC, OBJ_MATCOMP, OBJ_MLP = range(4)
 ARITH_FP64, ARITH_FP64_FMA, ARITH_FP32 = range(3)
+FLAG_MLP_KEEP_GRADIENTS = 1
 
 
 class LsgdError(RuntimeError):
@@ -52,7 +53,7 @@ class Config(C.Structure):
                 ("d", C.c_int64), ("ld", C.c_int64), ("eta", C.c_float), ("lambda_l", C.c_float),
                 ("lambda_g", C.c_float), ("tau", C.c_int32), ("objective", C.c_int32),
                 ("objective_desc", C.c_void_p), ("x", C.c_void_p), ("g", C.c_void_p), ("stream", C.c_void_p),
-                ("arithmetic", C.c_int32)]
+                ("arithmetic", C.c_int32), ("flags", C.c_uint32)]
 
 
 _lib = None
@@ -168,7 +169,7 @@ def mlp_scratch_bytes(dims: Sequence[int], P: int, batch: int, n_heldout: int) -
 
 def make_config(*, P: int, G: int, group_of: np.ndarray, d: int, ld: int, eta: float, lambda_l: float,
                 lambda_g: float, tau: int, objective: int, desc=None, x=None, g=None, stream: int = 0,
-                arithmetic: int = ARITH_FP64):
+                arithmetic: int = ARITH_FP64, flags: int = 0):
     """Returns (Config, keepalive) -- keepalive holds the host arrays the struct points to."""
     go = np.ascontiguousarray(group_of, dtype=np.int32)
     cfg = Config()
@@ -184,6 +185,7 @@ def make_config(*, P: int, G: int, group_of: np.ndarray, d: int, ld: int, eta: f
     cfg.g = _ptr(g)
     cfg.stream = stream or None
     cfg.arithmetic = int(arithmetic)
+    cfg.flags = int(flags)
     return cfg, (go, desc)
 
 

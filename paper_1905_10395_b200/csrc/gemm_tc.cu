@@ -200,6 +200,16 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     if (ok) mma_commit(&acc_bar);  // accumulator complete
   } else if (warp >= 2) {
     // ---------------------------------------------------------------- epilogue
+    if (p.epilogue == GEMM_EPI_SGD) {
+      // while the products run, pull this tile of x towards L2 (each thread one 512-byte row)
+      const int m = m0 + (warp & 3) * 32 + lane;
+      if (m < p.M) {
+        const float* xr = p.x_upd + (int64_t)z * p.stride_c + (int64_t)m * p.ldc + n0;
+#pragma unroll
+        for (int j = 0; j < BN; j += 32)
+          if (n0 + j < p.N) asm volatile("prefetch.global.L2 [%0];" ::"l"(xr + j));
+      }
+    }
     if (mbar_wait(&acc_bar, 0, abort_flag, p.status)) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       // All MMAs have completed, so the operand ring is free: it becomes a staging tile through which
@@ -227,6 +237,66 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           if (n + j < p.N) bias4[j] = p.bias[(int64_t)z * p.stride_bias + n + j];
       }
       const bool full = (n + 4 <= p.N) && p.vec_ok;
+      if (p.epilogue == GEMM_EPI_SGD) {
+        // The accumulator is this block of the gradient: take the plain step x <- x - eta g here, in
+        // place, and refresh the bf16 copy; g is not stored.  Rows are processed 8 at a time so that 8
+        // loads of x are in flight per lane.
+        constexpr int kBatch = 8;
+#pragma unroll 1
+        for (int r0 = 0; r0 < 32; r0 += kBatch) {
+          float4 xv[kBatch];
+#pragma unroll
+          for (int u = 0; u < kBatch; ++u) {
+            const int m = m0 + q * 32 + r0 + u;
+            xv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (m < p.M && n < p.N) {
+              const float* xo = p.x_upd + zc + (int64_t)m * p.ldc + n;
+              if (full) {
+                xv[u] = *reinterpret_cast<const float4*>(xo);
+              } else {
+                xv[u].x = xo[0];
+                if (n + 1 < p.N) xv[u].y = xo[1];
+                if (n + 2 < p.N) xv[u].z = xo[2];
+                if (n + 3 < p.N) xv[u].w = xo[3];
+              }
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < kBatch; ++u) {
+            const int m = m0 + q * 32 + r0 + u;
+            if (m < p.M && n < p.N) {
+              const float4 g4 = *reinterpret_cast<const float4*>(stage + (size_t)(q * 32 + r0 + u) * kStagePitch + lane * 4);
+              float xs[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w};
+              const float gs[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                if (p.arith == 0) xs[j] = (float)__dsub_rn((double)xs[j], __dmul_rn(p.eta, (double)gs[j]));
+                else if (p.arith == 1) xs[j] = (float)fma(-p.eta, (double)gs[j], (double)xs[j]);
+                else xs[j] = fmaf(-(float)p.eta, gs[j], xs[j]);
+              }
+              const int64_t off = zc + (int64_t)m * p.ldc + n;
+              float* xo = p.x_upd + off;
+              uint16_t* so = p.x_shadow + off;
+              if (full) {
+                *reinterpret_cast<float4*>(xo) = make_float4(xs[0], xs[1], xs[2], xs[3]);
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(xs[0], xs[1]), h1 = __floats2bfloat162_rn(xs[2], xs[3]);
+                uint2 u2;
+                u2.x = *reinterpret_cast<uint32_t*>(&h0);
+                u2.y = *reinterpret_cast<uint32_t*>(&h1);
+                *reinterpret_cast<uint2*>(so) = u2;
+              } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  if (n + j < p.N) {
+                    xo[j] = xs[j];
+                    __nv_bfloat16 hb = __float2bfloat16_rn(xs[j]);
+                    so[j] = *reinterpret_cast<uint16_t*>(&hb);
+                  }
+              }
+            }
+          }
+        }
+      } else
 #pragma unroll 4
       for (int rr = 0; rr < 32; ++rr) {
         const int m = m0 + q * 32 + rr;
@@ -319,8 +389,9 @@ cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, con
     attr_set = true;
   }
   GemmShape q = p;
-  const int64_t esz = (p.epilogue == GEMM_EPI_F32) ? 4 : 2;
-  q.vec_ok = ((reinterpret_cast<uintptr_t>(p.c) & 15u) == 0 && (p.ldc * esz) % 16 == 0 && (p.stride_c * esz) % 16 == 0) ? 1 : 0;
+  const int64_t esz = (p.epilogue == GEMM_EPI_F32 || p.epilogue == GEMM_EPI_SGD) ? 4 : 2;
+  const void* cbase = p.epilogue == GEMM_EPI_SGD ? static_cast<const void*>(p.x_upd) : p.c;
+  q.vec_ok = ((reinterpret_cast<uintptr_t>(cbase) & 15u) == 0 && (p.ldc * esz) % 16 == 0 && (p.stride_c * esz) % 16 == 0) ? 1 : 0;
   dim3 grid((unsigned)((p.N + BN - 1) / BN), (unsigned)((p.M + BM - 1) / BM), (unsigned)p.batch);
   bgemm_bf16_kernel<<<grid, kThreads, kSmemBytes, s>>>(map_a, map_b, q);
   return cudaGetLastError();

@@ -11,6 +11,7 @@ enum GemmEpilogue : int {
   GEMM_EPI_BIAS_RELU_BF16 = 1,  // C bf16 = relu(acc + bias[n])
   GEMM_EPI_MASK_BF16 = 2,       // C bf16 = mask[m][n] > 0 ? acc : 0
   GEMM_EPI_BF16 = 3,            // C bf16 = acc
+  GEMM_EPI_SGD = 4,             // internal: x[m][n] <- x[m][n] - eta * acc (fp32, in place) and its bf16 copy
 };
 
 struct GemmShape {
@@ -25,6 +26,10 @@ struct GemmShape {
   int64_t stride_bias;
   const void* mask;             // bf16 [batch][M][ld_mask]
   int64_t ld_mask, stride_mask;
+  float* x_upd;                 // GEMM_EPI_SGD: parameters, indexed like C (ldc, stride_c)
+  uint16_t* x_shadow;           // GEMM_EPI_SGD: bf16 copy of the parameters, indexed like C
+  double eta;                   // GEMM_EPI_SGD
+  int arith;                    // GEMM_EPI_SGD: 0 fp64 unfused, 1 fp64 fma, 2 fp32 fma (as the update kernel)
   uint32_t* status;             // device status word (bounded-wait failures)
 };
 

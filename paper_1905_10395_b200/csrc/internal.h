@@ -114,6 +114,7 @@ struct lsgd_ctx {
   int64_t t;
   int64_t n_elections;
   bool grad_ready;
+  bool fused_applied;        // MLP: the pending gradient has already stepped W1, W2 (plain step)
   const float* armed_noise;  // QUADRATIC with g == NULL: noise pointer for the next step
   void* mlp_state;           // opaque MLP pipeline state
 };

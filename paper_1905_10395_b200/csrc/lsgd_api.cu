@@ -97,6 +97,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->t = 0;
   h->n_elections = 0;
   h->grad_ready = false;
+  h->fused_applied = false;
   h->armed_noise = nullptr;
   h->slab = nullptr;
   h->mlp_state = nullptr;
@@ -196,8 +197,11 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
     }
     case LSGD_OBJ_MLP: {
       if (!batch) return LSGD_ERR_INVALID_ARG;
-      lsgd_status st = mlp_grad(h, static_cast<const int32_t*>(batch));
+      if (h->fused_applied) return LSGD_ERR_STATE;   // the pending gradient has already moved W1, W2
+      const bool fuse = (h->t % c.tau) != 0 && !(c.flags & LSGD_FLAG_MLP_KEEP_GRADIENTS);
+      lsgd_status st = mlp_grad(h, static_cast<const int32_t*>(batch), fuse);
       if (st != LSGD_OK) return st;
+      h->fused_applied = fuse;
       break;
     }
     default:
@@ -242,6 +246,7 @@ lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
         break;
       }
       case LSGD_OBJ_MLP: {
+        if (h->fused_applied) return LSGD_ERR_STATE;   // x is between two steps: no loss at x_t any more
         lsgd_status st = mlp_heldout_loss(h, h->d_loss);
         if (st != LSGD_OK) return st;
         e.loss_in = h->d_loss;
@@ -285,8 +290,23 @@ lsgd_status lsgd_step(lsgd_handle h) {
   a.arith = c.arithmetic;
   a.status = h->d_status;
   a.pull = pull;
-  LSGD_CUDA(launch_update(a, h->stream));
+  if (h->fused_applied) {
+    // W1 and W2 were stepped inside lsgd_grad; finish the biases and the last layer
+    int64_t ranges[4][2];
+    const int nr = mlp_unfused_ranges(h, ranges);
+    for (int r = 0; r < nr; ++r) {
+      UpdateArgs b = a;
+      b.x = a.x + ranges[r][0];
+      b.g = a.g + ranges[r][0];
+      b.x_bf16 = a.x_bf16 + ranges[r][0];
+      b.d = ranges[r][1];
+      LSGD_CUDA(launch_update(b, h->stream));
+    }
+  } else {
+    LSGD_CUDA(launch_update(a, h->stream));
+  }
   h->t++;
+  h->fused_applied = false;
   h->grad_ready = false;
   h->armed_noise = nullptr;
   return LSGD_OK;

@@ -390,7 +390,7 @@ lsgd_status mlp_create(lsgd_ctx* h) {
   return LSGD_OK;
 }
 
-lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx) {
+lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   MlpState* st = state(h);
   const lsgd_config& c = h->cfg;
   const lsgd_mlp_desc& m = h->mlp;
@@ -420,12 +420,20 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx) {
   gd.stride_mask = (int64_t)B * d[1];
   if (launch_bgemm(st->m_dh2, st->m_w2, gd, s) != cudaSuccess) return LSGD_ERR_CUDA;
   // dW2 = dH2^T . H1                          [d2 x d1], contraction over the batch
-  GemmShape g2 = shape(d[2], d[1], B, P, 1, 1, 1, GEMM_EPI_F32, c.g + st->L.w[1], d[1], ld, h->d_status);
+  GemmShape g2 = shape(d[2], d[1], B, P, 1, 1, 1, fuse_sgd ? GEMM_EPI_SGD : GEMM_EPI_F32, c.g + st->L.w[1], d[1], ld, h->d_status);
+  g2.x_upd = c.x + st->L.w[1];
+  g2.x_shadow = reinterpret_cast<uint16_t*>(st->wb) + st->L.w[1];
+  g2.eta = (double)c.eta;
+  g2.arith = c.arithmetic;
   if (launch_bgemm(st->m_dh2, st->m_h1, g2, s) != cudaSuccess) return LSGD_ERR_CUDA;
   column_sum_kernel<<<dim3((d[1] + 127) / 128, P), 128, 0, s>>>(st->dh1, c.g, B, d[1], ld, st->L.b[0]);
   if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
   // dW1 = dH1^T . X                           [d1 x d0]
-  GemmShape g1 = shape(d[1], d[0], B, P, 1, 1, 1, GEMM_EPI_F32, c.g + st->L.w[0], d[0], ld, h->d_status);
+  GemmShape g1 = shape(d[1], d[0], B, P, 1, 1, 1, fuse_sgd ? GEMM_EPI_SGD : GEMM_EPI_F32, c.g + st->L.w[0], d[0], ld, h->d_status);
+  g1.x_upd = c.x + st->L.w[0];
+  g1.x_shadow = reinterpret_cast<uint16_t*>(st->wb) + st->L.w[0];
+  g1.eta = (double)c.eta;
+  g1.arith = c.arithmetic;
   if (launch_bgemm(st->m_dh1, st->m_xb, g1, s) != cudaSuccess) return LSGD_ERR_CUDA;
   return LSGD_OK;
 }
@@ -450,6 +458,16 @@ lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss) {
   if (!st) return LSGD_ERR_STATE;
   row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_b, loss, st->B);
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
+}
+
+int mlp_unfused_ranges(lsgd_ctx* h, int64_t (*ranges)[2]) {
+  MlpState* st = state(h);
+  // everything except W1 and W2: b1, then b2 | W3 | b3 (contiguous)
+  ranges[0][0] = st->L.b[0];
+  ranges[0][1] = st->L.w[1] - st->L.b[0];
+  ranges[1][0] = st->L.b[1];
+  ranges[1][1] = st->L.d - st->L.b[1];
+  return 2;
 }
 
 lsgd_status mlp_refresh_shadow(lsgd_ctx* h) {

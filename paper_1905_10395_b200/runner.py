@@ -15,7 +15,7 @@ from .inputs import Workload
 class Population:
     def __init__(self, w: Workload, *, fused_quadratic: bool = False, arithmetic: int = api.ARITH_FP64,
                  device: str = "cuda:0", x: Optional[torch.Tensor] = None, g: Optional[torch.Tensor] = None,
-                 upload_noise: bool = True):
+                 upload_noise: bool = True, flags: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.w = w
@@ -77,7 +77,8 @@ class Population:
             raise ValueError(w.objective)
         cfg, keep = api.make_config(P=w.P, G=w.G, group_of=w.group_of, d=w.d, ld=w.ld, eta=w.eta,
                                     lambda_l=w.lambda_l, lambda_g=w.lambda_g, tau=w.tau, objective=obj, desc=desc,
-                                    x=self.x, g=self.g, stream=self.stream.cuda_stream, arithmetic=arithmetic)
+                                    x=self.x, g=self.g, stream=self.stream.cuda_stream, arithmetic=arithmetic,
+                                    flags=flags)
         self._keep.append(keep)
         self.lsgd = api.Lsgd(cfg, keep)
         self.t = 0
