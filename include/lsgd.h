@@ -229,9 +229,9 @@ LSGD_API uint64_t lsgd_mlp_scratch_bytes(const int32_t* dims, int32_t P, int32_t
  * against a library matmul on its own.  All pointers DEVICE.
  *   a_mn_major = 0: A is stored [M][lda] (K contiguous);  1: A is stored [K][lda] (M contiguous).
  *   b_mn_major = 0: B is stored [N][ldb] (K contiguous);  1: B is stored [K][ldb] (N contiguous).
- *   lda, ldb, ldc: row pitch in elements; lda, ldb multiples of 8.  stride_*: elements between batch
- *   entries (stride_a / stride_b = 0 shares the operand across the batch; multiples of 8 otherwise).
- *   a, b 16-byte aligned.  epilogue: 0 C fp32 = acc; 1 C bf16 = relu(acc + bias[z][n]);
+ *   lda, ldb, ldc: row pitch in elements; lda, ldb and the pitch of a bf16 C / mask multiples of 8, the
+ *   pitch of an fp32 C a multiple of 4.  stride_*: elements between batch entries (stride_a / stride_b
+ *   = 0 shares the operand across the batch; multiples of 8 otherwise).  a, b, c, mask 16-byte aligned.  epilogue: 0 C fp32 = acc; 1 C bf16 = relu(acc + bias[z][n]);
  *   2 C bf16 = (mask[z][m][n] > 0 ? acc : 0), mask bf16; 3 C bf16 = acc.
  * Enqueues on `stream` and returns.  LSGD_ERR_ALIGNMENT if an operand breaks the rules above.      */
 typedef struct {

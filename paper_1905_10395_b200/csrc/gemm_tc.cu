@@ -1,24 +1,31 @@
 // Batched bf16 x bf16 -> fp32 matrix product on the 5th-generation tensor cores (tcgen05), used by
 // the MLP population objective.  C[z] = A[z] . B[z], C is M x N, the contraction length is K.
 //
-//   * operands are fetched by TMA (cp.async.bulk.tensor, 128-byte swizzle) into a 3-stage shared
-//     memory ring guarded by mbarriers; each stage holds a 128 x 64 slice of A and of B;
-//   * one elected thread issues tcgen05.mma (M = 128, N = 128, K = 16, cta_group::1) with the fp32
-//     accumulator tile (128 lanes x 128 columns) in tensor memory;
-//   * four epilogue warps read the accumulator back with tcgen05.ld and apply the fused epilogue
-//     (bias + ReLU + bf16 store, ReLU-mask + bf16 store, or plain fp32 / bf16 store).
+// Persistent kernel, one CTA per SM, tiles of 128 x 128 handed out round-robin (tile = CTA, CTA +
+// grid, ...), three roles:
+//   * warp 0 (one thread): TMA producer.  cp.async.bulk.tensor loads of the operands (128-byte swizzle)
+//     into a 3-stage shared-memory ring guarded by mbarriers; each stage holds a 128 x 64 slice of A
+//     and of B.  For epilogues that read a tile (the parameters x for the fused SGD step, the ReLU
+//     mask) it also loads that tile into the epilogue buffer.
+//   * warp 1 (one thread): issues tcgen05.mma (M = 128, N = 128, K = 16, cta_group::1) into one of TWO
+//     fp32 accumulator tiles in tensor memory (2 x 128 columns), so the products of tile i+1 overlap
+//     the epilogue of tile i.
+//   * warps 2..5: epilogue.  tcgen05.ld of the accumulator (thread = row), fused arithmetic, swizzled
+//     st.shared into the epilogue buffers, then ONE thread issues TMA stores of the whole tile
+//     (cp.async.bulk.tensor shared -> global): all global traffic of the kernel goes through TMA, edge
+//     tiles are clipped by the tensor maps.
 //
 // Either operand may be "K-major" (the contraction index is contiguous in memory) or "MN-major"
 // (the M resp. N index is contiguous): weights W[out][in], activations H[batch][feature] and their
-// transposes are all consumed in place, nothing is transposed in memory.  In shared memory a
-// 64-element-wide box is always 128 bytes per row, so both majors use 1024-byte swizzle atoms:
+// transposes are all consumed in place.  In shared memory a 64-element-wide box is always 128 bytes
+// per row, so both majors use 1024-byte swizzle atoms:
 //   K-major : rows = M/N index, 8-row groups 1024 B apart (SBO); one K = 16 step is +32 B;
 //   MN-major: rows = K index, 64-wide M/N blocks 8192 B apart (LBO), 8-row K groups 1024 B apart
 //             (SBO); one K = 16 step is +2048 B.
 //
 // Every wait on an mbarrier is bounded by a clock budget; on expiry the kernel raises
-// FLAG_WAIT_TIMEOUT in the status word, drains what it has in flight, frees its tensor memory and
-// returns.
+// FLAG_WAIT_TIMEOUT in the status word, every role leaves its loop, outstanding bulk stores are
+// drained, tensor memory is freed and the CTA returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -31,11 +38,11 @@ constexpr int BM = 128, BN = 128, BK = 64;
 constexpr int kStages = 3;
 constexpr int kStageBytes = (BM * BK + BN * BK) * 2;       // 32 KiB
 constexpr int kABytes = BM * BK * 2;                        // 16 KiB
+constexpr int kEpiF32Bytes = BM * BN * 4;                   // 64 KiB: fp32 tile, 4 boxes of [128][32 floats]
+constexpr int kEpiBf16Bytes = BM * BN * 2;                  // 32 KiB: bf16 tile, 2 boxes of [128][64 bf16]
 constexpr int kThreads = 192;                               // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
-constexpr int kSmemBytes = kStages * kStageBytes + 1024;    // + slack for 1024-byte alignment
-constexpr uint32_t kTmemCols = 128;
-constexpr int kStagePitch = BN + 4;                         // floats; 16-byte accesses stay conflict-free
-static_assert((size_t)BM * kStagePitch * 4 <= (size_t)kStages * kStageBytes, "staging tile must fit in the ring");
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiF32Bytes + kEpiBf16Bytes + 1024;
+constexpr uint32_t kTmemCols = 256;                         // two accumulator tiles
 constexpr long long kWaitBudgetCycles = 2000000000LL;       // about one second
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -45,6 +52,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
@@ -75,6 +85,11 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
       : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const void* src, const CUtensorMap* map, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
+               : "memory");
 }
 
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -108,18 +123,40 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-__global__ void __launch_bounds__(kThreads)
-bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmShape p) {
+// Byte offset of the 16-byte unit `u` (0..7) of row `r` inside a [rows][128 B] box written / read by TMA
+// with the 128-byte swizzle: the unit index is XORed with the row index modulo 8.
+__device__ __forceinline__ uint32_t swz(int r, int u) { return (uint32_t)(r * 128 + ((u ^ (r & 7)) << 4)); }
+
+struct Tile {
+  int z, m0, n0;
+};
+__device__ __forceinline__ Tile tile_of(int t, int mt, int nt) {
+  Tile q;
+  q.n0 = (t % nt) * BN;
+  t /= nt;
+  q.m0 = (t % mt) * BM;
+  q.z = t / mt;
+  return q;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_aux, GemmShape p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ uint64_t full_bar[kStages], empty_bar[kStages], acc_bar;
+  uint8_t* buf_f32 = smem + kStages * kStageBytes;          // fp32 tile: C out, or x in/out (SGD)
+  uint8_t* buf_b16 = buf_f32 + kEpiF32Bytes;                // bf16 tile: C out, mask in, or bf16 copy of x out
+  __shared__ uint64_t full_bar[kStages], empty_bar[kStages], acc_full[2], acc_empty[2], in_full, in_free;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, z = blockIdx.z;
+  const int mt = (p.M + BM - 1) / BM, nt = (p.N + BN - 1) / BN;
+  const int n_tiles = mt * nt * p.batch;
   const int nk = (p.K + BK - 1) / BK;
+  const bool reads_tile = (p.epilogue == GEMM_EPI_SGD) || (p.epilogue == GEMM_EPI_MASK_BF16);
 
   if (threadIdx.x == 0) {
     abort_s = 0;
@@ -127,10 +164,17 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(&acc_bar, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 4);      // one arrival per epilogue warp
+    }
+    mbar_init(&in_full, 1);
+    mbar_init(&in_free, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_aux) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(kTmemCols) : "memory");
@@ -144,199 +188,198 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
   if (warp == 0 && lane == 0) {
     // ---------------------------------------------------------------- TMA producer
-    const int za = p.a_batched ? z : 0, zb = p.b_batched ? z : 0;
-    int issued = 0;
-    for (int kt = 0; kt < nk; ++kt) {
-      const int s = kt % kStages;
-      if (kt >= kStages && !mbar_wait(&empty_bar[s], ((kt / kStages) - 1) & 1, abort_flag, p.status)) break;
-      uint8_t* sa = smem + s * kStageBytes;
-      uint8_t* sb = sa + kABytes;
-      mbar_expect_tx(&full_bar[s], kStageBytes);
-      const int k0 = kt * BK;
-      // two 64-wide boxes per operand; a box is [64 rows][64 elements = 128 B]
-      if (p.a_mn) {
-        tma_load_3d(sa, &map_a, &full_bar[s], m0, k0, za);
-        tma_load_3d(sa + 8192, &map_a, &full_bar[s], m0 + 64, k0, za);
-      } else {
-        tma_load_3d(sa, &map_a, &full_bar[s], k0, m0, za);
-        tma_load_3d(sa + 8192, &map_a, &full_bar[s], k0, m0 + 64, za);
+    uint32_t it = 0;        // operand stages issued so far (all tiles)
+    int local = 0;          // tiles this CTA has started
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
+      const Tile q = tile_of(t, mt, nt);
+      const int za = p.a_batched ? q.z : 0, zb = p.b_batched ? q.z : 0;
+      for (int kt = 0; kt < nk; ++kt, ++it) {
+        const int s = it % kStages;
+        ok = mbar_wait(&empty_bar[s], ((it / kStages) & 1) ^ 1, abort_flag, p.status);
+        if (!ok) break;
+        uint8_t* sa = smem + s * kStageBytes;
+        uint8_t* sb = sa + kABytes;
+        mbar_expect_tx(&full_bar[s], kStageBytes);
+        const int k0 = kt * BK;
+        // two 64-wide boxes per operand; a box is [64 rows][64 elements = 128 B]
+        if (p.a_mn) {
+          tma_load_3d(sa, &map_a, &full_bar[s], q.m0, k0, za);
+          tma_load_3d(sa + 8192, &map_a, &full_bar[s], q.m0 + 64, k0, za);
+        } else {
+          tma_load_3d(sa, &map_a, &full_bar[s], k0, q.m0, za);
+          tma_load_3d(sa + 8192, &map_a, &full_bar[s], k0, q.m0 + 64, za);
+        }
+        if (p.b_mn) {
+          tma_load_3d(sb, &map_b, &full_bar[s], q.n0, k0, zb);
+          tma_load_3d(sb + 8192, &map_b, &full_bar[s], q.n0 + 64, k0, zb);
+        } else {
+          tma_load_3d(sb, &map_b, &full_bar[s], k0, q.n0, zb);
+          tma_load_3d(sb + 8192, &map_b, &full_bar[s], k0, q.n0 + 64, zb);
+        }
       }
-      if (p.b_mn) {
-        tma_load_3d(sb, &map_b, &full_bar[s], n0, k0, zb);
-        tma_load_3d(sb + 8192, &map_b, &full_bar[s], n0 + 64, k0, zb);
-      } else {
-        tma_load_3d(sb, &map_b, &full_bar[s], k0, n0, zb);
-        tma_load_3d(sb + 8192, &map_b, &full_bar[s], k0, n0 + 64, zb);
-      }
-      issued = kt + 1;
-    }
-    if (*abort_flag) {
-      // drain: wait (bounded) for the copies already issued before the CTA may exit
-      const int first = issued > kStages ? issued - kStages : 0;
-      for (int kt = first; kt < issued; ++kt) {
-        const long long t0 = clock64();
-        while (!mbar_try(&full_bar[kt % kStages], (kt / kStages) & 1) && clock64() - t0 < kWaitBudgetCycles) {}
+      if (ok && reads_tile) {
+        // the epilogue's input tile, once the previous tile's stores have finished reading the buffers
+        ok = mbar_wait(&in_free, (local & 1) ^ 1, abort_flag, p.status);
+        if (!ok) break;
+        if (p.epilogue == GEMM_EPI_SGD) {
+          mbar_expect_tx(&in_full, kEpiF32Bytes);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tma_load_3d(buf_f32 + c * 16384, &map_c, &in_full, q.n0 + c * 32, q.m0, q.z);
+        } else {
+          mbar_expect_tx(&in_full, kEpiBf16Bytes);
+#pragma unroll
+          for (int c = 0; c < 2; ++c) tma_load_3d(buf_b16 + c * 16384, &map_aux, &in_full, q.n0 + c * 64, q.m0, q.z);
+        }
       }
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------------------------------------------------------- MMA issuer
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.a_mn ? 1 : 0) << 15) |
                            ((uint32_t)(p.b_mn ? 1 : 0) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    uint32_t it = 0;
+    int local = 0;
     bool ok = true;
-    for (int kt = 0; kt < nk && ok; ++kt) {
-      const int s = kt % kStages;
-      ok = mbar_wait(&full_bar[s], (kt / kStages) & 1, abort_flag, p.status);
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
+      const int b = local & 1;
+      ok = mbar_wait(&acc_empty[b], ((local >> 1) & 1) ^ 1, abort_flag, p.status);   // epilogue has drained it
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t sa = smem_u32(smem + s * kStageBytes), sb = sa + kABytes;
+      const uint32_t tacc = tmem_base + (uint32_t)(b * BN);
+      for (int kt = 0; kt < nk; ++kt, ++it) {
+        const int s = it % kStages;
+        ok = mbar_wait(&full_bar[s], (it / kStages) & 1, abort_flag, p.status);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t sa = smem_u32(smem + s * kStageBytes), sb = sa + kABytes;
 #pragma unroll
-      for (int k = 0; k < BK / 16; ++k) {
-        const uint64_t da = p.a_mn ? smem_desc(sa + k * 2048, 8192, 1024) : smem_desc(sa + k * 32, 16, 1024);
-        const uint64_t db = p.b_mn ? smem_desc(sb + k * 2048, 8192, 1024) : smem_desc(sb + k * 32, 16, 1024);
-        mma_bf16(tmem_base, da, db, idesc, (kt | k) != 0 ? 1u : 0u);
+        for (int k = 0; k < BK / 16; ++k) {
+          const uint64_t da = p.a_mn ? smem_desc(sa + k * 2048, 8192, 1024) : smem_desc(sa + k * 32, 16, 1024);
+          const uint64_t db = p.b_mn ? smem_desc(sb + k * 2048, 8192, 1024) : smem_desc(sb + k * 32, 16, 1024);
+          mma_bf16(tacc, da, db, idesc, (kt | k) != 0 ? 1u : 0u);
+        }
+        mma_commit(&empty_bar[s]);   // the stage is free once these MMAs have read it
       }
-      mma_commit(&empty_bar[s]);   // the stage is free once these MMAs have read it
+      if (ok) mma_commit(&acc_full[b]);  // accumulator complete
     }
-    if (ok) mma_commit(&acc_bar);  // accumulator complete
   } else if (warp >= 2) {
-    // ---------------------------------------------------------------- epilogue
-    if (p.epilogue == GEMM_EPI_SGD) {
-      // while the products run, pull this tile of x towards L2 (each thread one 512-byte row)
-      const int m = m0 + (warp & 3) * 32 + lane;
-      if (m < p.M) {
-        const float* xr = p.x_upd + (int64_t)z * p.stride_c + (int64_t)m * p.ldc + n0;
-#pragma unroll
-        for (int j = 0; j < BN; j += 32)
-          if (n0 + j < p.N) asm volatile("prefetch.global.L2 [%0];" ::"l"(xr + j));
-      }
-    }
-    if (mbar_wait(&acc_bar, 0, abort_flag, p.status)) {
+    // ---------------------------------------------------------------- epilogue (128 threads)
+    const int q4 = warp & 3;                  // TMEM lane quarter this warp may read
+    const int row = q4 * 32 + lane;           // row of the tile owned by this thread
+    const bool leader = (threadIdx.x == 64);  // issues the bulk stores
+    int local = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
+      const Tile q = tile_of(t, mt, nt);
+      const int b = local & 1;
+      ok = mbar_wait(&acc_full[b], (local >> 1) & 1, abort_flag, p.status);
+      if (ok && reads_tile) ok = mbar_wait(&in_full, local & 1, abort_flag, p.status);
+      if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      // All MMAs have completed, so the operand ring is free: it becomes a staging tile through which
-      // the accumulator is transposed from "one row per thread" (tensor-memory order) to "one row per
-      // warp instruction" (512 contiguous bytes per store).  A warp only touches its own 32 rows.
-      float* stage = reinterpret_cast<float*>(smem);
-      const int q = warp & 3;                 // TMEM lane quarter this warp may read
-      float* my_row = stage + (size_t)(q * 32 + lane) * kStagePitch;
+      const uint32_t tacc = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * BN);
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+        tmem_ld32(tacc + (uint32_t)(c * 32), r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-        for (int j = 0; j < 32; j += 4)
-          *reinterpret_cast<uint4*>(my_row + c * 32 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
-      }
-      __syncwarp();
-      const int n = n0 + lane * 4;            // this lane's 4 columns
-      const int64_t zc = (int64_t)z * p.stride_c;
-      float bias4[4] = {0.f, 0.f, 0.f, 0.f};
-      if (p.epilogue == GEMM_EPI_BIAS_RELU_BF16) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          if (n + j < p.N) bias4[j] = p.bias[(int64_t)z * p.stride_bias + n + j];
-      }
-      const bool full = (n + 4 <= p.N) && p.vec_ok;
-      if (p.epilogue == GEMM_EPI_SGD) {
-        // The accumulator is this block of the gradient: take the plain step x <- x - eta g here, in
-        // place, and refresh the bf16 copy; g is not stored.  Rows are processed 8 at a time so that 8
-        // loads of x are in flight per lane.
-        constexpr int kBatch = 8;
-#pragma unroll 1
-        for (int r0 = 0; r0 < 32; r0 += kBatch) {
-          float4 xv[kBatch];
-#pragma unroll
-          for (int u = 0; u < kBatch; ++u) {
-            const int m = m0 + q * 32 + r0 + u;
-            xv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (m < p.M && n < p.N) {
-              const float* xo = p.x_upd + zc + (int64_t)m * p.ldc + n;
-              if (full) {
-                xv[u] = *reinterpret_cast<const float4*>(xo);
-              } else {
-                xv[u].x = xo[0];
-                if (n + 1 < p.N) xv[u].y = xo[1];
-                if (n + 2 < p.N) xv[u].z = xo[2];
-                if (n + 3 < p.N) xv[u].w = xo[3];
-              }
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < kBatch; ++u) {
-            const int m = m0 + q * 32 + r0 + u;
-            if (m < p.M && n < p.N) {
-              const float4 g4 = *reinterpret_cast<const float4*>(stage + (size_t)(q * 32 + r0 + u) * kStagePitch + lane * 4);
-              float xs[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w};
-              const float gs[4] = {g4.x, g4.y, g4.z, g4.w};
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                if (p.arith == 0) xs[j] = (float)__dsub_rn((double)xs[j], __dmul_rn(p.eta, (double)gs[j]));
-                else if (p.arith == 1) xs[j] = (float)fma(-p.eta, (double)gs[j], (double)xs[j]);
-                else xs[j] = fmaf(-(float)p.eta, gs[j], xs[j]);
-              }
-              const int64_t off = zc + (int64_t)m * p.ldc + n;
-              float* xo = p.x_upd + off;
-              uint16_t* so = p.x_shadow + off;
-              if (full) {
-                *reinterpret_cast<float4*>(xo) = make_float4(xs[0], xs[1], xs[2], xs[3]);
-                __nv_bfloat162 h0 = __floats2bfloat162_rn(xs[0], xs[1]), h1 = __floats2bfloat162_rn(xs[2], xs[3]);
-                uint2 u2;
-                u2.x = *reinterpret_cast<uint32_t*>(&h0);
-                u2.y = *reinterpret_cast<uint32_t*>(&h1);
-                *reinterpret_cast<uint2*>(so) = u2;
-              } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                  if (n + j < p.N) {
-                    xo[j] = xs[j];
-                    __nv_bfloat16 hb = __float2bfloat16_rn(xs[j]);
-                    so[j] = *reinterpret_cast<uint16_t*>(&hb);
-                  }
-              }
-            }
-          }
-        }
-      } else
-#pragma unroll 4
-      for (int rr = 0; rr < 32; ++rr) {
-        const int m = m0 + q * 32 + rr;
-        if (m >= p.M || n >= p.N) break;
-        const float4 a4 = *reinterpret_cast<const float4*>(stage + (size_t)(q * 32 + rr) * kStagePitch + lane * 4);
-        float v[4] = {a4.x, a4.y, a4.z, a4.w};
+        uint8_t* f32_box = buf_f32 + c * 16384;                 // [128 rows][32 floats]
+        uint8_t* b16_box = buf_b16 + (c >> 1) * 16384;          // [128 rows][64 bf16]; this chunk is half a row
+        const int b16_u0 = (c & 1) * 4;
         if (p.epilogue == GEMM_EPI_F32) {
-          float* out = static_cast<float*>(p.c) + zc + (int64_t)m * p.ldc + n;
-          if (full) {
-            *reinterpret_cast<float4*>(out) = a4;
-          } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (n + j < p.N) out[j] = v[j];
+          for (int u = 0; u < 8; ++u)
+            *reinterpret_cast<uint4*>(f32_box + swz(row, u)) = make_uint4(r[4 * u], r[4 * u + 1], r[4 * u + 2], r[4 * u + 3]);
+        } else if (p.epilogue == GEMM_EPI_SGD) {
+          // the accumulator is this block of the gradient: plain step x <- x - eta g on the staged x tile
+          float xn[32];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const float4 x4 = *reinterpret_cast<const float4*>(f32_box + swz(row, u));
+            const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float g = __uint_as_float(r[4 * u + j]);
+              if (p.arith == 0) xn[4 * u + j] = (float)__dsub_rn((double)xs[j], __dmul_rn(p.eta, (double)g));
+              else if (p.arith == 1) xn[4 * u + j] = (float)fma(-p.eta, (double)g, (double)xs[j]);
+              else xn[4 * u + j] = fmaf(-(float)p.eta, g, xs[j]);
+            }
+            *reinterpret_cast<float4*>(f32_box + swz(row, u)) = make_float4(xn[4 * u], xn[4 * u + 1], xn[4 * u + 2], xn[4 * u + 3]);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(xn[8 * u], xn[8 * u + 1]), h1 = __floats2bfloat162_rn(xn[8 * u + 2], xn[8 * u + 3]);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(xn[8 * u + 4], xn[8 * u + 5]), h3 = __floats2bfloat162_rn(xn[8 * u + 6], xn[8 * u + 7]);
+            uint4 w;
+            w.x = *reinterpret_cast<uint32_t*>(&h0);
+            w.y = *reinterpret_cast<uint32_t*>(&h1);
+            w.z = *reinterpret_cast<uint32_t*>(&h2);
+            w.w = *reinterpret_cast<uint32_t*>(&h3);
+            *reinterpret_cast<uint4*>(b16_box + swz(row, b16_u0 + u)) = w;
           }
         } else {
+          // bf16 outputs: bias + ReLU, ReLU mask, or plain conversion
+          float v[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
           if (p.epilogue == GEMM_EPI_BIAS_RELU_BF16) {
+            const float* bias = p.bias + (int64_t)q.z * p.stride_bias + q.n0 + c * 32;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j] + bias4[j], 0.f);
+            for (int j = 0; j < 32; ++j) {
+              const float bj = (q.n0 + c * 32 + j < p.N) ? bias[j] : 0.f;
+              v[j] = fmaxf(v[j] + bj, 0.f);
+            }
           } else if (p.epilogue == GEMM_EPI_MASK_BF16) {
-            const __nv_bfloat16* mk = static_cast<const __nv_bfloat16*>(p.mask) + (int64_t)z * p.stride_mask + (int64_t)m * p.ld_mask + n;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (n + j < p.N) v[j] = (__bfloat162float(mk[j]) > 0.f) ? v[j] : 0.f;
+            for (int u = 0; u < 4; ++u) {
+              const uint4 mk = *reinterpret_cast<const uint4*>(b16_box + swz(row, b16_u0 + u));
+              const __nv_bfloat162* mh = reinterpret_cast<const __nv_bfloat162*>(&mk);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 mf = __bfloat1622float2(mh[j]);
+                if (!(mf.x > 0.f)) v[8 * u + 2 * j] = 0.f;
+                if (!(mf.y > 0.f)) v[8 * u + 2 * j + 1] = 0.f;
+              }
+            }
           }
-          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.c) + zc + (int64_t)m * p.ldc + n;
-          if (full) {
-            __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
-            uint2 u;
-            u.x = *reinterpret_cast<uint32_t*>(&h0);
-            u.y = *reinterpret_cast<uint32_t*>(&h1);
-            *reinterpret_cast<uint2*>(out) = u;
-          } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (n + j < p.N) out[j] = __float2bfloat16_rn(v[j]);
+          for (int u = 0; u < 4; ++u) {
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(v[8 * u], v[8 * u + 1]), h1 = __floats2bfloat162_rn(v[8 * u + 2], v[8 * u + 3]);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * u + 4], v[8 * u + 5]), h3 = __floats2bfloat162_rn(v[8 * u + 6], v[8 * u + 7]);
+            uint4 w;
+            w.x = *reinterpret_cast<uint32_t*>(&h0);
+            w.y = *reinterpret_cast<uint32_t*>(&h1);
+            w.z = *reinterpret_cast<uint32_t*>(&h2);
+            w.w = *reinterpret_cast<uint32_t*>(&h3);
+            *reinterpret_cast<uint4*>(b16_box + swz(row, b16_u0 + u)) = w;
           }
         }
       }
+      // the accumulator has been read: hand it back to the MMA issuer (one arrival per warp)
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[b]);
+      // make the tile visible to the bulk-copy engine, then one thread stores it
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      epi_barrier();
+      if (leader) {
+        if (p.epilogue == GEMM_EPI_F32 || p.epilogue == GEMM_EPI_SGD) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            if (q.n0 + c * 32 < p.N) tma_store_3d(buf_f32 + c * 16384, &map_c, q.n0 + c * 32, q.m0, q.z);
+        }
+        if (p.epilogue != GEMM_EPI_F32) {
+          const CUtensorMap* mo = (p.epilogue == GEMM_EPI_SGD) ? &map_aux : &map_c;
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+            if (q.n0 + c * 64 < p.N) tma_store_3d(buf_b16 + c * 16384, mo, q.n0 + c * 64, q.m0, q.z);
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the buffers may be overwritten again
+        if (reads_tile) mbar_arrive(&in_free);
+      }
+      epi_barrier();
     }
+    if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores complete before the CTA exits
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -362,38 +405,78 @@ EncodeFn encode_fn() {
   return fn;
 }
 
+bool encode(CUtensorMap* map, CUtensorMapDataType dt, int esz, const void* base, int64_t inner, int64_t outer,
+            int64_t pitch_elems, int64_t batch, int64_t batch_stride_elems, int box_inner, int box_outer) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) || (pitch_elems * esz) % 16 != 0) return false;
+  if (batch > 1 && (batch_stride_elems * esz) % 16 != 0) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)(batch < 1 ? 1 : batch)};
+  cuuint64_t strides[2] = {(cuuint64_t)pitch_elems * esz,
+                           (cuuint64_t)(batch > 1 ? batch_stride_elems : pitch_elems * outer) * esz};
+  cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool make_operand_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t pitch_elems, int64_t batch,
                       int64_t batch_stride_elems) {
-  EncodeFn fn = encode_fn();
-  if (!fn) return false;
-  if ((reinterpret_cast<uintptr_t>(base) & 15u) || (pitch_elems * 2) % 16 != 0) return false;
-  if (batch > 1 && (batch_stride_elems * 2) % 16 != 0) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)(batch < 1 ? 1 : batch)};
-  cuuint64_t strides[2] = {(cuuint64_t)pitch_elems * 2,
-                           (cuuint64_t)(batch > 1 ? batch_stride_elems : pitch_elems * outer) * 2};
-  cuuint32_t box[3] = {64, 64, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, inner, outer, pitch_elems, batch, batch_stride_elems, 64, 64);
+}
+
+bool make_tile_map_f32(CUtensorMap* map, const void* base, int64_t N, int64_t M, int64_t pitch_elems, int64_t batch,
+                       int64_t batch_stride_elems) {
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, N, M, pitch_elems, batch, batch_stride_elems, 32, 128);
+}
+
+bool make_tile_map_bf16(CUtensorMap* map, const void* base, int64_t N, int64_t M, int64_t pitch_elems, int64_t batch,
+                        int64_t batch_stride_elems) {
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, N, M, pitch_elems, batch, batch_stride_elems, 64, 128);
 }
 
 cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmShape& p, cudaStream_t s) {
   static bool attr_set = false;
+  static int sms = 0;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(bgemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
     attr_set = true;
   }
-  GemmShape q = p;
-  const int64_t esz = (p.epilogue == GEMM_EPI_F32 || p.epilogue == GEMM_EPI_SGD) ? 4 : 2;
-  const void* cbase = p.epilogue == GEMM_EPI_SGD ? static_cast<const void*>(p.x_upd) : p.c;
-  q.vec_ok = ((reinterpret_cast<uintptr_t>(cbase) & 15u) == 0 && (p.ldc * esz) % 16 == 0 && (p.stride_c * esz) % 16 == 0) ? 1 : 0;
-  dim3 grid((unsigned)((p.N + BN - 1) / BN), (unsigned)((p.M + BM - 1) / BM), (unsigned)p.batch);
-  bgemm_bf16_kernel<<<grid, kThreads, kSmemBytes, s>>>(map_a, map_b, q);
+  // Tensor maps of the epilogue: map_c is C (fp32 or bf16) -- for the fused SGD step the parameter block
+  // itself, loaded and stored; map_aux is the ReLU mask (input) or the bf16 copy of the parameters (output).
+  CUtensorMap map_c, map_aux;
+  bool ok = true;
+  const int64_t nb = p.batch;
+  switch (p.epilogue) {
+    case GEMM_EPI_F32:
+      ok = make_tile_map_f32(&map_c, p.c, p.N, p.M, p.ldc, nb, p.stride_c);
+      map_aux = map_c;
+      break;
+    case GEMM_EPI_SGD:
+      ok = make_tile_map_f32(&map_c, p.x_upd, p.N, p.M, p.ldc, nb, p.stride_c) &&
+           make_tile_map_bf16(&map_aux, p.x_shadow, p.N, p.M, p.ldc, nb, p.stride_c);
+      break;
+    case GEMM_EPI_MASK_BF16:
+      ok = make_tile_map_bf16(&map_c, p.c, p.N, p.M, p.ldc, nb, p.stride_c) &&
+           make_tile_map_bf16(&map_aux, p.mask, p.N, p.M, p.ld_mask, nb, p.stride_mask);
+      break;
+    default:
+      ok = make_tile_map_bf16(&map_c, p.c, p.N, p.M, p.ldc, nb, p.stride_c);
+      map_aux = map_c;
+      break;
+  }
+  if (!ok) return cudaErrorInvalidValue;
+  const int64_t tiles = (int64_t)((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM) * p.batch;
+  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+  bgemm_bf16_kernel<<<grid, kThreads, kSmemBytes, s>>>(map_a, map_b, map_c, map_aux, p);
   return cudaGetLastError();
 }
 

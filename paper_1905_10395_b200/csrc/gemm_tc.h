@@ -19,7 +19,6 @@ struct GemmShape {
   int a_mn, b_mn;               // 1: the M (resp. N) index is contiguous in memory, 0: the K index is
   int a_batched, b_batched;     // 0: every batch entry reads batch 0 of that operand
   int epilogue;
-  int vec_ok;                   // set by the launcher: C rows allow 16-byte stores
   void* c;                      // [batch][M][ldc]
   int64_t ldc, stride_c;        // in elements of C
   const float* bias;            // [batch][N] fp32 (stride_bias apart)
@@ -37,6 +36,12 @@ struct GemmShape {
 // K-major operand: inner = K, outer = M or N.  MN-major operand: inner = M or N, outer = K.
 bool make_operand_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t pitch_elems,
                       int64_t batch, int64_t batch_stride_elems);
+
+// Tile maps of the epilogue (128-row boxes, 128 bytes wide): fp32 {32, 128, 1}, bf16 {64, 128, 1}.
+bool make_tile_map_f32(CUtensorMap* map, const void* base, int64_t N, int64_t M, int64_t pitch_elems, int64_t batch,
+                       int64_t batch_stride_elems);
+bool make_tile_map_bf16(CUtensorMap* map, const void* base, int64_t N, int64_t M, int64_t pitch_elems, int64_t batch,
+                        int64_t batch_stride_elems);
 
 cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmShape& p, cudaStream_t s);
 
