@@ -261,7 +261,8 @@ def run_ours(args):
         pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith)
     else:
         w = inputs.config(spec["cfg"], tau=spec["tau"])
-        pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith)
+        pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith,
+                         flags=api.FLAG_MLP_FUSED_STEP if args.mlp_fused_step else 0)
     launches_per_step = lambda t: spec["launches"][0] if t % spec["tau"] == 0 else spec["launches"][1]
     torch.cuda.synchronize(dev)
 
@@ -392,6 +393,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--sample-cols", type=int, default=0)
     ap.add_argument("--d", type=int, default=0, help="shrink the c4 workload (profiler captures on a small case)")
+    ap.add_argument("--mlp-fused-step", action="store_true", help="c3: LSGD_FLAG_MLP_FUSED_STEP")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -131,13 +131,13 @@ typedef struct {
   uint32_t flags;            /* bit set of LSGD_FLAG_*; 0 = defaults                                 */
 } lsgd_config;
 
-/* MLP objective: keep the weight gradients materialised in g on every step.  By default, on steps that
- * are not pull steps, lsgd_grad applies x <- x - eta g for W1 and W2 inside the epilogue of the
- * weight-gradient products (same arithmetic, bit-identical result; g is then not written for those
- * two blocks and lsgd_step only finishes the biases and W3).  With that default, lsgd_grad may be
- * called once per step and lsgd_elect(h, NULL) must not be called between lsgd_grad and lsgd_step on a
- * non-pull step (LSGD_ERR_STATE): the parameters are already partly advanced.                       */
-#define LSGD_FLAG_MLP_KEEP_GRADIENTS 1u
+/* MLP objective: on steps that are not pull steps, let lsgd_grad apply x <- x - eta g for W1 and W2
+ * inside the epilogue of the weight-gradient products (same arithmetic, bit-identical result; g is then
+ * not written for those two blocks and lsgd_step only finishes the biases and W3).  With this flag,
+ * lsgd_grad may be called once per step and lsgd_elect(h, NULL) must not be called between lsgd_grad
+ * and lsgd_step on a non-pull step (LSGD_ERR_STATE): the parameters are already partly advanced.
+ * Off by default: the separate update kernel is currently the faster path.                          */
+#define LSGD_FLAG_MLP_FUSED_STEP 1u
 
 /* Validates the configuration on the host, copies the group map, builds the group tables and
  * allocates O(P + G) words of device state plus reduction scratch for the objective's election

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "liblsgd.so")
  ERR_TOO_LARGE) = range(9)
 OBJ_EXTERNAL, OBJ_QUADRATIC, OBJ_MATCOMP, OBJ_MLP = range(4)
 ARITH_FP64, ARITH_FP64_FMA, ARITH_FP32 = range(3)
-FLAG_MLP_KEEP_GRADIENTS = 1
+FLAG_MLP_FUSED_STEP = 1
 
 
 class LsgdError(RuntimeError):

@@ -4,8 +4,8 @@
 // Persistent kernel, one CTA per SM, tiles of 128 x 128 handed out round-robin (tile = CTA, CTA +
 // grid, ...), three roles:
 //   * warp 0 (one thread): TMA producer.  cp.async.bulk.tensor loads of the operands (128-byte swizzle)
-//     into a 3-stage shared-memory ring guarded by mbarriers; each stage holds a 128 x 64 slice of A
-//     and of B.  For epilogues that read a tile (the parameters x for the fused SGD step, the ReLU
+//     into a shared-memory ring (2 to 6 stages, see kSmemBytes) guarded by mbarriers; each stage holds a
+//     128 x 64 slice of A and of B.  For epilogues that read a tile (the parameters x for the fused SGD step, the ReLU
 //     mask) it also loads that tile into the epilogue buffer.
 //   * warp 1 (one thread): issues tcgen05.mma (M = 128, N = 128, K = 16, cta_group::1) into one of TWO
 //     fp32 accumulator tiles in tensor memory (2 x 128 columns), so the products of tile i+1 overlap
@@ -35,13 +35,18 @@ namespace lsgd {
 namespace {
 
 constexpr int BM = 128, BN = 128, BK = 64;
-constexpr int kStages = 3;
+constexpr int kMaxStages = 6;
 constexpr int kStageBytes = (BM * BK + BN * BK) * 2;       // 32 KiB
 constexpr int kABytes = BM * BK * 2;                        // 16 KiB
 constexpr int kEpiF32Bytes = BM * BN * 4;                   // 64 KiB: fp32 tile, 4 boxes of [128][32 floats]
 constexpr int kEpiBf16Bytes = BM * BN * 2;                  // 32 KiB: bf16 tile, 2 boxes of [128][64 bf16]
 constexpr int kThreads = 192;                               // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
-constexpr int kSmemBytes = kStages * kStageBytes + kEpiF32Bytes + kEpiBf16Bytes + 1024;
+// Shared memory is carved per epilogue kind (224 KiB + alignment slack in every case):
+//   bf16 outputs      : 6 operand stages + 1 bf16 tile
+//   fp32 output       : 5 operand stages + 1 fp32 tile
+//   fused SGD step    : 2 operand stages (these products have K <= 128) + 2 fp32 tiles (the x tile of the
+//                       next tile is loaded while the current one is updated) + 1 bf16 tile
+constexpr int kSmemBytes = 224 * 1024 + 1024;
 constexpr uint32_t kTmemCols = 256;                         // two accumulator tiles
 constexpr long long kWaitBudgetCycles = 2000000000LL;       // about one second
 
@@ -146,9 +151,12 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                   const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_aux, GemmShape p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* buf_f32 = smem + kStages * kStageBytes;          // fp32 tile: C out, or x in/out (SGD)
-  uint8_t* buf_b16 = buf_f32 + kEpiF32Bytes;                // bf16 tile: C out, mask in, or bf16 copy of x out
-  __shared__ uint64_t full_bar[kStages], empty_bar[kStages], acc_full[2], acc_empty[2], in_full, in_free;
+  const bool sgd = (p.epilogue == GEMM_EPI_SGD);
+  const int kStages = sgd ? 2 : (p.epilogue == GEMM_EPI_F32 ? 5 : 6);
+  const int nx = sgd ? 2 : 1;                               // input-tile buffers (x is double-buffered)
+  uint8_t* buf_f32_0 = smem + kStages * kStageBytes;        // fp32 tile(s): C out, or x in/out (SGD)
+  uint8_t* buf_b16 = buf_f32_0 + (sgd ? 2 : (p.epilogue == GEMM_EPI_F32 ? 1 : 0)) * kEpiF32Bytes;   // bf16 tile: C out, mask in, bf16 x out
+  __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2], in_full[2], in_free[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
 
@@ -168,8 +176,10 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       mbar_init(&acc_full[b], 1);
       mbar_init(&acc_empty[b], 4);      // one arrival per epilogue warp
     }
-    mbar_init(&in_full, 1);
-    mbar_init(&in_free, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&in_full[b], 1);
+      mbar_init(&in_free[b], 1);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
@@ -220,16 +230,19 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       }
       if (ok && reads_tile) {
         // the epilogue's input tile, once the previous tile's stores have finished reading the buffers
-        ok = mbar_wait(&in_free, (local & 1) ^ 1, abort_flag, p.status);
+        const int xb = local % nx;
+        const int use = local / nx;       // how often this buffer has been used before
+        ok = mbar_wait(&in_free[xb], (use & 1) ^ 1, abort_flag, p.status);
         if (!ok) break;
-        if (p.epilogue == GEMM_EPI_SGD) {
-          mbar_expect_tx(&in_full, kEpiF32Bytes);
+        if (sgd) {
+          uint8_t* dst = buf_f32_0 + xb * kEpiF32Bytes;
+          mbar_expect_tx(&in_full[xb], kEpiF32Bytes);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tma_load_3d(buf_f32 + c * 16384, &map_c, &in_full, q.n0 + c * 32, q.m0, q.z);
+          for (int c = 0; c < 4; ++c) tma_load_3d(dst + c * 16384, &map_c, &in_full[xb], q.n0 + c * 32, q.m0, q.z);
         } else {
-          mbar_expect_tx(&in_full, kEpiBf16Bytes);
+          mbar_expect_tx(&in_full[xb], kEpiBf16Bytes);
 #pragma unroll
-          for (int c = 0; c < 2; ++c) tma_load_3d(buf_b16 + c * 16384, &map_aux, &in_full, q.n0 + c * 64, q.m0, q.z);
+          for (int c = 0; c < 2; ++c) tma_load_3d(buf_b16 + c * 16384, &map_aux, &in_full[xb], q.n0 + c * 64, q.m0, q.z);
         }
       }
     }
@@ -273,8 +286,19 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const Tile q = tile_of(t, mt, nt);
       const int b = local & 1;
       ok = mbar_wait(&acc_full[b], (local >> 1) & 1, abort_flag, p.status);
-      if (ok && reads_tile) ok = mbar_wait(&in_full, local & 1, abort_flag, p.status);
+      const int xb = local % nx;
+      if (ok && reads_tile) ok = mbar_wait(&in_full[xb], (local / nx) & 1, abort_flag, p.status);
       if (!ok) break;
+      uint8_t* buf_f32 = buf_f32_0 + xb * kEpiF32Bytes;
+      if (nx == 2) {
+        // double-buffered input: the previous tile's stores were left in flight; before the shared bf16
+        // tile is overwritten they must have been read, and then the previous x buffer is free again
+        if (leader) {
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          if (local > 0) mbar_arrive(&in_free[xb ^ 1]);
+        }
+        epi_barrier();
+      }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t tacc = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * BN);
 #pragma unroll 1
@@ -374,10 +398,12 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             if (q.n0 + c * 64 < p.N) tma_store_3d(buf_b16 + c * 16384, mo, q.n0 + c * 64, q.m0, q.z);
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the buffers may be overwritten again
-        if (reads_tile) mbar_arrive(&in_free);
+        if (nx == 1) {
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the buffers may be overwritten again
+          if (reads_tile) mbar_arrive(&in_free[0]);
+        }
       }
-      epi_barrier();
+      if (nx == 1) epi_barrier();
     }
     if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores complete before the CTA exits
   }

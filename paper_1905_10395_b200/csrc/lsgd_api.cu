@@ -198,7 +198,7 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
     case LSGD_OBJ_MLP: {
       if (!batch) return LSGD_ERR_INVALID_ARG;
       if (h->fused_applied) return LSGD_ERR_STATE;   // the pending gradient has already moved W1, W2
-      const bool fuse = (h->t % c.tau) != 0 && !(c.flags & LSGD_FLAG_MLP_KEEP_GRADIENTS);
+      const bool fuse = (h->t % c.tau) != 0 && (c.flags & LSGD_FLAG_MLP_FUSED_STEP);
       lsgd_status st = mlp_grad(h, static_cast<const int32_t*>(batch), fuse);
       if (st != LSGD_OK) return st;
       h->fused_applied = fuse;

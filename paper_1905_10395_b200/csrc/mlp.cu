@@ -107,7 +107,8 @@ __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
 }
 
 constexpr int kHeadWarps = 8;
-constexpr int kHeadSamplesPerWarp = 1;   // a CTA covers 8 samples and stages W3 once in shared memory
+// A CTA stages W3 once in shared memory and covers 8 x samples_per_warp samples: 1 sample per warp for a
+// training batch (parallelism), 8 for the large held-out batch (amortise the staging).
 
 // Last layer forward.  One warp per sample: logits Z = H2 W3^T + b3 from 16-byte (8 x bf16) loads, the
 // softmax cross-entropy of the sample, and (training) dZ = (p - onehot) / n rounded to bf16.
@@ -115,7 +116,7 @@ __global__ void __launch_bounds__(kHeadWarps * 32)
 head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ x,
                     const int32_t* __restrict__ labels, const int32_t* __restrict__ label_idx, float* __restrict__ dz,
                     float* __restrict__ loss_b, int32_t n, int32_t d2, int32_t C, int64_t ld, int64_t w3_off, int64_t b3_off,
-                    int32_t label_rows, uint32_t* status) {
+                    int32_t label_rows, int32_t samples_per_warp, uint32_t* status) {
   extern __shared__ uint4 s_w3[];   // [C][d2 / 8]
   const int i = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -124,8 +125,8 @@ head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* _
   for (int t = threadIdx.x; t < C * chunks; t += blockDim.x) s_w3[t] = w3[t];
   __syncthreads();
   const float* b3 = x + (int64_t)i * ld + b3_off;
-  for (int sidx = 0; sidx < kHeadSamplesPerWarp; ++sidx) {
-    const int b = (blockIdx.x * kHeadWarps + warp) * kHeadSamplesPerWarp + sidx;
+  for (int sidx = 0; sidx < samples_per_warp; ++sidx) {
+    const int b = (blockIdx.x * kHeadWarps + warp) * samples_per_warp + sidx;
     if (b >= n) break;
     const uint4* h = reinterpret_cast<const uint4*>(h2 + ((int64_t)i * n + b) * d2);
     float acc[kMaxClasses];
@@ -404,10 +405,11 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   lsgd_status fs = forward_hidden(h, st->m_xb, 1, B, st->h1, st->m_h1, st->h2);
   if (fs != LSGD_OK) return fs;
 
-  const int per_cta = kHeadWarps * kHeadSamplesPerWarp;
+  const int spw = B > 256 ? 8 : 1;
+  const int per_cta = kHeadWarps * spw;
   const size_t w3_smem = (size_t)d[3] * d[2] * 2;
   head_forward_kernel<<<dim3((B + per_cta - 1) / per_cta, P), kHeadWarps * 32, w3_smem, s>>>(st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2],
-                                                          d[3], ld, st->L.w[2], st->L.b[2], m.pool, h->d_status);
+                                                          d[3], ld, st->L.w[2], st->L.b[2], m.pool, spw, h->d_status);
   const size_t bwd_smem = sizeof(float) * ((size_t)B * d[3] + (size_t)kBwdSlices * (d[3] + 1) * kBwdCols);
   head_backward_kernel<<<dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdCols, kBwdSlices), bwd_smem, s>>>(
       st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]);
@@ -445,10 +447,11 @@ lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss) {
   const int32_t* d = st->dims;
   lsgd_status fs = forward_hidden(h, st->m_xh, 0, st->nH, st->hh1, st->m_hh1, st->hh2);
   if (fs != LSGD_OK) return fs;
-  const int per_cta = kHeadWarps * kHeadSamplesPerWarp;
+  const int spw = st->nH > 256 ? 8 : 1;
+  const int per_cta = kHeadWarps * spw;
   head_forward_kernel<<<dim3((st->nH + per_cta - 1) / per_cta, st->P), kHeadWarps * 32, (size_t)d[3] * d[2] * 2, h->stream>>>(st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr,
                                                                           st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2],
-                                                                          st->L.b[2], st->nH, h->d_status);
+                                                                          st->L.b[2], st->nH, spw, h->d_status);
   row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_h, loss, st->nH);
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
 }

@@ -154,14 +154,14 @@ def test_config3_single_steps_from_the_oracle_state():
 
 
 def test_fused_weight_step_is_bit_identical_to_the_materialised_gradient_path():
-    """On non-pull steps the plain step of W1, W2 is taken inside the weight-gradient products; it must
-    give exactly the parameters of the path that writes g and updates afterwards."""
+    """With LSGD_FLAG_MLP_FUSED_STEP the plain step of W1, W2 is taken inside the weight-gradient products
+    on non-pull steps; it must give exactly the parameters of the path that writes g and updates afterwards."""
     from paper_1905_10395_b200 import api
     from paper_1905_10395_b200.runner import Population
     w = inputs.make_mlp(3, 1, dims=(40, 72, 136, 7), pool=256, heldout=40, batch=24, n_classes=7, steps=7, tau=3,
                         config_id=82)
-    a = Population(w)
-    b = Population(w, flags=api.FLAG_MLP_KEEP_GRADIENTS)
+    a = Population(w, flags=api.FLAG_MLP_FUSED_STEP)
+    b = Population(w)
     a.run(7)
     b.run(7)
     xa, xb = a.x_host(), b.x_host()
