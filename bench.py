@@ -262,7 +262,7 @@ def run_ours(args):
     else:
         w = inputs.config(spec["cfg"], tau=spec["tau"])
         pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith,
-                         flags=api.FLAG_MLP_FUSED_STEP if args.mlp_fused_step else 0)
+                         flags=0 if args.mlp_unfused_step else api.FLAG_MLP_FUSED_STEP)
     launches_per_step = lambda t: spec["launches"][0] if t % spec["tau"] == 0 else spec["launches"][1]
     torch.cuda.synchronize(dev)
 
@@ -327,7 +327,8 @@ def run_ours(args):
                    "arithmetic": ["fp64 unfused", "fp64 fma", "fp32 fma"][args.arith],
                    "l2": ("per-step inputs exceed the 126 MB L2; no flush between steps" if P * d * 8 > 3e8 else
                           "working set fits in L2; steps run back to back as in training (no flush)"),
-                   "multi_gpu": "replicas only"},
+                   "multi_gpu": "replicas only",
+                   **({"mlp_fused_step": not args.mlp_unfused_step} if spec["kind"] == "mlp" else {})},
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
                      "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
@@ -393,7 +394,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--sample-cols", type=int, default=0)
     ap.add_argument("--d", type=int, default=0, help="shrink the c4 workload (profiler captures on a small case)")
-    ap.add_argument("--mlp-fused-step", action="store_true", help="c3: LSGD_FLAG_MLP_FUSED_STEP")
+    ap.add_argument("--mlp-unfused-step", action="store_true", help="c3: do not set LSGD_FLAG_MLP_FUSED_STEP")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -106,17 +106,19 @@ __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
   }
 }
 
+// A CTA stages W3 once in shared memory.  A warp takes S samples at a time, so each unpacked 16-byte piece
+// of W3 is used S times: S = 1 for a training batch (most parallelism), S = 4 for the large held-out batch
+// (the kernel is bound by unpacking W3, not by reading H2).
 constexpr int kHeadWarps = 8;
-// A CTA stages W3 once in shared memory and covers 8 x samples_per_warp samples: 1 sample per warp for a
-// training batch (parallelism), 8 for the large held-out batch (amortise the staging).
 
-// Last layer forward.  One warp per sample: logits Z = H2 W3^T + b3 from 16-byte (8 x bf16) loads, the
-// softmax cross-entropy of the sample, and (training) dZ = (p - onehot) / n rounded to bf16.
+// Last layer forward: logits Z = H2 W3^T + b3 from 16-byte (8 x bf16) loads, the softmax cross-entropy of
+// each sample, and (training) dZ = (p - onehot) / n rounded to bf16.
+template <int S>
 __global__ void __launch_bounds__(kHeadWarps * 32)
 head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ x,
                     const int32_t* __restrict__ labels, const int32_t* __restrict__ label_idx, float* __restrict__ dz,
                     float* __restrict__ loss_b, int32_t n, int32_t d2, int32_t C, int64_t ld, int64_t w3_off, int64_t b3_off,
-                    int32_t label_rows, int32_t samples_per_warp, uint32_t* status) {
+                    int32_t label_rows, int32_t groups_per_warp, uint32_t* status) {
   extern __shared__ uint4 s_w3[];   // [C][d2 / 8]
   const int i = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -125,65 +127,79 @@ head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* _
   for (int t = threadIdx.x; t < C * chunks; t += blockDim.x) s_w3[t] = w3[t];
   __syncthreads();
   const float* b3 = x + (int64_t)i * ld + b3_off;
-  for (int sidx = 0; sidx < samples_per_warp; ++sidx) {
-    const int b = (blockIdx.x * kHeadWarps + warp) * samples_per_warp + sidx;
-    if (b >= n) break;
-    const uint4* h = reinterpret_cast<const uint4*>(h2 + ((int64_t)i * n + b) * d2);
-    float acc[kMaxClasses];
+  for (int grp = 0; grp < groups_per_warp; ++grp) {
+    const int b0 = ((blockIdx.x * kHeadWarps + warp) * groups_per_warp + grp) * S;
+    if (b0 >= n) break;
+    float acc[S][kMaxClasses];
 #pragma unroll
-    for (int c = 0; c < kMaxClasses; ++c) acc[c] = 0.f;
+    for (int sx = 0; sx < S; ++sx)
+#pragma unroll
+      for (int c = 0; c < kMaxClasses; ++c) acc[sx][c] = 0.f;
     for (int ch = lane; ch < chunks; ch += 32) {
-      float hv[8];
-      unpack8(h[ch], hv);
+      float hv[S][8];
+#pragma unroll
+      for (int sx = 0; sx < S; ++sx) {
+        const int b = b0 + sx < n ? b0 + sx : n - 1;
+        unpack8(reinterpret_cast<const uint4*>(h2 + ((int64_t)i * n + b) * d2)[ch], hv[sx]);
+      }
 #pragma unroll
       for (int c = 0; c < kMaxClasses; ++c)
         if (c < C) {
           float wv[8];
           unpack8(s_w3[c * chunks + ch], wv);
 #pragma unroll
-          for (int j = 0; j < 8; ++j) acc[c] = fmaf(hv[j], wv[j], acc[c]);
+          for (int sx = 0; sx < S; ++sx)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[sx][c] = fmaf(hv[sx][j], wv[j], acc[sx][c]);
         }
     }
 #pragma unroll
-    for (int c = 0; c < kMaxClasses; ++c)
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xFFFFFFFFu, acc[c], o);
-    if (lane == 0) {
-      int y = label_idx ? label_idx[(int64_t)i * n + b] : b;   // training: pool row of this sample
-      if (y < 0 || y >= label_rows) {
-        atomicOr(status, FLAG_BAD_INDEX);
-        y = 0;
-      }
-      int cls = labels[y];
-      if (cls < 0 || cls >= C) {
-        atomicOr(status, FLAG_BAD_INDEX);
-        cls = 0;
-      }
-      float zmax = -INFINITY;
+    for (int sx = 0; sx < S; ++sx)
 #pragma unroll
       for (int c = 0; c < kMaxClasses; ++c)
-        if (c < C) {
-          acc[c] += b3[c];
-          zmax = fmaxf(zmax, acc[c]);
-        }
-      float sum = 0.f, zy = 0.f;
 #pragma unroll
-      for (int c = 0; c < kMaxClasses; ++c)
-        if (c < C) {
-          sum += expf(acc[c] - zmax);
-          if (c == cls) zy = acc[c];
+        for (int o = 16; o > 0; o >>= 1) acc[sx][c] += __shfl_xor_sync(0xFFFFFFFFu, acc[sx][c], o);
+    // lane sx finishes sample b0 + sx (every lane holds all the reduced sums)
+#pragma unroll
+    for (int sx = 0; sx < S; ++sx) {
+      const int b = b0 + sx;
+      if (lane == sx && b < n) {
+        int y = label_idx ? label_idx[(int64_t)i * n + b] : b;   // training: pool row of this sample
+        if (y < 0 || y >= label_rows) {
+          atomicOr(status, FLAG_BAD_INDEX);
+          y = 0;
         }
-      const float lse = zmax + logf(sum);
-      loss_b[(int64_t)i * n + b] = lse - zy;
-      if (dz) {
-        const float inv_n = 1.f / (float)n;
+        int cls = labels[y];
+        if (cls < 0 || cls >= C) {
+          atomicOr(status, FLAG_BAD_INDEX);
+          cls = 0;
+        }
+        float zmax = -INFINITY;
 #pragma unroll
         for (int c = 0; c < kMaxClasses; ++c)
           if (c < C) {
-            const float pc = expf(acc[c] - lse);
-            const float v = (pc - (c == cls ? 1.f : 0.f)) * inv_n;
-            dz[((int64_t)i * n + b) * C + c] = __bfloat162float(__float2bfloat16_rn(v));
+            acc[sx][c] += b3[c];
+            zmax = fmaxf(zmax, acc[sx][c]);
           }
+        float sum = 0.f, zy = 0.f;
+#pragma unroll
+        for (int c = 0; c < kMaxClasses; ++c)
+          if (c < C) {
+            sum += expf(acc[sx][c] - zmax);
+            if (c == cls) zy = acc[sx][c];
+          }
+        const float lse = zmax + logf(sum);
+        loss_b[(int64_t)i * n + b] = lse - zy;
+        if (dz) {
+          const float inv_n = 1.f / (float)n;
+#pragma unroll
+          for (int c = 0; c < kMaxClasses; ++c)
+            if (c < C) {
+              const float pc = expf(acc[sx][c] - lse);
+              const float v = (pc - (c == cls ? 1.f : 0.f)) * inv_n;
+              dz[((int64_t)i * n + b) * C + c] = __bfloat162float(__float2bfloat16_rn(v));
+            }
+        }
       }
     }
   }
@@ -405,11 +421,10 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   lsgd_status fs = forward_hidden(h, st->m_xb, 1, B, st->h1, st->m_h1, st->h2);
   if (fs != LSGD_OK) return fs;
 
-  const int spw = B > 256 ? 8 : 1;
-  const int per_cta = kHeadWarps * spw;
   const size_t w3_smem = (size_t)d[3] * d[2] * 2;
-  head_forward_kernel<<<dim3((B + per_cta - 1) / per_cta, P), kHeadWarps * 32, w3_smem, s>>>(st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2],
-                                                          d[3], ld, st->L.w[2], st->L.b[2], m.pool, spw, h->d_status);
+  head_forward_kernel<1><<<dim3((B + kHeadWarps - 1) / kHeadWarps, P), kHeadWarps * 32, w3_smem, s>>>(
+      st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], m.pool, 1,
+      h->d_status);
   const size_t bwd_smem = sizeof(float) * ((size_t)B * d[3] + (size_t)kBwdSlices * (d[3] + 1) * kBwdCols);
   head_backward_kernel<<<dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdCols, kBwdSlices), bwd_smem, s>>>(
       st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]);
@@ -447,11 +462,11 @@ lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss) {
   const int32_t* d = st->dims;
   lsgd_status fs = forward_hidden(h, st->m_xh, 0, st->nH, st->hh1, st->m_hh1, st->hh2);
   if (fs != LSGD_OK) return fs;
-  const int spw = st->nH > 256 ? 8 : 1;
-  const int per_cta = kHeadWarps * spw;
-  head_forward_kernel<<<dim3((st->nH + per_cta - 1) / per_cta, st->P), kHeadWarps * 32, (size_t)d[3] * d[2] * 2, h->stream>>>(st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr,
-                                                                          st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2],
-                                                                          st->L.b[2], st->nH, spw, h->d_status);
+  constexpr int kS = 4, kGroups = 2;   // 8 warps x 2 groups x 4 samples = 64 samples per CTA
+  const int per_cta = kHeadWarps * kGroups * kS;
+  head_forward_kernel<kS><<<dim3((st->nH + per_cta - 1) / per_cta, st->P), kHeadWarps * 32, (size_t)d[3] * d[2] * 2, h->stream>>>(
+      st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr, st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2], st->L.b[2], st->nH,
+      kGroups, h->d_status);
   row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_h, loss, st->nH);
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
 }
