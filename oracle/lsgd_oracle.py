@@ -338,3 +338,80 @@ class LsgdOracle:
         for _ in range(steps):
             self.step()
         return self.x
+
+
+# ----------------------------------------------------------------------------------------------
+# Algorithm 1 (the paper's asynchronous LSGD listing), run synchronously
+# ----------------------------------------------------------------------------------------------
+class Algorithm1Oracle:
+    """Algorithm 1 with all workers in lock-step (the sum of the workers' counters is then n l t, so
+    "n l tau divides the sum" reads "tau divides t").  State: x, t, and the leaders' parameters
+    x~^j (one per group) and x~ as COPIES taken when they are determined -- between communications
+    they are stale, as in the paper's description of the modification.
+
+      initialise:  x~^j, x~ <- parameters of the argmin workers at x_0
+      repeat:      g_i at x_i
+                   x_i <- x_i - eta g_i - eta (gamma/tau) (x_i - x~^{group(i)}) - eta (gamma_G/tau_G) (x_i - x~)
+                   t <- t + 1
+                   if tau   | t:  x~^j <- argmin inside each group (losses at the new x);  x_i <- x_i - eta lambda   (x_i - x~^j)
+                   if tau_G | t:  x~   <- argmin over all workers;                         x_i <- x_i - eta lambda_G (x_i - x~)
+
+    Readings: every pull is scaled by eta like the gradient (Section 3.1.1; the listing prints them
+    unscaled -- pass coefficient / eta to obtain that form).  One loss vector per communication,
+    evaluated after the gradient step, serves both elections of that communication."""
+
+    def __init__(self, x0, objective, group_of, G, eta, lambda_l, lambda_g, gamma_l, gamma_g, tau, tau_g):
+        assert tau >= 1 and tau_g >= 1
+        self.x = np.array(x0, dtype=F32, copy=True)
+        self.obj = objective
+        self.group_of = np.asarray(group_of, dtype=np.int32)
+        self.G = int(G)
+        self.eta = float(F32(eta))
+        self.lambda_l, self.lambda_g = float(F32(lambda_l)), float(F32(lambda_g))
+        self.gamma_l, self.gamma_g = float(F32(gamma_l)), float(F32(gamma_g))
+        self.tau, self.tau_g = int(tau), int(tau_g)
+        self.t = 0
+        self.n_elections = 0
+        self.history: List[dict] = []
+        loss = np.asarray(self.obj.loss(self.x, self.n_elections), dtype=F32)
+        self.n_elections += 1
+        self.ll, self.gl = elect(loss, self.group_of, self.G)
+        self.z_l = [self.x[int(l)].copy() for l in self.ll]      # x~^j
+        self.z_g = self.x[int(self.gl)].copy()                   # x~
+        self.history.append({"t": 0, "loss": loss.copy(), "ll": self.ll.copy(), "gl": self.gl})
+
+    def _pull(self, coef, target_of_worker):
+        for i in range(self.x.shape[0]):
+            xi = self.x[i].astype(F64)
+            self.x[i] = (xi - coef * (xi - target_of_worker(i).astype(F64))).astype(F32)
+
+    def step(self, forced_loss: Optional[np.ndarray] = None) -> None:
+        g = self.obj.grad(self.x, self.t)
+        cl = self.eta * (self.gamma_l / self.tau)
+        cg = self.eta * (self.gamma_g / self.tau_g)
+        for i in range(self.x.shape[0]):
+            xi = self.x[i].astype(F64)
+            new = xi - self.eta * g[i].astype(F64) - cl * (xi - self.z_l[int(self.group_of[i])].astype(F64)) \
+                - cg * (xi - self.z_g.astype(F64))
+            self.x[i] = new.astype(F32)
+        self.t += 1
+        local, glob = self.t % self.tau == 0, self.t % self.tau_g == 0
+        if local or glob:
+            loss = np.asarray(self.obj.loss(self.x, self.n_elections) if forced_loss is None else forced_loss, dtype=F32)
+            self.n_elections += 1
+            ll, gl = elect(loss, self.group_of, self.G)
+            if local:
+                self.ll = ll
+                self.z_l = [self.x[int(l)].copy() for l in ll]
+                self._pull(self.eta * self.lambda_l, lambda i: self.z_l[int(self.group_of[i])])
+            if glob:
+                self.gl = gl
+                self.z_g = self.x[int(gl)].copy()
+                self._pull(self.eta * self.lambda_g, lambda i: self.z_g)
+            self.history.append({"t": self.t, "loss": loss.copy(), "ll": self.ll.copy(), "gl": self.gl,
+                                 "local": local, "global": glob})
+
+    def run(self, steps: int) -> np.ndarray:
+        for _ in range(steps):
+            self.step()
+        return self.x
