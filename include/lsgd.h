@@ -129,6 +129,12 @@ typedef struct {
   void* stream;              /* cudaStream_t; NULL = the legacy default stream                       */
   int32_t arithmetic;        /* lsgd_arithmetic                                                      */
   uint32_t flags;            /* bit set of LSGD_FLAG_*; 0 = defaults                                 */
+  /* --- only read with LSGD_FLAG_ALGORITHM1 (see below) --- */
+  float gamma_l;             /* searching scope gamma: every step pulls with strength eta gamma / tau  */
+  float gamma_g;             /* gamma_G: every step pulls with strength eta gamma_G / tau_G           */
+  int32_t tau_g;             /* global communication period tau_G >= 1                               */
+  float* leader_copies;      /* DEVICE float[(G+1)*ld], 16-byte aligned: the leaders' parameters as of
+                                their last election (rows 0..G-1 local, row G global); library-written */
 } lsgd_config;
 
 /* MLP objective: on steps that are not pull steps, let lsgd_grad apply x <- x - eta g for W1 and W2
@@ -138,6 +144,19 @@ typedef struct {
  * and lsgd_step on a non-pull step (LSGD_ERR_STATE): the parameters are already partly advanced.
  * Off by default: the separate update kernel is currently the faster path.                          */
 #define LSGD_FLAG_MLP_FUSED_STEP 1u
+
+/* The schedule of the paper's Algorithm 1, run synchronously, instead of the fused Eq. (1) step:
+ *   lsgd_elect at t = 0          initialisation: both elections, leader parameters copied, no pull;
+ *   lsgd_grad, lsgd_step         x_i <- x_i - eta g_i - eta (gamma/tau)(x_i - x~^j) - eta (gamma_G/tau_G)(x_i - x~)
+ *                                where x~^j, x~ are the COPIES in leader_copies (stale between
+ *                                communications, as in the paper), then t <- t + 1;
+ *   lsgd_elect when tau | t or tau_G | t (t after the step; LSGD_ERR_STATE otherwise):
+ *                                if tau | t:   local leaders re-elected, x_i <- x_i - eta lambda (x_i - x~^j), copies refreshed;
+ *                                if tau_G | t: global leader re-elected, x_i <- x_i - eta lambda_G (x_i - x~), copy refreshed.
+ * All pulls are scaled by eta (Section 3.1.1; pass coefficient / eta for the unscaled form the listing
+ * prints).  One loss vector (given, or the objective's own loss at the current x) serves both
+ * elections of a communication.  LSGD_FLAG_MLP_FUSED_STEP is ignored in this mode.                  */
+#define LSGD_FLAG_ALGORITHM1 2u
 
 /* Validates the configuration on the host, copies the group map, builds the group tables and
  * allocates O(P + G) words of device state plus reduction scratch for the objective's election

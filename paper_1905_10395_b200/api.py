@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "liblsgd.so")
 OBJ_EXTERNAL, OBJ_QUADRATIC, OBJ_MATCOMP, OBJ_MLP = range(4)
 ARITH_FP64, ARITH_FP64_FMA, ARITH_FP32 = range(3)
 FLAG_MLP_FUSED_STEP = 1
+FLAG_ALGORITHM1 = 2
 
 
 class LsgdError(RuntimeError):
@@ -53,7 +54,8 @@ class Config(C.Structure):
                 ("d", C.c_int64), ("ld", C.c_int64), ("eta", C.c_float), ("lambda_l", C.c_float),
                 ("lambda_g", C.c_float), ("tau", C.c_int32), ("objective", C.c_int32),
                 ("objective_desc", C.c_void_p), ("x", C.c_void_p), ("g", C.c_void_p), ("stream", C.c_void_p),
-                ("arithmetic", C.c_int32), ("flags", C.c_uint32)]
+                ("arithmetic", C.c_int32), ("flags", C.c_uint32), ("gamma_l", C.c_float), ("gamma_g", C.c_float),
+                ("tau_g", C.c_int32), ("leader_copies", C.c_void_p)]
 
 
 _lib = None
@@ -169,7 +171,8 @@ def mlp_scratch_bytes(dims: Sequence[int], P: int, batch: int, n_heldout: int) -
 
 def make_config(*, P: int, G: int, group_of: np.ndarray, d: int, ld: int, eta: float, lambda_l: float,
                 lambda_g: float, tau: int, objective: int, desc=None, x=None, g=None, stream: int = 0,
-                arithmetic: int = ARITH_FP64, flags: int = 0):
+                arithmetic: int = ARITH_FP64, flags: int = 0, gamma_l: float = 0.0, gamma_g: float = 0.0,
+                tau_g: int = 1, leader_copies=None):
     """Returns (Config, keepalive) -- keepalive holds the host arrays the struct points to."""
     go = np.ascontiguousarray(group_of, dtype=np.int32)
     cfg = Config()
@@ -186,6 +189,8 @@ def make_config(*, P: int, G: int, group_of: np.ndarray, d: int, ld: int, eta: f
     cfg.stream = stream or None
     cfg.arithmetic = int(arithmetic)
     cfg.flags = int(flags)
+    cfg.gamma_l, cfg.gamma_g, cfg.tau_g = float(gamma_l), float(gamma_g), int(tau_g)
+    cfg.leader_copies = _ptr(leader_copies)
     return cfg, (go, desc)
 
 

@@ -57,9 +57,11 @@ __global__ void __launch_bounds__(kElectThreads) elect_kernel(ElectArgs p) {
     best = warp_min(best);
     if (lane == 0) {
       p.group_keys[j] = best;
-      const int l = (int)(uint32_t)best;
-      p.ll[j] = l;
-      atomicAdd(p.count_local + l, 1);
+      if (p.update_local) {
+        const int l = (int)(uint32_t)best;
+        p.ll[j] = l;
+        atomicAdd(p.count_local + l, 1);
+      }
     }
   }
   __syncthreads();
@@ -70,7 +72,7 @@ __global__ void __launch_bounds__(kElectThreads) elect_kernel(ElectArgs p) {
       best = k < best ? k : best;
     }
     best = warp_min(best);
-    if (lane == 0) {
+    if (lane == 0 && p.update_global) {
       const int l = (int)(uint32_t)best;
       *p.gl = l;
       atomicAdd(p.count_global + l, 1);
@@ -78,7 +80,31 @@ __global__ void __launch_bounds__(kElectThreads) elect_kernel(ElectArgs p) {
   }
 }
 
+// copies[r] <- the parameters of leader r (rows 0..G-1: local leaders, row G: the global leader)
+__global__ void __launch_bounds__(256)
+leader_copies_kernel(const float* __restrict__ x, float* __restrict__ copies, const int32_t* __restrict__ ll,
+                     const int32_t* __restrict__ gl, int32_t G, int32_t r0, int64_t n4, int64_t ld) {
+  const int r = r0 + blockIdx.y;
+  const int src = r < G ? ll[r] : *gl;
+  const float4* s4 = reinterpret_cast<const float4*>(x + (int64_t)src * ld);
+  float4* d4 = reinterpret_cast<float4*>(copies + (int64_t)r * ld);
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < n4; c += stride) d4[c] = s4[c];
+}
+
 }  // namespace
+
+cudaError_t launch_leader_copies(const float* x, float* copies, const int32_t* ll, const int32_t* gl, int32_t G, int32_t r0,
+                                 int32_t r1, int64_t d, int64_t ld, cudaStream_t s) {
+  if (r1 > G + 1) r1 = G + 1;
+  if (r1 <= r0) return cudaSuccess;
+  const int64_t n4 = (d + 3) / 4;
+  int64_t bx = (n4 + 255) / 256;
+  if (bx > 1184) bx = 1184;
+  dim3 grid((unsigned)bx, (unsigned)(r1 - r0));
+  leader_copies_kernel<<<grid, 256, 0, s>>>(x, copies, ll, gl, G, r0, n4, ld);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_elect(const ElectArgs& a, cudaStream_t s) {
   elect_kernel<<<1, kElectThreads, 0, s>>>(a);

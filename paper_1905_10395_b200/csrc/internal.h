@@ -47,6 +47,9 @@ struct UpdateArgs {
   GroupTables tab;
   const int32_t* ll;        // DEVICE int32[G]
   const int32_t* gl;        // DEVICE int32[1]
+  const float* snap;        // leaders' parameters as copies [(G+1)][ld] (rows 0..G-1 local, G global), or
+                            // nullptr = read the leader rows of x itself (staged before anything is written)
+  bool use_g;               // false: pure pull, the gradient term is dropped (g / noise are not read)
   Coef k;
   int arith;                // 0 fp64 unfused, 1 fp64 fma, 2 fp32 fma (see update.cu)
   uint32_t* status;
@@ -67,8 +70,13 @@ struct ElectArgs {
   unsigned long long* group_keys;  // DEVICE u64[G] scratch
   int32_t* count_global;    // DEVICE int32[P]
   int32_t* count_local;     // DEVICE int32[P]
+  bool update_local;        // write ll (and count)
+  bool update_global;       // write gl (and count)
 };
 cudaError_t launch_elect(const ElectArgs& a, cudaStream_t s);
+// copies[r] <- x[ll[r]] for r in [r0, min(r1, G)), and copies[G] <- x[gl] if r1 > G
+cudaError_t launch_leader_copies(const float* x, float* copies, const int32_t* ll, const int32_t* gl, int32_t G,
+                                 int32_t r0, int32_t r1, int64_t d, int64_t ld, cudaStream_t s);
 
 // Quadratic objective.
 cudaError_t launch_quadratic_grad(const float* x, float* g, const float* a, const float* b,

@@ -39,6 +39,11 @@ lsgd_status validate(const lsgd_config* c) {
       if (cnt[j] == 0) return LSGD_ERR_BAD_GROUPS;
   }
   if (c->arithmetic < LSGD_ARITH_FP64 || c->arithmetic > LSGD_ARITH_FP32) return LSGD_ERR_INVALID_ARG;
+  if (c->flags & LSGD_FLAG_ALGORITHM1) {
+    if (c->tau_g < 1 || !std::isfinite(c->gamma_l) || !std::isfinite(c->gamma_g)) return LSGD_ERR_INVALID_ARG;
+    if (!c->leader_copies) return LSGD_ERR_INVALID_ARG;
+    if (!aligned16(c->leader_copies)) return LSGD_ERR_ALIGNMENT;
+  }
   if (c->P > kMaxWorkers) return LSGD_ERR_UNSUPPORTED;
   if (c->ld % 32 != 0) return LSGD_ERR_ALIGNMENT;
   if (!c->x) return LSGD_ERR_INVALID_ARG;
@@ -75,6 +80,8 @@ lsgd_status validate(const lsgd_config* c) {
   }
   return LSGD_OK;
 }
+
+lsgd_status algorithm1_pulls(lsgd_ctx* h, bool local, bool glob);
 
 GroupTables tables(const lsgd_ctx* h) { return GroupTables{h->d_rows_by_group, h->d_group_start, h->d_group_of}; }
 
@@ -198,7 +205,7 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
     case LSGD_OBJ_MLP: {
       if (!batch) return LSGD_ERR_INVALID_ARG;
       if (h->fused_applied) return LSGD_ERR_STATE;   // the pending gradient has already moved W1, W2
-      const bool fuse = (h->t % c.tau) != 0 && (c.flags & LSGD_FLAG_MLP_FUSED_STEP);
+      const bool fuse = (h->t % c.tau) != 0 && (c.flags & LSGD_FLAG_MLP_FUSED_STEP) && !(c.flags & LSGD_FLAG_ALGORITHM1);
       lsgd_status st = mlp_grad(h, static_cast<const int32_t*>(batch), fuse);
       if (st != LSGD_OK) return st;
       h->fused_applied = fuse;
@@ -228,6 +235,16 @@ lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
   e.group_keys = h->d_group_keys;
   e.count_global = h->d_count_g;
   e.count_local = h->d_count_l;
+  e.update_local = true;
+  e.update_global = true;
+  const bool alg1 = (c.flags & LSGD_FLAG_ALGORITHM1) != 0;
+  const bool alg1_init = alg1 && h->n_elections == 0;
+  if (alg1 && !alg1_init) {
+    if (h->t == 0) return LSGD_ERR_STATE;                     // initialisation was already done
+    e.update_local = (h->t % c.tau) == 0;
+    e.update_global = (h->t % c.tau_g) == 0;
+    if (!e.update_local && !e.update_global) return LSGD_ERR_STATE;   // not a communication step
+  }
   if (!loss) {
     switch (c.objective) {
       case LSGD_OBJ_QUADRATIC:
@@ -258,20 +275,27 @@ lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
   }
   LSGD_CUDA(launch_elect(e, h->stream));
   h->n_elections++;
+  if (alg1_init) {
+    LSGD_CUDA(launch_leader_copies(c.x, c.leader_copies, h->d_ll, h->d_gl, c.G, 0, c.G + 1, c.d, c.ld, h->stream));
+  } else if (alg1) {
+    return algorithm1_pulls(h, e.update_local, e.update_global);
+  }
   return LSGD_OK;
 }
 
-lsgd_status lsgd_step(lsgd_handle h) {
-  if (!h) return LSGD_ERR_INVALID_ARG;
+}  // extern "C"
+
+namespace {
+
+UpdateArgs base_update_args(lsgd_ctx* h) {
   const lsgd_config& c = h->cfg;
-  const bool pull = (h->t % c.tau) == 0;
-  if (pull && h->n_elections == 0) return LSGD_ERR_STATE;
-  if (c.objective != LSGD_OBJ_EXTERNAL && !h->grad_ready) return LSGD_ERR_STATE;
   UpdateArgs a{};
   a.x = c.x;
   a.g = c.g;
   a.quad = QuadInline{h->quad.a, h->quad.b, h->armed_noise, h->quad.sigma};
   a.x_bf16 = (c.objective == LSGD_OBJ_MLP) ? mlp_weight_shadow(h) : nullptr;
+  a.snap = nullptr;
+  a.use_g = true;
   a.d = c.d;
   a.ld = c.ld;
   a.P = c.P;
@@ -289,7 +313,57 @@ lsgd_status lsgd_step(lsgd_handle h) {
   a.k.sigma_f = h->quad.sigma;
   a.arith = c.arithmetic;
   a.status = h->d_status;
+  a.pull = false;
+  return a;
+}
+
+void set_pull_coefficients(UpdateArgs& a, double cl, double cg) {
+  a.k.cl = cl;
+  a.k.cg = cg;
+  a.k.cl_f = (float)cl;
+  a.k.cg_f = (float)cg;
+}
+
+// Algorithm 1, communication part: pure pulls towards freshly elected leaders, in place.  A leader's
+// own pull is zero, so reading the leader rows of x while x is rewritten is exact.
+lsgd_status algorithm1_pulls(lsgd_ctx* h, bool local, bool glob) {
+  const lsgd_config& c = h->cfg;
+  if (local) {
+    UpdateArgs a = base_update_args(h);
+    a.pull = true;
+    a.use_g = false;
+    set_pull_coefficients(a, (double)c.eta * (double)c.lambda_l, 0.0);
+    LSGD_CUDA(launch_update(a, h->stream));
+    LSGD_CUDA(launch_leader_copies(c.x, c.leader_copies, h->d_ll, h->d_gl, c.G, 0, c.G, c.d, c.ld, h->stream));
+  }
+  if (glob) {
+    UpdateArgs a = base_update_args(h);
+    a.pull = true;
+    a.use_g = false;
+    set_pull_coefficients(a, 0.0, (double)c.eta * (double)c.lambda_g);
+    LSGD_CUDA(launch_update(a, h->stream));
+    LSGD_CUDA(launch_leader_copies(c.x, c.leader_copies, h->d_ll, h->d_gl, c.G, c.G, c.G + 1, c.d, c.ld, h->stream));
+  }
+  return LSGD_OK;
+}
+
+}  // namespace
+
+extern "C" lsgd_status lsgd_step(lsgd_handle h) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  const lsgd_config& c = h->cfg;
+  const bool alg1 = (c.flags & LSGD_FLAG_ALGORITHM1) != 0;
+  const bool pull = alg1 ? (c.gamma_l != 0.f || c.gamma_g != 0.f) : (h->t % c.tau) == 0;
+  if ((pull || alg1) && h->n_elections == 0) return LSGD_ERR_STATE;
+  if (c.objective != LSGD_OBJ_EXTERNAL && !h->grad_ready) return LSGD_ERR_STATE;
+  UpdateArgs a = base_update_args(h);
   a.pull = pull;
+  if (alg1 && pull) {
+    // small pulls towards the (stale) copies of the leaders' parameters
+    a.snap = c.leader_copies;
+    set_pull_coefficients(a, (double)c.eta * ((double)c.gamma_l / (double)c.tau),
+                          (double)c.eta * ((double)c.gamma_g / (double)c.tau_g));
+  }
   if (h->fused_applied) {
     // W1 and W2 were stepped inside lsgd_grad; finish the biases and the last layer
     int64_t ranges[4][2];
@@ -311,6 +385,8 @@ lsgd_status lsgd_step(lsgd_handle h) {
   h->armed_noise = nullptr;
   return LSGD_OK;
 }
+
+extern "C" {
 
 lsgd_status lsgd_destroy(lsgd_handle h) {
   if (!h) return LSGD_OK;

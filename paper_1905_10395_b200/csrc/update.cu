@@ -140,7 +140,8 @@ pull_update_kernel(UpdateArgs p, int64_t n4) {
     const int64_t col = c * 4;
     float* xc = p.x + col;
     const float* gc = (QUAD ? p.quad.noise : p.g) + col;
-    const float4 xg = ld4(xc + (int64_t)gl * ld);
+    const float* snap = p.snap;
+    const float4 xg = snap ? ld4_cached(snap + (int64_t)p.G * ld + col) : ld4(xc + (int64_t)gl * ld);
     float4 av, bv;
     if (QUAD) {
       av = ld4_cached(p.quad.a + col);
@@ -148,7 +149,7 @@ pull_update_kernel(UpdateArgs p, int64_t n4) {
     }
     for (int j = 0; j < p.G; ++j) {
       const int l = s_ll[j];
-      const float4 xl = (l == gl) ? xg : ld4(xc + (int64_t)l * ld);
+      const float4 xl = snap ? ld4_cached(snap + (int64_t)j * ld + col) : ((l == gl) ? xg : ld4(xc + (int64_t)l * ld));
       const int m1 = s_start[j + 1];
       for (int m = s_start[j]; m < m1; m += kPullRows) {
         float4 xs[kPullRows], gs[kPullRows];
@@ -158,8 +159,8 @@ pull_update_kernel(UpdateArgs p, int64_t n4) {
           if (m + u < m1) {
             const int i = s_rows[m + u];
             rows[u] = i;
-            xs[u] = (i == l) ? xl : ld4(xc + (int64_t)i * ld);
-            if (!QUAD || NOISE) gs[u] = ld4(gc + (int64_t)i * ld);
+            xs[u] = (!snap && i == l) ? xl : ld4(xc + (int64_t)i * ld);
+            if ((!QUAD || NOISE) && p.use_g) gs[u] = ld4(gc + (int64_t)i * ld);
           }
         }
 #pragma unroll
@@ -172,6 +173,7 @@ pull_update_kernel(UpdateArgs p, int64_t n4) {
               g.z = quad_g<MODE>(x.z, av.z, bv.z, g.z, k, NOISE);
               g.w = quad_g<MODE>(x.w, av.w, bv.w, g.w, k, NOISE);
             }
+            if (!p.use_g) g = make_float4(0.f, 0.f, 0.f, 0.f);   // pure pull: x - eta * 0 = x exactly
             float4 r;
             r.x = pull1<MODE>(x.x, g.x, xl.x, xg.x, k);
             r.y = pull1<MODE>(x.y, g.y, xl.y, xg.y, k);

@@ -15,7 +15,7 @@ from .inputs import Workload
 class Population:
     def __init__(self, w: Workload, *, fused_quadratic: bool = False, arithmetic: int = api.ARITH_FP64,
                  device: str = "cuda:0", x: Optional[torch.Tensor] = None, g: Optional[torch.Tensor] = None,
-                 upload_noise: bool = True, flags: int = 0):
+                 upload_noise: bool = True, flags: int = 0, algorithm1: Optional[dict] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.w = w
@@ -75,10 +75,18 @@ class Population:
                 self.g = torch.empty_like(self.x)
         else:
             raise ValueError(w.objective)
+        extra = {}
+        self.alg1 = algorithm1
+        if algorithm1 is not None:
+            # the paper's Algorithm 1 schedule: dict(gamma_l=, gamma_g=, tau_g=)
+            self.leader_copies = torch.zeros((w.G + 1, w.ld), dtype=torch.float32, device=dev)
+            flags |= api.FLAG_ALGORITHM1
+            extra = dict(gamma_l=algorithm1["gamma_l"], gamma_g=algorithm1["gamma_g"], tau_g=algorithm1["tau_g"],
+                         leader_copies=self.leader_copies)
         cfg, keep = api.make_config(P=w.P, G=w.G, group_of=w.group_of, d=w.d, ld=w.ld, eta=w.eta,
                                     lambda_l=w.lambda_l, lambda_g=w.lambda_g, tau=w.tau, objective=obj, desc=desc,
                                     x=self.x, g=self.g, stream=self.stream.cuda_stream, arithmetic=arithmetic,
-                                    flags=flags)
+                                    flags=flags, **extra)
         self._keep.append(keep)
         self.lsgd = api.Lsgd(cfg, keep)
         self.t = 0
@@ -86,7 +94,32 @@ class Population:
         self.history: List[dict] = []
 
     # one synchronous step, in the order gradient -> (election loss, election) -> update
+    def _elect(self, forced_loss, record):
+        if forced_loss is not None:
+            self.lsgd.elect(forced_loss)
+        elif self.loss_ring is not None:
+            self.lsgd.elect(self.loss_ring[self.n_elections % self.loss_ring.shape[0]])
+        else:
+            self.lsgd.elect(None)
+        self.n_elections += 1
+        if record:
+            ll, gl = self.lsgd.leaders()
+            self.history.append({"t": self.t, "ll": ll, "gl": gl, "loss": self.lsgd.loss()})
+
+    def _step_algorithm1(self, forced_loss, record):
+        # initialise the leaders at x_0; then: gradient + step (small pulls), and the communication when due
+        if self.t == 0 and self.n_elections == 0:
+            self._elect(None, record)
+        batch = self.batches[self.t % len(self.batches)] if self.batches else None
+        self.lsgd.grad(batch)
+        self.lsgd.step()
+        self.t += 1
+        if self.t % self.w.tau == 0 or self.t % self.alg1["tau_g"] == 0:
+            self._elect(forced_loss, record)
+
     def step(self, forced_loss: Optional[torch.Tensor] = None, record: bool = False) -> None:
+        if self.alg1 is not None:
+            return self._step_algorithm1(forced_loss, record)
         w = self.w
         batch = self.batches[self.t % len(self.batches)] if self.batches else None
         self.lsgd.grad(batch)
