@@ -258,7 +258,8 @@ def run_ours(args):
                                  tau=spec["tau"], steps=steps, config_id=4, x_out=hx.numpy(), g_out=hg.numpy())
         x = hx.to(dev, non_blocking=True)
         g = hg.to(dev, non_blocking=True)
-        pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith)
+        alg1 = dict(gamma_l=0.1, gamma_g=0.05, tau_g=4 * spec["tau"]) if args.schedule == "algorithm1" else None
+        pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith, algorithm1=alg1)
     else:
         w = inputs.config(spec["cfg"], tau=spec["tau"])
         pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith,
@@ -271,6 +272,7 @@ def run_ours(args):
             import torch.distributed as dist
             dist.barrier()
 
+    alg1_mode = getattr(pop, "alg1", None) is not None
     # ---- device-resident timing
     for _ in range(warmup):
         pop.step()
@@ -290,6 +292,19 @@ def run_ours(args):
         t = pop.t
         batch = pop.batches[t % len(pop.batches)] if pop.batches else None
         pop.lsgd.grad(batch)
+        if alg1_mode:
+            # Algorithm 1: step with small pulls towards the leader copies, then the communication when due
+            k_ev[s][0].record()
+            pop.lsgd.step()
+            k_ev[s][1].record()
+            pop.t += 1
+            n_launch += 1
+            pull_flags.append(True)
+            loc, glo = pop.t % spec["tau"] == 0, pop.t % pop.alg1["tau_g"] == 0
+            if loc or glo:
+                pop._elect(None, False)
+                n_launch += 1 + 2 * (int(loc) + int(glo))
+            continue
         if t % spec["tau"] == 0:
             pop.lsgd.elect(pop.loss_ring[pop.n_elections % pop.loss_ring.shape[0]] if pop.loss_ring is not None else None)
             pop.n_elections += 1
@@ -309,10 +324,12 @@ def run_ours(args):
     k_ms = [a.elapsed_time(b) for a, b in k_ev]
     upd_ms = float(np.mean(k_ms))
     alg_bytes = bytes_per_worker_param(spec) * P * d
+    if alg1_mode:
+        alg_bytes += 4.0 * (G + 1) * d          # the G + 1 leader copies are read once per step
     peak, peak_src = read_peaks()
     achieved = alg_bytes / (upd_ms * 1e-3) / 1e9
     traffic = None
-    if spec["kind"] == "external" and args.arith == 0:
+    if spec["kind"] == "external" and args.arith == 0 and not alg1_mode:
         n_pull = sum(pull_flags)
         traffic = P * d * (n_pull * MEASURED_TRAFFIC_PER_WORKER_PARAM["pull"] +
                            (steps - n_pull) * MEASURED_TRAFFIC_PER_WORKER_PARAM["plain"]) / steps
@@ -327,7 +344,7 @@ def run_ours(args):
                    "arithmetic": ["fp64 unfused", "fp64 fma", "fp32 fma"][args.arith],
                    "l2": ("per-step inputs exceed the 126 MB L2; no flush between steps" if P * d * 8 > 3e8 else
                           "working set fits in L2; steps run back to back as in training (no flush)"),
-                   "multi_gpu": "replicas only",
+                   "multi_gpu": "replicas only", "schedule": args.schedule,
                    **({"mlp_fused_step": not args.mlp_unfused_step} if spec["kind"] == "mlp" else {})},
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
@@ -340,7 +357,7 @@ def run_ours(args):
     }
 
     # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs, D2H of its result
-    if rank == 0 and world == 1 and not args.no_e2e and hx is not None:
+    if rank == 0 and world == 1 and not args.no_e2e and hx is not None and not alg1_mode:
         e_steps = args.e2e_steps
         hout = hx                                   # result is read back into the pinned x buffer
         torch.cuda.synchronize(dev)
@@ -394,6 +411,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--sample-cols", type=int, default=0)
     ap.add_argument("--d", type=int, default=0, help="shrink the c4 workload (profiler captures on a small case)")
+    ap.add_argument("--schedule", default="fused", choices=["fused", "algorithm1"],
+                    help="c4 only: algorithm1 = the paper's Algorithm 1 schedule (gamma 0.1 / 0.05, tau_G = 4 tau)")
     ap.add_argument("--mlp-unfused-step", action="store_true", help="c3: do not set LSGD_FLAG_MLP_FUSED_STEP")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
