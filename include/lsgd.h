@@ -202,6 +202,11 @@ LSGD_API lsgd_status lsgd_get_leader_counts(lsgd_handle h, int32_t* global_count
                                    int32_t* local_counts /* HOST int32[P] */);
 /* Reads and clears the device status word; LSGD_ERR_DEVICE_FLAG if any kernel has set it.        */
 LSGD_API lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out /* HOST, may be NULL */);
+/* The "center variable" the paper reports at test time for LSGD (Section 4.1): the average of the
+ * parameters of all workers, center[k] = (1/P) sum_i x[i][k], summed in worker order in fp64 and rounded
+ * once.  center: DEVICE float[ld] (columns d..ld-1 are written as the mean of the padding).  Enqueued
+ * on the stream.                                                                                     */
+LSGD_API lsgd_status lsgd_center(lsgd_handle h, float* center);
 /* Call after overwriting x from outside (restoring a checkpoint, re-seeding a worker): re-derives
  * the library's internal copies of the parameters (the bf16 weight copy of the MLP objective) on the
  * stream.  The step counter and the leaders are kept.                                               */

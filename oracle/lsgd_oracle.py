@@ -293,6 +293,15 @@ class FromCallables(Objective):
         return np.asarray([F32(self.loss_fn(x[i].astype(F64))) for i in range(x.shape[0])], dtype=F32)
 
 
+def center_variable(x: np.ndarray) -> np.ndarray:
+    """The "center variable" reported at test time for LSGD (Section 4.1): the average of the parameters
+    of all workers, accumulated in float64 in worker order and rounded once."""
+    acc = np.zeros(x.shape[1], dtype=F64)
+    for i in range(x.shape[0]):
+        acc = acc + x[i].astype(F64)
+    return (acc * (1.0 / x.shape[0])).astype(F32)
+
+
 # ----------------------------------------------------------------------------------------------
 # The loop
 # ----------------------------------------------------------------------------------------------

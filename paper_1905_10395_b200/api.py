@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
         L.lsgd_get_loss.argtypes = [H, C.c_void_p]
         L.lsgd_get_train_loss.argtypes = [H, C.c_void_p]
         L.lsgd_get_train_loss.restype = C.c_int
+        L.lsgd_center.argtypes = [H, C.c_void_p]
+        L.lsgd_center.restype = C.c_int
         L.lsgd_sync_parameters.argtypes = [H]
         L.lsgd_sync_parameters.restype = C.c_int
         L.lsgd_get_step.argtypes = [H, C.POINTER(C.c_int64)]
@@ -226,6 +228,10 @@ class Lsgd:
         out = np.empty(self.P, dtype=np.float32)
         _check(lib().lsgd_get_train_loss(self.h, out.ctypes.data), "lsgd_get_train_loss")
         return out
+
+    def center(self, out):
+        """out (device float[ld]) <- average of all workers' parameters (the paper's center variable)."""
+        _check(lib().lsgd_center(self.h, _ptr(out)), "lsgd_center")
 
     def sync_parameters(self):
         _check(lib().lsgd_sync_parameters(self.h), "lsgd_sync_parameters")

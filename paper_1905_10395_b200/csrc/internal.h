@@ -56,6 +56,7 @@ struct UpdateArgs {
   bool pull;
 };
 cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s);
+cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, int64_t ld, cudaStream_t s);
 
 struct ElectArgs {
   const float* loss_in;     // DEVICE float[P] or nullptr when partials are given

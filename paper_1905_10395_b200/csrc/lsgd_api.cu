@@ -449,6 +449,13 @@ lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out) {
   return f ? LSGD_ERR_DEVICE_FLAG : LSGD_OK;
 }
 
+lsgd_status lsgd_center(lsgd_handle h, float* center) {
+  if (!h || !center) return LSGD_ERR_INVALID_ARG;
+  if (!aligned16(center)) return LSGD_ERR_ALIGNMENT;
+  LSGD_CUDA(launch_center(h->cfg.x, center, h->cfg.P, h->cfg.d, h->cfg.ld, h->stream));
+  return LSGD_OK;
+}
+
 lsgd_status lsgd_sync_parameters(lsgd_handle h) {
   if (!h) return LSGD_ERR_INVALID_ARG;
   if (h->cfg.objective == LSGD_OBJ_MLP) return mlp_refresh_shadow(h);

@@ -306,6 +306,24 @@ cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
   return cudaGetLastError();
 }
 
+// center[k] = mean over the P workers of x[i][k] (fp64 accumulation in worker order, one rounding)
+__global__ void __launch_bounds__(256)
+center_kernel(const float* __restrict__ x, float* __restrict__ center, int32_t P, int64_t n4, int64_t ld) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const double inv = 1.0 / (double)P;
+  for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < n4; c += stride) {
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    for (int i = 0; i < P; ++i) {
+      const float4 v = ld4(x + (int64_t)i * ld + c * 4);
+      s0 += (double)v.x;
+      s1 += (double)v.y;
+      s2 += (double)v.z;
+      s3 += (double)v.w;
+    }
+    *reinterpret_cast<float4*>(center + c * 4) = make_float4((float)(s0 * inv), (float)(s1 * inv), (float)(s2 * inv), (float)(s3 * inv));
+  }
+}
+
 template <int MODE>
 cudaError_t launch_m(const UpdateArgs& a, cudaStream_t s) {
   const bool quad = (a.g == nullptr);
@@ -317,6 +335,14 @@ cudaError_t launch_m(const UpdateArgs& a, cudaStream_t s) {
 }
 
 }  // namespace
+
+cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, int64_t ld, cudaStream_t s) {
+  const int64_t n4 = (d + 3) / 4;
+  int64_t blocks = (n4 + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  center_kernel<<<(unsigned)blocks, 256, 0, s>>>(x, center, P, n4, ld);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s) {
   switch (a.arith) {

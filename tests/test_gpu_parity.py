@@ -293,3 +293,16 @@ def test_step_protocol_errors():
     pop.lsgd.step()                                                       # t = 1: plain step, no election
     assert pop.lsgd.t() == 2
     pop.close()
+
+
+def test_center_variable_bit_exact():
+    import torch
+    w = inputs.make_external(11, 3, 70001, eta=0.05, lambda_l=0.1, lambda_g=0.05, tau=2, steps=3, config_id=55)
+    pop = _pop(w)
+    pop.run(3)
+    out = torch.empty(w.ld, device="cuda")
+    pop.lsgd.center(out)
+    o = _oracle(w)
+    o.run(3)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), orc.center_variable(o.x).view(np.uint32))
+    pop.close()

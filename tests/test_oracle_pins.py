@@ -427,3 +427,12 @@ def test_mlp_bf16emu_is_close_to_fp32_and_rounding_matches_library():
     g32, g16 = o32.grad(w.x0, 0), o16.grad(w.x0, 0)
     assert np.abs(g32 - g16).max() <= 2e-2 * np.abs(g32).max()
     assert not np.array_equal(g32, g16)
+
+
+# ---- center variable = plain average of the workers (Section 4.1) ---------------------------------
+def test_center_variable_is_the_average():
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal((7, 50)).astype(F32)
+    c = orc.center_variable(x)
+    assert np.allclose(c, x.astype(F64).mean(axis=0), rtol=0, atol=1e-7)
+    assert np.array_equal(orc.center_variable(np.tile(x[:1], (5, 1))), x[0])     # identical workers
