@@ -57,7 +57,8 @@ typedef enum {
   LSGD_OBJ_EXTERNAL = 0,     /* caller writes g and supplies the loss vector                         */
   LSGD_OBJ_QUADRATIC = 1,    /* f(x) = 1/2 sum_k a_k (x_k - b_k)^2                                    */
   LSGD_OBJ_MATCOMP = 2,      /* factorised matrix completion on observed entries                     */
-  LSGD_OBJ_MLP = 3           /* population of ReLU MLP classifiers, bf16 GEMMs, fp32 accumulate      */
+  LSGD_OBJ_MLP = 3,          /* population of ReLU MLP classifiers, bf16 GEMMs, fp32 accumulate      */
+  LSGD_OBJ_PSD_COMPLETION = 4 /* F(X) = 1/4 ||M - X X^T||_F^2, the paper's own completion experiment  */
 } lsgd_objective;
 
 /* How the per-element formulas (update, quadratic gradient) are evaluated.  Storage is always fp32. */
@@ -90,6 +91,15 @@ typedef struct {
   int32_t n_heldout;
   const int32_t* heldout_pos;/* DEVICE int32[n_heldout] positions into the observed list             */
 } lsgd_matcomp_desc;
+
+/* Positive semi-definite low-rank completion, the paper's motivating example (Section 2.1; settings in
+ * the supplement's "Low-Rank Matrix Completion Experiments"): row i of x is X_i (n x r, row-major),
+ * F(X) = 1/4 ||M - X X^T||_F^2, exact gradient (X X^T - M) X (batch LGD, no sampling; lsgd_grad ignores
+ * its batch argument), election loss F(X_i).  d must equal n * r; r <= 128.                         */
+typedef struct {
+  int32_t n, r;
+  const float* M;            /* DEVICE float[n*n], row-major, symmetric; shared by all workers       */
+} lsgd_psd_desc;
 
 /* MLP population: row i of x is [W1 | b1 | W2 | b2 | W3 | b3]; W_l is [n_out][n_in] row-major
  * (input index contiguous); each segment starts at a multiple of 32 floats (see

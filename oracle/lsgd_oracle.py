@@ -193,6 +193,34 @@ class MatComp(Objective):
         return out
 
 
+class PsdCompletion(Objective):
+    """The paper's low-rank matrix completion experiment (Section 2.1 and the supplement):
+    F(X) = 1/4 ||M - X X^T||_F^2 with X in R^{n x r} (the worker's parameter row, row-major),
+    grad F(X) = (X X^T - M) X, exact (batch LGD); election loss F(X_i)."""
+
+    def __init__(self, n: int, r: int, M: np.ndarray):
+        self.n, self.r = int(n), int(r)
+        self.M = np.asarray(M, dtype=F64).reshape(n, n)
+
+    def _residual(self, xi):
+        X = xi[: self.n * self.r].astype(F64).reshape(self.n, self.r)
+        return X, X @ X.T - self.M
+
+    def grad(self, x, t):
+        g = np.zeros_like(x)
+        for i in range(x.shape[0]):
+            X, R = self._residual(x[i])
+            g[i, : self.n * self.r] = (R @ X).ravel().astype(F32)
+        return g
+
+    def loss(self, x, n):
+        out = np.empty(x.shape[0], dtype=F32)
+        for i in range(x.shape[0]):
+            _, R = self._residual(x[i])
+            out[i] = F32(0.25 * np.sum(R * R))
+        return out
+
+
 def bf16_round(a: np.ndarray) -> np.ndarray:
     """Round float32 to the nearest bfloat16 (ties to even), returned as float32 (finite inputs)."""
     u = np.ascontiguousarray(a, dtype=F32).view(np.uint32).astype(np.uint64)

@@ -13,7 +13,7 @@ LIB_PATH = os.path.join(_HERE, "liblsgd.so")
 
 (OK, ERR_INVALID_ARG, ERR_BAD_GROUPS, ERR_ALIGNMENT, ERR_STATE, ERR_CUDA, ERR_UNSUPPORTED, ERR_DEVICE_FLAG,
  ERR_TOO_LARGE) = range(9)
-OBJ_EXTERNAL, OBJ_QUADRATIC, OBJ_MATCOMP, OBJ_MLP = range(4)
+OBJ_EXTERNAL, OBJ_QUADRATIC, OBJ_MATCOMP, OBJ_MLP, OBJ_PSD_COMPLETION = range(5)
 ARITH_FP64, ARITH_FP64_FMA, ARITH_FP32 = range(3)
 FLAG_MLP_FUSED_STEP = 1
 FLAG_ALGORITHM1 = 2
@@ -33,6 +33,10 @@ class MatcompDesc(C.Structure):
     _fields_ = [("n_rows", C.c_int32), ("n_cols", C.c_int32), ("rank", C.c_int32), ("n_obs", C.c_int32),
                 ("obs_r", C.c_void_p), ("obs_c", C.c_void_p), ("obs_v", C.c_void_p), ("batch", C.c_int32),
                 ("n_heldout", C.c_int32), ("heldout_pos", C.c_void_p)]
+
+
+class PsdDesc(C.Structure):
+    _fields_ = [("n", C.c_int32), ("r", C.c_int32), ("M", C.c_void_p)]
 
 
 class MlpDesc(C.Structure):

@@ -102,6 +102,11 @@ int32_t matcomp_loss_blocks(int32_t n_heldout);
 cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials, int32_t n_partials,
                                          cudaStream_t s);
 
+// Dense PSD completion objective.
+int32_t psd_loss_blocks(int32_t n);
+cudaError_t launch_psd_grad(const float* x, float* g, const float* M, int32_t n, int32_t r, int32_t P, int64_t ld,
+                            double* partials, int32_t n_partials, bool write_g, cudaStream_t s);
+
 }  // namespace lsgd
 
 struct lsgd_ctx {
@@ -109,6 +114,8 @@ struct lsgd_ctx {
   lsgd_quadratic_desc quad;
   lsgd_matcomp_desc mc;
   lsgd_mlp_desc mlp;
+  lsgd_psd_desc psd;
+  bool loss_partials_valid;  // PSD: the partial sums of F in d_partials belong to the current x
   cudaStream_t stream;
   int device;
   std::vector<int32_t> group_of;

@@ -68,6 +68,13 @@ lsgd_status validate(const lsgd_config* c) {
       if (m->rank > 32) return LSGD_ERR_UNSUPPORTED;
       break;
     }
+    case LSGD_OBJ_PSD_COMPLETION: {
+      const auto* m = static_cast<const lsgd_psd_desc*>(c->objective_desc);
+      if (!m || !c->g || !m->M || m->n < 1 || m->r < 1) return LSGD_ERR_INVALID_ARG;
+      if ((int64_t)m->n * m->r != c->d) return LSGD_ERR_INVALID_ARG;
+      if (m->r > 128) return LSGD_ERR_UNSUPPORTED;
+      break;
+    }
     case LSGD_OBJ_MLP: {
       const auto* m = static_cast<const lsgd_mlp_desc*>(c->objective_desc);
       if (!m || !c->g) return LSGD_ERR_INVALID_ARG;
@@ -111,6 +118,8 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   std::memset(&h->quad, 0, sizeof(h->quad));
   std::memset(&h->mc, 0, sizeof(h->mc));
   std::memset(&h->mlp, 0, sizeof(h->mlp));
+  std::memset(&h->psd, 0, sizeof(h->psd));
+  h->loss_partials_valid = false;
   h->n_partials = 0;
   if (cfg->objective == LSGD_OBJ_QUADRATIC) {
     h->quad = *static_cast<const lsgd_quadratic_desc*>(cfg->objective_desc);
@@ -120,6 +129,9 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
     h->n_partials = matcomp_loss_blocks(h->mc.n_heldout);
   } else if (cfg->objective == LSGD_OBJ_MLP) {
     h->mlp = *static_cast<const lsgd_mlp_desc*>(cfg->objective_desc);
+  } else if (cfg->objective == LSGD_OBJ_PSD_COMPLETION) {
+    h->psd = *static_cast<const lsgd_psd_desc*>(cfg->objective_desc);
+    h->n_partials = psd_loss_blocks(h->psd.n);
   }
   h->cfg.objective_desc = nullptr;
 
@@ -171,6 +183,9 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   // the host vectors die at return: drain the copies now (creation is not on the hot path)
   ok = ok && cudaStreamSynchronize(h->stream) == cudaSuccess;
   if (ok && cfg->objective == LSGD_OBJ_MLP) ok = (mlp_create(h) == LSGD_OK);
+  // the gradient kernel of this objective writes columns < d only: clear the padding of g once
+  if (ok && cfg->objective == LSGD_OBJ_PSD_COMPLETION && cfg->ld > cfg->d)
+    ok = cudaMemsetAsync(cfg->g, 0, sizeof(float) * (size_t)P * (size_t)cfg->ld, h->stream) == cudaSuccess;
   if (!ok) {
     cudaFree(h->slab);
     delete h;
@@ -202,6 +217,11 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
       LSGD_CUDA(launch_matcomp_grad(a, static_cast<const int32_t*>(batch), h->stream));
       break;
     }
+    case LSGD_OBJ_PSD_COMPLETION:
+      LSGD_CUDA(launch_psd_grad(c.x, c.g, h->psd.M, h->psd.n, h->psd.r, c.P, c.ld, h->d_partials, h->n_partials, true,
+                                h->stream));
+      h->loss_partials_valid = true;
+      break;
     case LSGD_OBJ_MLP: {
       if (!batch) return LSGD_ERR_INVALID_ARG;
       if (h->fused_applied) return LSGD_ERR_STATE;   // the pending gradient has already moved W1, W2
@@ -262,6 +282,15 @@ lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
         e.partial_scale = 1.0 / (double)h->mc.n_heldout;
         break;
       }
+      case LSGD_OBJ_PSD_COMPLETION:
+        if (!h->loss_partials_valid)   // otherwise lsgd_grad has just summed F at this x
+          LSGD_CUDA(launch_psd_grad(c.x, c.g, h->psd.M, h->psd.n, h->psd.r, c.P, c.ld, h->d_partials, h->n_partials,
+                                    false, h->stream));
+        h->loss_partials_valid = true;
+        e.partials = h->d_partials;
+        e.n_partials = h->n_partials;
+        e.partial_scale = 0.25;
+        break;
       case LSGD_OBJ_MLP: {
         if (h->fused_applied) return LSGD_ERR_STATE;   // x is between two steps: no loss at x_t any more
         lsgd_status st = mlp_heldout_loss(h, h->d_loss);
@@ -328,6 +357,7 @@ void set_pull_coefficients(UpdateArgs& a, double cl, double cg) {
 // own pull is zero, so reading the leader rows of x while x is rewritten is exact.
 lsgd_status algorithm1_pulls(lsgd_ctx* h, bool local, bool glob) {
   const lsgd_config& c = h->cfg;
+  h->loss_partials_valid = false;   // x moves
   if (local) {
     UpdateArgs a = base_update_args(h);
     a.pull = true;
@@ -380,6 +410,7 @@ extern "C" lsgd_status lsgd_step(lsgd_handle h) {
     LSGD_CUDA(launch_update(a, h->stream));
   }
   h->t++;
+  h->loss_partials_valid = false;
   h->fused_applied = false;
   h->grad_ready = false;
   h->armed_noise = nullptr;
@@ -458,6 +489,7 @@ lsgd_status lsgd_center(lsgd_handle h, float* center) {
 
 lsgd_status lsgd_sync_parameters(lsgd_handle h) {
   if (!h) return LSGD_ERR_INVALID_ARG;
+  h->loss_partials_valid = false;
   if (h->cfg.objective == LSGD_OBJ_MLP) return mlp_refresh_shadow(h);
   return LSGD_OK;
 }

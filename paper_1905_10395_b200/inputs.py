@@ -196,6 +196,25 @@ def make_matcomp(P: int, G: int, *, n_rows: int = 10000, n_cols: int = 10000, ra
 
 
 # --------------------------------------------------------------------------------------
+# Dense positive semi-definite completion (the paper's own experiment)
+# --------------------------------------------------------------------------------------
+def make_psd(P: int = 8, n: int = 1000, r: int = 10, *, eta: float = 5e-4, lambda_l: float = 0.2,
+             lambda_g: float = 0.0, tau: int = 1, steps: int = 10, G: int = 1, config_id: int = 5,
+             name: str = "psd") -> Workload:
+    """M = U U^T with U in R^{n x r}, i.i.d. N(0,1) entries; every worker starts from its own X ~ N(0,1);
+    defaults are the settings the paper lists for this experiment (eta 5e-4, lambda 1/5, 8 workers,
+    tau 1, n 1000)."""
+    U = rng(config_id, 0).standard_normal((n, r))
+    M = (U @ U.T).astype(np.float32)
+    d = n * r
+    ld = round_up(d, 32)
+    x0 = _padded(P, d, ld, config_id, 1000)
+    return Workload(name=name, objective="psd", P=P, G=G, d=d, ld=ld, group_of=contiguous_groups(P, G), eta=eta,
+                    lambda_l=lambda_l, lambda_g=lambda_g, tau=tau, steps=steps, x0=x0, arrays={"M": M},
+                    meta={"n": n, "r": r})
+
+
+# --------------------------------------------------------------------------------------
 # MLP population on a synthetic Gaussian mixture
 # --------------------------------------------------------------------------------------
 def mlp_layout(dims=MLP_DIMS):

@@ -57,6 +57,12 @@ class Population:
             self.batches = [torch.from_numpy(np.ascontiguousarray(p)).to(dev) for p in A["batch_pos"]]
             if self.g is None:
                 self.g = torch.empty_like(self.x)
+        elif w.objective == "psd":
+            obj = api.OBJ_PSD_COMPLETION
+            self.M = torch.from_numpy(A["M"]).to(dev)
+            desc = api.PsdDesc(w.meta["n"], w.meta["r"], self.M.data_ptr())
+            if self.g is None:
+                self.g = torch.empty_like(self.x)
         elif w.objective == "mlp":
             obj = api.OBJ_MLP
             m = w.meta

@@ -37,6 +37,8 @@ def _oracle(w, **over):
         m = w.meta
         obj = orc.MatComp(m["n_rows"], m["n_cols"], m["rank"], A["obs_r"], A["obs_c"], A["obs_v"],
                           A["batch_pos"], A["heldout_pos"])
+    elif w.objective == "psd":
+        obj = orc.PsdCompletion(w.meta["n"], w.meta["r"], A["M"])
     else:
         raise ValueError
     return orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
@@ -305,4 +307,21 @@ def test_center_variable_bit_exact():
     o = _oracle(w)
     o.run(3)
     assert np.array_equal(out.cpu().numpy().view(np.uint32), orc.center_variable(o.x).view(np.uint32))
+    pop.close()
+
+
+# -------------------------------------------------- dense PSD completion (the paper's own experiment) ----
+@pytest.mark.parametrize("n,r", [(100, 1), (203, 10), (1000, 50), (257, 128)])
+def test_psd_completion_lgd(n, r):
+    """LGD at the paper's settings (eta 5e-4, lambda 1/5, 8 workers, tau 1), ragged n and all rank regimes."""
+    w = inputs.make_psd(P=8, n=n, r=r, steps=10, config_id=56)
+    pop = _pop(w)
+    pop.run(10, record=True)
+    o = _oracle(w)
+    o.run(10)
+    _leaders_equal(pop, o)
+    for hg, ho in zip(pop.history, o.history):
+        assert np.allclose(hg["loss"], ho["loss"], rtol=1e-6, atol=0)
+    assert rel_err(pop.x_host(), o.x) <= TOL
+    assert pop.lsgd.check_device() == 0
     pop.close()

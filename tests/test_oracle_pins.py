@@ -436,3 +436,23 @@ def test_center_variable_is_the_average():
     c = orc.center_variable(x)
     assert np.allclose(c, x.astype(F64).mean(axis=0), rtol=0, atol=1e-7)
     assert np.array_equal(orc.center_variable(np.tile(x[:1], (5, 1))), x[0])     # identical workers
+
+
+# ---- the paper's completion experiment: F = 1/4 ||M - X X^T||^2, grad = (X X^T - M) X ---------------
+def test_psd_completion_gradient_and_monotone_descent():
+    w = inputs.make_psd(P=3, n=7, r=2, steps=3, config_id=45)
+    obj = orc.PsdCompletion(7, 2, w.arrays["M"])
+    g = obj.grad(w.x0, 0)
+    loss = obj.loss(w.x0, 0)
+    M = w.arrays["M"].astype(F64)
+    for i in range(w.P):
+        f = lambda v: 0.25 * np.sum((M - v.reshape(7, 2) @ v.reshape(7, 2).T) ** 2)
+        x = w.x0[i, :14].astype(F64)
+        assert np.allclose(g[i, :14], _fd(f, x, h=1e-5), rtol=1e-6, atol=1e-6)
+        assert math.isclose(loss[i], f(x), rel_tol=1e-6)
+    # "a value was found for which both methods exhibited monotonic decrease": LGD at the paper's settings
+    w = inputs.make_psd(P=8, n=120, r=10, steps=60, config_id=46)
+    o = orc.LsgdOracle(w.x0, orc.PsdCompletion(120, 10, w.arrays["M"]), w.group_of, 1, w.eta, w.lambda_l, 0.0, 1)
+    o.run(60)
+    best = [float(h["loss"].min()) for h in o.history]
+    assert all(b1 <= b0 for b0, b1 in zip(best, best[1:])) and best[-1] < 0.5 * best[0]
