@@ -147,6 +147,11 @@ def workload_spec(args):
         return dict(kind="mlp", cfg=3, P=32, G=4, d=1863712, eta=0.05, lambda_l=0.1, lambda_g=0.05, tau=args.tau or 4,
                     name="C3 MLP population: P=32 G=4, 784-1024-1024-10, batch 128, bf16 GEMM fp32 accumulate",
                     launches=(15, 10))
+    if wl == "psd":
+        r = args.rank
+        return dict(kind="psd", cfg=5, P=8, G=1, d=1000 * r, n=1000, r=r, eta=5e-4, lambda_l=0.2, lambda_g=0.0,
+                    tau=args.tau or 1, name=f"PSD completion (the paper's experiment): 8 workers, n=1000, rank {r}, "
+                    "eta 5e-4, lambda 1/5, tau 1", launches=(3, 2))
     raise SystemExit("unknown workload")
 
 
@@ -191,6 +196,10 @@ def oracle_sample_run(spec, steps, warmup, sample_cols):
         obj = orc.MatComp(m["n_rows"], m["n_cols"], m["rank"], A["obs_r"], A["obs_c"], A["obs_v"], A["batch_pos"],
                           A["heldout_pos"])
         what = "the full workload"
+    elif spec["kind"] == "psd":
+        w = inputs.make_psd(P=P, n=spec["n"], r=spec["r"], steps=steps + warmup)
+        obj = orc.PsdCompletion(spec["n"], spec["r"], w.arrays["M"])
+        what = "the full workload"
     else:
         P = 4
         w = inputs.config(3, P=P, G=1, steps=steps + warmup, tau=spec["tau"], pool=8192)
@@ -222,7 +231,7 @@ def run_reference(args):
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": spec["name"], "tau": spec["tau"],
                    "sample": f"each step covers {what}"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _threads_used() if spec["kind"] == "mlp" else 1,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _threads_used() if spec["kind"] in ("mlp", "psd") else 1,
                          "kind": "oracle",
                          "sample": f"{steps} steps x {what}"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -260,6 +269,9 @@ def run_ours(args):
         g = hg.to(dev, non_blocking=True)
         alg1 = dict(gamma_l=0.1, gamma_g=0.05, tau_g=4 * spec["tau"]) if args.schedule == "algorithm1" else None
         pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith, algorithm1=alg1)
+    elif spec["kind"] == "psd":
+        w = inputs.make_psd(P=P, n=spec["n"], r=spec["r"], steps=steps)
+        pop = Population(w, device=str(dev), arithmetic=args.arith)
     else:
         w = inputs.config(spec["cfg"], tau=spec["tau"])
         pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith,
@@ -282,6 +294,7 @@ def run_ours(args):
     time.sleep(0.3)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     k_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    g_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     barrier()
     torch.cuda.synchronize(dev)
     wall0 = time.time()
@@ -291,7 +304,11 @@ def run_ours(args):
     for s in range(steps):
         t = pop.t
         batch = pop.batches[t % len(pop.batches)] if pop.batches else None
+        if spec["kind"] == "psd":
+            g_ev[s][0].record()
         pop.lsgd.grad(batch)
+        if spec["kind"] == "psd":
+            g_ev[s][1].record()
         if alg1_mode:
             # Algorithm 1: step with small pulls towards the leader copies, then the communication when due
             k_ev[s][0].record()
@@ -336,6 +353,21 @@ def run_ours(args):
     if pop.lsgd.check_device() != 0:
         raise SystemExit("device status word set during the bench")
 
+    roofline = {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
+                "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": traffic, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
+                "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags)),
+                "ms_pull": float(np.mean([m for m, f in zip(k_ms, pull_flags) if f])) if any(pull_flags) else None,
+                "ms_plain": float(np.mean([m for m, f in zip(k_ms, pull_flags) if not f])) if not all(pull_flags) else None}
+    if spec["kind"] == "psd":
+        # the gradient kernel dominates and is bound by fp64 arithmetic: 148 SMs x 64 FMA/clk x 2 x 1.965 GHz
+        g_ms = float(np.mean([a.elapsed_time(b) for a, b in g_ev]))
+        flops = 4.0 * P * spec["n"] ** 2 * spec["r"]           # two passes of n^2 r fused multiply-adds per worker
+        fp64_peak = 148 * 64 * 2 * 1.965e9 / 1e12
+        roofline = {"bound": "alu", "kernel": "psd_grad_kernel", "achieved": flops / (g_ms * 1e-3) / 1e12,
+                    "peak": fp64_peak, "peak_source": "148 SMs x 64 fp64 FMA/clk x 1.965 GHz", "unit": "TFLOP/s",
+                    "frac": flops / (g_ms * 1e-3) / 1e12 / fp64_peak, "traffic": None, "ms_per_launch": g_ms,
+                    "flops_per_launch": flops}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": elapsed_ms / steps, "steps_per_s": steps * world / (elapsed_ms * 1e-3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -347,12 +379,7 @@ def run_ours(args):
                    "multi_gpu": "replicas only", "schedule": args.schedule,
                    **({"mlp_fused_step": not args.mlp_unfused_step} if spec["kind"] == "mlp" else {})},
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
-                     "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
-                     "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags)),
-                     "ms_pull": float(np.mean([m for m, f in zip(k_ms, pull_flags) if f])) if any(pull_flags) else None,
-                     "ms_plain": float(np.mean([m for m, f in zip(k_ms, pull_flags) if not f])) if not all(pull_flags) else None},
+        "roofline": roofline,
         "gpu_launches": n_launch,
     }
 
@@ -387,9 +414,9 @@ def run_ours(args):
     # ---- CPU oracle beside it (rank 0, N = 1 only)
     if rank == 0 and world == 1 and not args.no_cpu:
         sample = args.sample_cols or (1 << 22)
-        osteps = {"external": 3, "quadratic": 3, "matcomp": 8, "mlp": 4}[spec["kind"]]
+        osteps = {"external": 3, "quadratic": 3, "matcomp": 8, "mlp": 4, "psd": 4}[spec["kind"]]
         v, dt, what = oracle_sample_run(spec, osteps, 1, sample)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": _threads_used() if spec["kind"] == "mlp" else 1,
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": _threads_used() if spec["kind"] in ("mlp", "psd") else 1,
                                 "kind": "oracle",
                                 "sample": f"{osteps} steps x {what}, {dt:.1f} s"}
     if rank == 0:
@@ -405,7 +432,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4"])
+    ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4", "psd"])
+    ap.add_argument("--rank", type=int, default=10, help="psd workload: rank r")
     ap.add_argument("--tau", type=int, default=0)
     ap.add_argument("--arith", type=int, default=0, choices=[0, 1, 2])
     ap.add_argument("--e2e-steps", type=int, default=3)
