@@ -81,19 +81,29 @@ __global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16*
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) dst[i] = __float2bfloat16_rn(src[i]);
 }
 
-// xb[row][:] = bf16(pool[idx[row]][:])
-__global__ void gather_rows_kernel(const float* __restrict__ pool, const int32_t* __restrict__ idx, __nv_bfloat16* __restrict__ xb,
-                                   int32_t rows_total, int32_t d0, int32_t pool_rows, uint32_t* status) {
+// xb[row][:] = bf16(pool[idx[row]][:]); 16-byte loads, 8-byte stores (d0 is a multiple of 8)
+__global__ void __launch_bounds__(128)
+gather_rows_kernel(const float* __restrict__ pool, const int32_t* __restrict__ idx, __nv_bfloat16* __restrict__ xb,
+                   int32_t rows_total, int32_t d0, int32_t pool_rows, uint32_t* status) {
   const int row = blockIdx.x;
   if (row >= rows_total) return;
-  const int src = idx[row];
-  if (src < 0 || src >= pool_rows) {
+  int src = idx[row];
+  const bool bad = src < 0 || src >= pool_rows;
+  if (bad) {
     if (threadIdx.x == 0) atomicOr(status, FLAG_BAD_INDEX);
-    for (int k = threadIdx.x; k < d0; k += blockDim.x) xb[(int64_t)row * d0 + k] = __float2bfloat16_rn(0.f);
-    return;
+    src = 0;
   }
-  const float* s = pool + (int64_t)src * d0;
-  for (int k = threadIdx.x; k < d0; k += blockDim.x) xb[(int64_t)row * d0 + k] = __float2bfloat16_rn(s[k]);
+  const float4* s4 = reinterpret_cast<const float4*>(pool + (int64_t)src * d0);
+  uint2* o2 = reinterpret_cast<uint2*>(xb + (int64_t)row * d0);
+  for (int k = threadIdx.x; k < (d0 >> 2); k += blockDim.x) {
+    float4 v = __ldg(s4 + k);
+    if (bad) v = make_float4(0.f, 0.f, 0.f, 0.f);
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t*>(&lo);
+    u.y = *reinterpret_cast<uint32_t*>(&hi);
+    o2[k] = u;
+  }
 }
 
 __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
@@ -205,66 +215,84 @@ head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* _
   }
 }
 
-constexpr int kBwdCols = 128;    // hidden units per CTA
-constexpr int kBwdSlices = 4;    // batch slices per CTA (blockDim.y), combined in a fixed order
+constexpr int kBwdThreadsX = 64;   // each thread owns two adjacent hidden units (one bf16x2)
+constexpr int kBwdCols = 2 * kBwdThreadsX;
+constexpr int kBwdSlices = 8;      // batch slices per CTA (blockDim.y), combined in a fixed order
+constexpr int kDzPitch = kMaxClasses;
 
-// Last layer backward.  Thread (k, s) walks the samples b = s, s + 4, ... of hidden unit k:
+// Last layer backward.  Thread (k, s) walks the samples b = s, s + 8, ... of hidden units 2k, 2k + 1:
 // dH2[b][k] = [H2 > 0] * sum_c dZ[b][c] W3[c][k] (rounded to bf16 and stored), and its share of
 // dW3[:, k] and db2[k]; the slices are added in slice order.  Block 0 of each worker also writes db3.
-__global__ void __launch_bounds__(kBwdCols * kBwdSlices)
+__global__ void __launch_bounds__(kBwdThreadsX * kBwdSlices)
 head_backward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ dz,
                      __nv_bfloat16* __restrict__ dh2, float* __restrict__ g, int32_t n, int32_t d2, int32_t C, int64_t ld,
                      int64_t w3_off, int64_t b3_off, int64_t b2_off) {
-  extern __shared__ float s_mem[];
-  float* s_dz = s_mem;                       // [n][C]
-  float* s_red = s_mem + (size_t)n * C;      // [kBwdSlices][C + 1][kBwdCols]
+  extern __shared__ __align__(16) float s_mem[];
+  float* s_dz = s_mem;                              // [n][kDzPitch], zero beyond C
+  float* s_red = s_mem + (size_t)n * kDzPitch;      // [kBwdSlices][C + 1][kBwdCols]
   const int i = blockIdx.y;
   const int tx = threadIdx.x, ty = threadIdx.y;
-  const int tid = ty * kBwdCols + tx;
+  const int tid = ty * kBwdThreadsX + tx;
   const float* dzi = dz + (int64_t)i * n * C;
-  for (int t = tid; t < n * C; t += kBwdCols * kBwdSlices) s_dz[t] = dzi[t];
+  for (int t = tid; t < n * kDzPitch; t += kBwdThreadsX * kBwdSlices) {
+    const int b = t / kDzPitch, c = t - b * kDzPitch;
+    s_dz[t] = c < C ? dzi[b * C + c] : 0.f;
+  }
   __syncthreads();
   float* gi = g + (int64_t)i * ld;
   if (blockIdx.x == 0 && tid < C) {
     float s = 0.f;
-    for (int b = 0; b < n; ++b) s += s_dz[b * C + tid];
+    for (int b = 0; b < n; ++b) s += s_dz[b * kDzPitch + tid];
     gi[b3_off + tid] = s;
   }
-  const int k = blockIdx.x * kBwdCols + tx;
+  const int k = blockIdx.x * kBwdCols + 2 * tx;     // d2 is even: k and k + 1 are both valid or both not
   const bool live = k < d2;
   const __nv_bfloat16* w3 = wb + (int64_t)i * ld + w3_off;
-  float w[kMaxClasses], aw[kMaxClasses];
+  float w0[kMaxClasses], w1[kMaxClasses], a0[kMaxClasses], a1[kMaxClasses];
 #pragma unroll
   for (int c = 0; c < kMaxClasses; ++c) {
-    w[c] = (live && c < C) ? __bfloat162float(w3[(int64_t)c * d2 + k]) : 0.f;
-    aw[c] = 0.f;
+    float2 wv = make_float2(0.f, 0.f);
+    if (live && c < C) wv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(w3 + (int64_t)c * d2 + k));
+    w0[c] = wv.x;
+    w1[c] = wv.y;
+    a0[c] = 0.f;
+    a1[c] = 0.f;
   }
-  float ab = 0.f;
+  float ab0 = 0.f, ab1 = 0.f;
   if (live) {
     const __nv_bfloat16* hcol = h2 + (int64_t)i * n * d2 + k;
     __nv_bfloat16* dcol = dh2 + (int64_t)i * n * d2 + k;
     for (int b0 = ty; b0 < n; b0 += 4 * kBwdSlices) {
-      float hv[4];
+      float2 hv[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int b = b0 + u * kBwdSlices;
-        hv[u] = b < n ? __bfloat162float(hcol[(int64_t)b * d2]) : 0.f;
+        hv[u] = b < n ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hcol + (int64_t)b * d2)) : make_float2(0.f, 0.f);
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int b = b0 + u * kBwdSlices;
         if (b < n) {
-          float dh = 0.f;
+          float z[kMaxClasses];
+#pragma unroll
+          for (int q = 0; q < kMaxClasses / 4; ++q) {
+            const float4 t = *reinterpret_cast<const float4*>(s_dz + b * kDzPitch + 4 * q);
+            z[4 * q] = t.x; z[4 * q + 1] = t.y; z[4 * q + 2] = t.z; z[4 * q + 3] = t.w;
+          }
+          float dh0 = 0.f, dh1 = 0.f;
 #pragma unroll
           for (int c = 0; c < kMaxClasses; ++c)
             if (c < C) {
-              const float z = s_dz[b * C + c];
-              aw[c] = fmaf(z, hv[u], aw[c]);
-              dh = fmaf(z, w[c], dh);
+              a0[c] = fmaf(z[c], hv[u].x, a0[c]);
+              a1[c] = fmaf(z[c], hv[u].y, a1[c]);
+              dh0 = fmaf(z[c], w0[c], dh0);
+              dh1 = fmaf(z[c], w1[c], dh1);
             }
-          const __nv_bfloat16 r = __float2bfloat16_rn(hv[u] > 0.f ? dh : 0.f);
-          dcol[(int64_t)b * d2] = r;
-          ab += __bfloat162float(r);
+          const __nv_bfloat162 r = __floats2bfloat162_rn(hv[u].x > 0.f ? dh0 : 0.f, hv[u].y > 0.f ? dh1 : 0.f);
+          *reinterpret_cast<__nv_bfloat162*>(dcol + (int64_t)b * d2) = r;
+          const float2 rf = __bfloat1622float2(r);
+          ab0 += rf.x;
+          ab1 += rf.y;
         }
       }
     }
@@ -272,33 +300,63 @@ head_backward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* 
   float* red = s_red + (size_t)ty * (C + 1) * kBwdCols;
 #pragma unroll
   for (int c = 0; c < kMaxClasses; ++c)
-    if (c < C) red[c * kBwdCols + tx] = aw[c];
-  red[C * kBwdCols + tx] = ab;
+    if (c < C) {
+      red[c * kBwdCols + 2 * tx] = a0[c];
+      red[c * kBwdCols + 2 * tx + 1] = a1[c];
+    }
+  red[C * kBwdCols + 2 * tx] = ab0;
+  red[C * kBwdCols + 2 * tx + 1] = ab1;
   __syncthreads();
-  if (ty == 0 && live) {
-#pragma unroll
-    for (int c = 0; c < kMaxClasses; ++c)
-      if (c < C) {
-        float t = 0.f;
-        for (int sl = 0; sl < kBwdSlices; ++sl) t += s_red[((size_t)sl * (C + 1) + c) * kBwdCols + tx];
-        gi[w3_off + (int64_t)c * d2 + k] = t;
-      }
-    float t = 0.f;
-    for (int sl = 0; sl < kBwdSlices; ++sl) t += s_red[((size_t)sl * (C + 1) + C) * kBwdCols + tx];
-    gi[b2_off + k] = t;
+  // (C + 1) x kBwdCols sums over the slices, in slice order
+  for (int t = tid; t < (C + 1) * kBwdCols; t += kBwdThreadsX * kBwdSlices) {
+    const int c = t / kBwdCols, kk = t - c * kBwdCols;
+    const int kcol = blockIdx.x * kBwdCols + kk;
+    if (kcol >= d2) continue;
+    float acc = 0.f;
+    for (int sl = 0; sl < kBwdSlices; ++sl) acc += s_red[((size_t)sl * (C + 1) + c) * kBwdCols + kk];
+    if (c < C) gi[w3_off + (int64_t)c * d2 + kcol] = acc;
+    else gi[b2_off + kcol] = acc;
   }
 }
 
-// db[k] = sum_b delta[b][k] for a stored (bf16) delta matrix.
-__global__ void __launch_bounds__(128)
+constexpr int kSumThreadsX = 64, kSumSlices = 8;
+
+// db[k] = sum_b delta[b][k] for a stored (bf16) delta matrix; thread (k, s) adds the samples s, s + 8, ...
+// of columns 2k, 2k + 1 and the slices are combined in slice order.
+__global__ void __launch_bounds__(kSumThreadsX * kSumSlices)
 column_sum_kernel(const __nv_bfloat16* __restrict__ delta, float* __restrict__ g, int32_t n, int32_t dcols, int64_t ld, int64_t off) {
-  const int i = blockIdx.y;
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= dcols) return;
-  const __nv_bfloat16* col = delta + (int64_t)i * n * dcols + k;
-  float s = 0.f;
-  for (int b = 0; b < n; ++b) s += __bfloat162float(col[(int64_t)b * dcols]);
-  g[(int64_t)i * ld + off + k] = s;
+  __shared__ float s_part[kSumSlices][2 * kSumThreadsX];
+  const int i = blockIdx.y, tx = threadIdx.x, ty = threadIdx.y;
+  const int k = blockIdx.x * 2 * kSumThreadsX + 2 * tx;
+  float s0 = 0.f, s1 = 0.f;
+  if (k < dcols) {
+    const __nv_bfloat16* col = delta + (int64_t)i * n * dcols + k;
+    for (int b0 = ty; b0 < n; b0 += 4 * kSumSlices) {
+      float2 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int b = b0 + u * kSumSlices;
+        v[u] = b < n ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(col + (int64_t)b * dcols)) : make_float2(0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        s0 += v[u].x;
+        s1 += v[u].y;
+      }
+    }
+  }
+  s_part[ty][2 * tx] = s0;
+  s_part[ty][2 * tx + 1] = s1;
+  __syncthreads();
+  const int t = ty * kSumThreadsX + tx;
+  if (t < 2 * kSumThreadsX) {
+    const int kcol = blockIdx.x * 2 * kSumThreadsX + t;
+    if (kcol < dcols) {
+      float acc = 0.f;
+      for (int sl = 0; sl < kSumSlices; ++sl) acc += s_part[sl][t];
+      g[(int64_t)i * ld + off + kcol] = acc;
+    }
+  }
 }
 
 // out[i] = mean_b v[i][b], summed in a fixed order by one warp per worker.
@@ -350,7 +408,7 @@ lsgd_status mlp_validate(const lsgd_config& c, const lsgd_mlp_desc& m) {
   if (m.batch % 8 || m.n_heldout % 8 || m.batch > 1024) return LSGD_ERR_UNSUPPORTED;
   // shared-memory budgets of the last-layer kernels (48 KB without opting in)
   if ((size_t)m.dims[3] * m.dims[2] * 2 > 48 * 1024) return LSGD_ERR_UNSUPPORTED;
-  if (sizeof(float) * ((size_t)m.batch * m.dims[3] + (size_t)kBwdSlices * (m.dims[3] + 1) * kBwdCols) > 48 * 1024)
+  if (sizeof(float) * ((size_t)m.batch * kDzPitch + (size_t)kBwdSlices * (m.dims[3] + 1) * kBwdCols) > 160 * 1024)
     return LSGD_ERR_UNSUPPORTED;
   const Layout L = param_layout(m.dims);
   if (L.d != c.d || c.ld != c.d) return LSGD_ERR_INVALID_ARG;
@@ -425,8 +483,14 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   head_forward_kernel<1><<<dim3((B + kHeadWarps - 1) / kHeadWarps, P), kHeadWarps * 32, w3_smem, s>>>(
       st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], m.pool, 1,
       h->d_status);
-  const size_t bwd_smem = sizeof(float) * ((size_t)B * d[3] + (size_t)kBwdSlices * (d[3] + 1) * kBwdCols);
-  head_backward_kernel<<<dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdCols, kBwdSlices), bwd_smem, s>>>(
+  const size_t bwd_smem = sizeof(float) * ((size_t)B * kDzPitch + (size_t)kBwdSlices * (d[3] + 1) * kBwdCols);
+  static bool bwd_attr = false;
+  if (!bwd_attr) {
+    if (cudaFuncSetAttribute(head_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
+      return LSGD_ERR_CUDA;
+    bwd_attr = true;
+  }
+  head_backward_kernel<<<dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdThreadsX, kBwdSlices), bwd_smem, s>>>(
       st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]);
   if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
 
@@ -443,7 +507,8 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   g2.eta = (double)c.eta;
   g2.arith = c.arithmetic;
   if (launch_bgemm(st->m_dh2, st->m_h1, g2, s) != cudaSuccess) return LSGD_ERR_CUDA;
-  column_sum_kernel<<<dim3((d[1] + 127) / 128, P), 128, 0, s>>>(st->dh1, c.g, B, d[1], ld, st->L.b[0]);
+  column_sum_kernel<<<dim3((d[1] + 2 * kSumThreadsX - 1) / (2 * kSumThreadsX), P), dim3(kSumThreadsX, kSumSlices), 0, s>>>(
+      st->dh1, c.g, B, d[1], ld, st->L.b[0]);
   if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
   // dW1 = dH1^T . X                           [d1 x d0]
   GemmShape g1 = shape(d[1], d[0], B, P, 1, 1, 1, fuse_sgd ? GEMM_EPI_SGD : GEMM_EPI_F32, c.g + st->L.w[0], d[0], ld, h->d_status);
