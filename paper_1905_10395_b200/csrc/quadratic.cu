@@ -2,8 +2,9 @@
 // Section 3.3 with a diagonal Hessian): materialised stochastic gradient g = a (x - b) + sigma eps
 // and the first stage of the exact election loss f(x_i).
 //
-// Loss: CTA (blk, i) sums worker i's terms over a fixed chunk of columns, every term evaluated and
-// accumulated in fp64, and writes one partial; the election kernel adds the partials in index order.
+// Loss: CTA (blk, row group) sums the terms of up to 8 workers over a fixed chunk of columns, every term
+// evaluated and accumulated in fp64, and writes one partial per worker; the election kernel adds the
+// partials in index order.
 // Chunking and tree shape depend only on d, so the result is reproducible run to run.
 #include "internal.h"
 
@@ -50,40 +51,59 @@ quadratic_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const 
   }
 }
 
-__device__ __forceinline__ double term(float x, float a, float b) {
-  const double r = (double)x - (double)b;
-  return (double)a * r * r;
+constexpr int kLossRows = 8;   // workers per CTA: a and b are loaded and converted once for all of them
+
+__device__ __forceinline__ double term(double x, double a, double b) {
+  const double r = x - b;
+  return a * r * r;
 }
 
+// CTA (chunk, row group): partial sums of f over 8192 columns for up to 8 workers.
 __global__ void __launch_bounds__(kThreads)
-quadratic_loss_kernel(const float* __restrict__ x, const float* __restrict__ a, const float* __restrict__ b,
+quadratic_loss_kernel(const float* __restrict__ x, const float* __restrict__ a, const float* __restrict__ b, int32_t P,
                       int64_t d, int64_t ld, double* __restrict__ partials, int32_t n_partials) {
-  const int i = blockIdx.y;
+  const int i0 = blockIdx.y * kLossRows;
+  const int rows = min(kLossRows, P - i0);
   const int64_t c0 = (int64_t)blockIdx.x * kChunkCols;
-  const float* xr = x + (int64_t)i * ld;
-  double acc = 0.0;
+  double acc[kLossRows];
 #pragma unroll
+  for (int r = 0; r < kLossRows; ++r) acc[r] = 0.0;
+#pragma unroll 2
   for (int v = 0; v < kVecPerThread; ++v) {
     const int64_t c = c0 + ((int64_t)v * kThreads + threadIdx.x) * 4;
     if (c + 3 < d) {
-      const float4 xv = __ldcs(reinterpret_cast<const float4*>(xr + c));
-      const float4 av = __ldg(reinterpret_cast<const float4*>(a + c));
-      const float4 bv = __ldg(reinterpret_cast<const float4*>(b + c));
-      acc += term(xv.x, av.x, bv.x) + term(xv.y, av.y, bv.y) + term(xv.z, av.z, bv.z) + term(xv.w, av.w, bv.w);
+      const float4 af = __ldg(reinterpret_cast<const float4*>(a + c));
+      const float4 bf = __ldg(reinterpret_cast<const float4*>(b + c));
+      const double a0 = af.x, a1 = af.y, a2 = af.z, a3 = af.w;
+      const double b0 = bf.x, b1 = bf.y, b2 = bf.z, b3 = bf.w;
+      float4 xv[kLossRows];
+#pragma unroll
+      for (int r = 0; r < kLossRows; ++r)
+        if (r < rows) xv[r] = __ldcs(reinterpret_cast<const float4*>(x + (int64_t)(i0 + r) * ld + c));
+#pragma unroll
+      for (int r = 0; r < kLossRows; ++r)
+        if (r < rows)
+          acc[r] += term((double)xv[r].x, a0, b0) + term((double)xv[r].y, a1, b1) + term((double)xv[r].z, a2, b2) +
+                    term((double)xv[r].w, a3, b3);
     } else {
-      for (int64_t k = c; k < d; ++k) acc += term(xr[k], a[k], b[k]);
+      for (int64_t k = c; k < d; ++k)
+        for (int r = 0; r < rows; ++r) acc[r] += term((double)x[(int64_t)(i0 + r) * ld + k], (double)a[k], (double)b[k]);
     }
   }
+  __shared__ double s_w[kLossRows][kThreads / 32];
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-  __shared__ double s_w[kThreads / 32];
-  if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = acc;
+  for (int r = 0; r < kLossRows; ++r) {
+    double t = acc[r];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+    if ((threadIdx.x & 31) == 0) s_w[r][threadIdx.x >> 5] = t;
+  }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (threadIdx.x < rows) {
     double t = 0.0;
 #pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) t += s_w[w];
-    partials[(int64_t)i * n_partials + blockIdx.x] = t;
+    for (int w = 0; w < kThreads / 32; ++w) t += s_w[threadIdx.x][w];
+    partials[(int64_t)(i0 + threadIdx.x) * n_partials + blockIdx.x] = t;
   }
 }
 
@@ -107,8 +127,8 @@ int32_t quadratic_loss_blocks(int64_t d) { return (int32_t)((d + kChunkCols - 1)
 
 cudaError_t launch_quadratic_loss_partials(const float* x, const float* a, const float* b, int32_t P, int64_t d,
                                            int64_t ld, double* partials, int32_t n_partials, cudaStream_t s) {
-  dim3 grid((unsigned)n_partials, (unsigned)P);
-  quadratic_loss_kernel<<<grid, kThreads, 0, s>>>(x, a, b, d, ld, partials, n_partials);
+  dim3 grid((unsigned)n_partials, (unsigned)((P + kLossRows - 1) / kLossRows));
+  quadratic_loss_kernel<<<grid, kThreads, 0, s>>>(x, a, b, P, d, ld, partials, n_partials);
   return cudaGetLastError();
 }
 
