@@ -25,6 +25,9 @@ namespace {
 //   pull form : 256 threads, 2 rows of loads in flight, registers capped for 4 CTAs per SM, 8 grid-stride
 //               CTAs per SM (more rows in flight cost occupancy and lose; 5+ CTAs per SM spill);
 //   plain form: 256 threads, 4 elements in flight, one CTA per 1024 columns up to 64 CTAs per SM.
+#ifndef LSGD_K1_NO_STAGED
+#define LSGD_K1_NO_STAGED 0     // 1: never use the shared-memory-staged pull kernel
+#endif
 #ifndef LSGD_K1_THREADS
 #define LSGD_K1_THREADS 256
 #endif
@@ -273,6 +276,177 @@ plain_update_kernel(UpdateArgs p, int64_t n4) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Pull form with the column tile staged in shared memory by the bulk-copy engine.
+//
+// A persistent CTA takes column tiles of W floats.  For a tile, one warp issues 2 P one-dimensional bulk
+// copies (cp.async.bulk, row i of x and of g -> shared memory, completion on an mbarrier) into one of
+// kTmaStages stages; eight consumer warps then read everything -- the row itself, its gradient and both
+// leaders -- from that snapshot of x_t, and write the new x straight to global memory with 512-byte
+// coalesced stores.  Leaders are therefore fetched once per tile together with the other rows, the
+// in-place update cannot disturb them, and the loads in flight (stages x 2 P W x 4 bytes per SM) no longer
+// depend on registers.  Waits are clock-bounded; on expiry the status word is flagged and the CTA leaves.
+// Shape found by timing sweeps on the 16 x 2^26 stress shape: what matters most is the length of the
+// contiguous piece fetched per row (3 KiB: 6.8 TB/s; 2 KiB: 6.4; 1 KiB: 5.5; 512 B: 2.9 -- DRAM pages are
+// used best by long bursts), then enough consumer warps to keep up (24), and only two stages: more stages
+// interleave more rows at the memory controllers and lose again.
+#ifndef LSGD_K1_STAGED_STAGES
+#define LSGD_K1_STAGED_STAGES 2
+#endif
+#ifndef LSGD_K1_STAGED_CONSUMERS
+#define LSGD_K1_STAGED_CONSUMERS 768
+#endif
+#ifndef LSGD_K1_STAGED_W
+#define LSGD_K1_STAGED_W 768
+#endif
+constexpr int kTmaStages = LSGD_K1_STAGED_STAGES;
+constexpr int kTmaConsumers = LSGD_K1_STAGED_CONSUMERS;
+constexpr int kTmaThreads = kTmaConsumers + 32;
+constexpr int kTmaSmemBudget = 208 * 1024;
+constexpr long long kTmaWaitCycles = 2000000000LL;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool bar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+  if (bar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (bar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kTmaWaitCycles) {
+      *abort_flag = 1;
+      atomicOr(status, FLAG_WAIT_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+template <int MODE, bool SHADOW>
+__global__ void __launch_bounds__(kTmaThreads, 1)
+pull_update_staged_kernel(UpdateArgs p, int64_t n_cols4, int W) {
+  extern __shared__ __align__(128) uint8_t s_raw[];
+  __shared__ uint64_t full_bar[kTmaStages], empty_bar[kTmaStages];
+  __shared__ int s_abort, s_bad, s_gl;
+  const int P = p.P;
+  const size_t stage_floats = (size_t)2 * P * W;                  // x rows then g rows
+  float* stage0 = reinterpret_cast<float*>(s_raw);
+  int32_t* s_lead = reinterpret_cast<int32_t*>(stage0 + kTmaStages * stage_floats);   // [P]: local leader row of worker i
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    s_bad = 0;
+    for (int s = 0; s < kTmaStages; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&full_bar[s])), "r"(1) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&empty_bar[s])), "r"(kTmaConsumers / 32) : "memory");
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const int gl = *p.gl;
+    if (gl < 0 || gl >= P) s_bad = 1;
+    s_gl = gl;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < P; i += blockDim.x) {
+    const int l = p.ll[p.tab.group_of[i]];
+    if (l < 0 || l >= P) s_bad = 1;
+    s_lead[i] = l;
+  }
+  __syncthreads();
+  if (s_bad) {   // never index shared memory with a leader that is out of range
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(p.status, FLAG_BAD_LEADER);
+    return;
+  }
+  volatile int* abort_flag = &s_abort;
+  const int64_t total_floats = n_cols4 * 4;
+  const int64_t n_tiles = (total_floats + W - 1) / W;
+  if (warp == kTmaConsumers / 32) {
+    // ------------------------------------------------------------------ producer warp
+    uint32_t it = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+      const int s = it % kTmaStages;
+      ok = bar_wait(&empty_bar[s], ((it / kTmaStages) & 1) ^ 1, abort_flag, p.status);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      const int64_t c0 = t * W;
+      const int wt = (int)((total_floats - c0) < W ? (total_floats - c0) : W);   // floats in this tile (multiple of 4)
+      const uint32_t bytes = (uint32_t)wt * 4u;
+      float* sx = stage0 + s * stage_floats;
+      float* sg = sx + (size_t)P * W;
+      if (lane == 0)
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&full_bar[s])), "r"(bytes * 2u * (uint32_t)P) : "memory");
+      __syncwarp();
+      for (int i = lane; i < P; i += 32) {
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_addr(sx + (size_t)i * W)), "l"(p.x + (int64_t)i * p.ld + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_addr(sg + (size_t)i * W)), "l"(p.g + (int64_t)i * p.ld + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
+      }
+    }
+    if (*abort_flag && lane == 0) {
+      // a wait ran out somewhere: let the copies already issued land before the CTA exits
+      const uint32_t first = it > kTmaStages ? it - kTmaStages : 0;
+      for (uint32_t j = first; j < it; ++j) {
+        const long long t0 = clock64();
+        while (!bar_try(&full_bar[j % kTmaStages], (j / kTmaStages) & 1) && clock64() - t0 < kTmaWaitCycles) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers
+    const Coef k = p.k;
+    const int gl = s_gl;
+    const int w4 = W >> 2;                          // 16-byte columns per tile row
+    const int c4 = threadIdx.x % w4;                // this thread's column
+    const int r0 = threadIdx.x / w4, rstep = kTmaConsumers / w4;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+      const int s = it % kTmaStages;
+      ok = bar_wait(&full_bar[s], (it / kTmaStages) & 1, abort_flag, p.status);
+      if (!ok) break;
+      const int64_t c0 = t * W;
+      const int wt4 = (int)(((total_floats - c0) < W ? (total_floats - c0) : W) >> 2);
+      const float* sx = stage0 + s * stage_floats;
+      const float* sg = sx + (size_t)P * W;
+      // thread (column c4, row lane r0) walks rows r0, r0 + rstep, ...; the global leader's value stays in registers
+      if (c4 < wt4) {
+        const float4 xg = *reinterpret_cast<const float4*>(sx + (size_t)gl * W + c4 * 4);
+        for (int i = r0; i < P; i += rstep) {
+          const float4 x = *reinterpret_cast<const float4*>(sx + (size_t)i * W + c4 * 4);
+          const float4 g = *reinterpret_cast<const float4*>(sg + (size_t)i * W + c4 * 4);
+          const float4 xl = *reinterpret_cast<const float4*>(sx + (size_t)s_lead[i] * W + c4 * 4);
+          float4 r;
+          r.x = pull1<MODE>(x.x, g.x, xl.x, xg.x, k);
+          r.y = pull1<MODE>(x.y, g.y, xl.y, xg.y, k);
+          r.z = pull1<MODE>(x.z, g.z, xl.z, xg.z, k);
+          r.w = pull1<MODE>(x.w, g.w, xl.w, xg.w, k);
+          const int64_t off = (int64_t)i * p.ld + c0 + c4 * 4;
+          st4(p.x + off, r);
+          if (SHADOW) st4_bf16(p.x_bf16 + off, r);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&empty_bar[s])) : "memory");
+    }
+  }
+}
+
+// Tile width (floats) for the staged kernel, 0 if the shape does not suit it: all P rows of a tile of at
+// least 512 columns (2 KiB per row) must fit twice over in shared memory, i.e. P <= 26; larger populations
+// use the register-staged kernel above.
+inline int staged_tile_width(const UpdateArgs& a) {
+  if (!a.pull || a.g == nullptr || a.snap != nullptr || !a.use_g) return 0;
+  for (int W = LSGD_K1_STAGED_W; W >= 512; W -= 256) {
+    const size_t bytes = (size_t)kTmaStages * 2 * a.P * W * 4 + (size_t)a.P * 4;
+    if (bytes <= (size_t)kTmaSmemBudget && (kTmaConsumers % (W / 4)) == 0) return W;
+  }
+  return 0;
+}
+
 template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
 cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
   static int sms = 0;
@@ -284,7 +458,20 @@ cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
   }
   const int64_t n4 = (a.d + 3) / 4;
   const int64_t cap = (int64_t)sms * (a.pull ? LSGD_K1_PULL_CTAS_PER_SM : LSGD_K1_PLAIN_CTAS_PER_SM);
-  if (a.pull) {
+  const int W = (QUAD || LSGD_K1_NO_STAGED) ? 0 : staged_tile_width(a);
+  if (W > 0) {
+    static bool attr_done = false;
+    if (!attr_done) {
+      cudaError_t e = cudaFuncSetAttribute(pull_update_staged_kernel<MODE, SHADOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           kTmaSmemBudget + 1024);
+      if (e != cudaSuccess) return e;
+      attr_done = true;
+    }
+    const size_t smem = (size_t)kTmaStages * 2 * a.P * W * 4 + (size_t)a.P * 4;
+    const int64_t tiles = (n4 * 4 + W - 1) / (W > 0 ? W : 1);
+    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    pull_update_staged_kernel<MODE, SHADOW><<<grid, kTmaThreads, smem, s>>>(a, n4, W);
+  } else if (a.pull) {
     int64_t blocks = (n4 + kThreads - 1) / kThreads;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
