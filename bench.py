@@ -157,7 +157,7 @@ def workload_spec(args):
 
 # DRAM bytes per worker-parameter of the update kernels, from the ncu counters of a d = 2^22 capture of
 # the same kernels (profiles/pull_update_kernel_c4.md); traffic is proportional to d.
-MEASURED_TRAFFIC_PER_WORKER_PARAM = {"pull": 11.34, "plain": 11.30}
+MEASURED_TRAFFIC_PER_WORKER_PARAM = {"pull": 11.27, "plain": 11.30}
 
 
 def bytes_per_worker_param(spec):
@@ -353,7 +353,7 @@ def run_ours(args):
     if pop.lsgd.check_device() != 0:
         raise SystemExit("device status word set during the bench")
 
-    roofline = {"bound": "hbm", "kernel": "pull_update_kernel / plain_update_kernel", "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": "pull_update_staged_kernel / plain_update_kernel", "achieved": achieved,
                 "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
                 "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags)),
