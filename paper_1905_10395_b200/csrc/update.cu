@@ -333,7 +333,9 @@ pull_update_staged_kernel(UpdateArgs p, int64_t n_cols4, int W) {
   __shared__ uint64_t full_bar[kTmaStages], empty_bar[kTmaStages];
   __shared__ int s_abort, s_bad, s_gl;
   const int P = p.P;
-  const size_t stage_floats = (size_t)2 * P * W;                  // x rows then g rows
+  const bool use_g = p.use_g, snap = p.snap != nullptr;
+  const int n_rows = P + (use_g ? P : 0) + (snap ? p.G + 1 : 0);  // x rows, g rows, leader copies
+  const size_t stage_floats = (size_t)n_rows * W;
   float* stage0 = reinterpret_cast<float*>(s_raw);
   int32_t* s_lead = reinterpret_cast<int32_t*>(stage0 + kTmaStages * stage_floats);   // [P]: local leader row of worker i
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -346,12 +348,14 @@ pull_update_staged_kernel(UpdateArgs p, int64_t n_cols4, int W) {
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     const int gl = *p.gl;
-    if (gl < 0 || gl >= P) s_bad = 1;
+    if (!snap && (gl < 0 || gl >= P)) s_bad = 1;
     s_gl = gl;
   }
   __syncthreads();
   for (int i = threadIdx.x; i < P; i += blockDim.x) {
-    const int l = p.ll[p.tab.group_of[i]];
+    // row of the stage that holds worker i's local leader: a row of x, or (with leader copies) a copy row
+    const int grp = p.tab.group_of[i];
+    const int l = snap ? grp : p.ll[grp];
     if (l < 0 || l >= P) s_bad = 1;
     s_lead[i] = l;
   }
@@ -376,15 +380,17 @@ pull_update_staged_kernel(UpdateArgs p, int64_t n_cols4, int W) {
       const int wt = (int)((total_floats - c0) < W ? (total_floats - c0) : W);   // floats in this tile (multiple of 4)
       const uint32_t bytes = (uint32_t)wt * 4u;
       float* sx = stage0 + s * stage_floats;
-      float* sg = sx + (size_t)P * W;
       if (lane == 0)
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&full_bar[s])), "r"(bytes * 2u * (uint32_t)P) : "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&full_bar[s])), "r"(bytes * (uint32_t)n_rows) : "memory");
       __syncwarp();
-      for (int i = lane; i < P; i += 32) {
+      for (int r = lane; r < n_rows; r += 32) {
+        // stage row r: worker r's x, then worker (r - P)'s g, then the leader copies
+        const float* src;
+        if (r < P) src = p.x + (int64_t)r * p.ld;
+        else if (use_g && r < 2 * P) src = p.g + (int64_t)(r - P) * p.ld;
+        else src = p.snap + (int64_t)(r - P - (use_g ? P : 0)) * p.ld;
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(smem_addr(sx + (size_t)i * W)), "l"(p.x + (int64_t)i * p.ld + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(smem_addr(sg + (size_t)i * W)), "l"(p.g + (int64_t)i * p.ld + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
+                     ::"r"(smem_addr(sx + (size_t)r * W)), "l"(src + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
       }
     }
     if (*abort_flag && lane == 0) {
@@ -412,13 +418,14 @@ pull_update_staged_kernel(UpdateArgs p, int64_t n_cols4, int W) {
       const int wt4 = (int)(((total_floats - c0) < W ? (total_floats - c0) : W) >> 2);
       const float* sx = stage0 + s * stage_floats;
       const float* sg = sx + (size_t)P * W;
+      const float* sl = snap ? sx + (size_t)(P + (use_g ? P : 0)) * W : sx;     // where the leaders' rows are
       // thread (column c4, row lane r0) walks rows r0, r0 + rstep, ...; the global leader's value stays in registers
       if (c4 < wt4) {
-        const float4 xg = *reinterpret_cast<const float4*>(sx + (size_t)gl * W + c4 * 4);
+        const float4 xg = *reinterpret_cast<const float4*>(sl + (size_t)(snap ? p.G : gl) * W + c4 * 4);
         for (int i = r0; i < P; i += rstep) {
           const float4 x = *reinterpret_cast<const float4*>(sx + (size_t)i * W + c4 * 4);
-          const float4 g = *reinterpret_cast<const float4*>(sg + (size_t)i * W + c4 * 4);
-          const float4 xl = *reinterpret_cast<const float4*>(sx + (size_t)s_lead[i] * W + c4 * 4);
+          const float4 g = use_g ? *reinterpret_cast<const float4*>(sg + (size_t)i * W + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 xl = *reinterpret_cast<const float4*>(sl + (size_t)s_lead[i] * W + c4 * 4);
           float4 r;
           r.x = pull1<MODE>(x.x, g.x, xl.x, xg.x, k);
           r.y = pull1<MODE>(x.y, g.y, xl.y, xg.y, k);
@@ -438,10 +445,11 @@ pull_update_staged_kernel(UpdateArgs p, int64_t n_cols4, int W) {
 // Tile width (floats) for the staged kernel, 0 if the shape does not suit it: all P rows of a tile of at
 // least 512 columns (2 KiB per row) must fit twice over in shared memory, i.e. P <= 26; larger populations
 // use the register-staged kernel above.
+inline int staged_rows(const UpdateArgs& a) { return a.P + (a.use_g ? a.P : 0) + (a.snap ? a.G + 1 : 0); }
 inline int staged_tile_width(const UpdateArgs& a) {
-  if (!a.pull || a.g == nullptr || a.snap != nullptr || !a.use_g) return 0;
+  if (!a.pull || (a.use_g && a.g == nullptr)) return 0;
   for (int W = LSGD_K1_STAGED_W; W >= 512; W -= 256) {
-    const size_t bytes = (size_t)kTmaStages * 2 * a.P * W * 4 + (size_t)a.P * 4;
+    const size_t bytes = (size_t)kTmaStages * staged_rows(a) * W * 4 + (size_t)a.P * 4;
     if (bytes <= (size_t)kTmaSmemBudget && (kTmaConsumers % (W / 4)) == 0) return W;
   }
   return 0;
@@ -467,7 +475,7 @@ cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
       if (e != cudaSuccess) return e;
       attr_done = true;
     }
-    const size_t smem = (size_t)kTmaStages * 2 * a.P * W * 4 + (size_t)a.P * 4;
+    const size_t smem = (size_t)kTmaStages * staged_rows(a) * W * 4 + (size_t)a.P * 4;
     const int64_t tiles = (n4 * 4 + W - 1) / (W > 0 ? W : 1);
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     pull_update_staged_kernel<MODE, SHADOW><<<grid, kTmaThreads, smem, s>>>(a, n4, W);
