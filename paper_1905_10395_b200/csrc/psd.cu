@@ -4,20 +4,26 @@
 // A worker's parameter row is X, row-major.  One pass computes the exact (batch) gradient of every worker
 // and the partial sums of F, so the election loss costs nothing extra on the step that also needs g.
 //
-// CTA (tile, worker) owns 32 rows I of X.  For every 32-row block J it forms the residual tile
-// R = X_I X_J^T - M_IJ (thread (a, b) one entry), adds R^2 to the loss, and accumulates G_I += R X_J.
-// R is never written to memory.  Products and sums are fp64 (the experiment is about reaching high
-// accuracy; fp64 runs at half the fp32 rate on this part and the problem is small), results are
-// rounded once to fp32.
+// CTA (tile, worker) owns 64 rows I of X.  For every 64-row block J it forms the residual tile
+// R = X_I X_J^T - M_IJ, adds R^2 to the loss, and accumulates G_I += R X_J.  R is never written to
+// memory.  Products and sums are fp64 (the experiment is about reaching high accuracy; fp64 runs at half
+// the fp32 rate on this part and the problem is small), results are rounded once to fp32.
+//
+// 256 threads as 16 x 16; each thread holds a 4 x 4 micro-tile of R (rows ty + 16 i, columns tx + 16 j)
+// and 4 x (r / 16) outputs of G, so one shared-memory load feeds four fused multiply-adds; the X tiles
+// are converted to fp64 once when they are staged.
 #include "internal.h"
 
 namespace lsgd {
 namespace {
 
-constexpr int T = 32;
+constexpr int T = 64;            // tile edge
+constexpr int TH = 16;           // threads per tile edge
+constexpr int MT = T / TH;       // micro-tile edge (4)
 constexpr int kMaxRank = 128;
+constexpr int KM = kMaxRank / TH;  // output columns per thread (8)
 
-__global__ void __launch_bounds__(T * T)
+__global__ void __launch_bounds__(TH * TH)
 psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float* __restrict__ M, int32_t n, int32_t r,
                 int64_t ld, double* __restrict__ partials, int32_t n_partials, int write_g) {
   extern __shared__ double s_psd[];
@@ -26,57 +32,91 @@ psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float*
   double* XJ = XI + T * pitch;                  // [T][pitch]
   double* Rt = XJ + T * pitch;                  // [T][T + 1]
   const int i = blockIdx.y, I0 = blockIdx.x * T;
-  const int a = threadIdx.y, b = threadIdx.x, tid = a * T + b;
+  const int ty = threadIdx.y, tx = threadIdx.x, tid = ty * TH + tx;
   const float* xi = x + (int64_t)i * ld;
-  for (int idx = tid; idx < T * r; idx += T * T) {
+  for (int idx = tid; idx < T * r; idx += TH * TH) {
     const int row = idx / r, k = idx - row * r;
     XI[row * pitch + k] = (I0 + row < n) ? (double)xi[(int64_t)(I0 + row) * r + k] : 0.0;
   }
-  double acc[kMaxRank / T];
+  double acc[MT][KM];
 #pragma unroll
-  for (int m = 0; m < kMaxRank / T; ++m) acc[m] = 0.0;
+  for (int a = 0; a < MT; ++a)
+#pragma unroll
+    for (int m = 0; m < KM; ++m) acc[a][m] = 0.0;
   double lsum = 0.0;
   for (int J0 = 0; J0 < n; J0 += T) {
-    for (int idx = tid; idx < T * r; idx += T * T) {
+    for (int idx = tid; idx < T * r; idx += TH * TH) {
       const int row = idx / r, k = idx - row * r;
       XJ[row * pitch + k] = (J0 + row < n) ? (double)xi[(int64_t)(J0 + row) * r + k] : 0.0;
     }
     __syncthreads();
-    double s = 0.0;
-    for (int k = 0; k < r; ++k) s = fma(XI[a * pitch + k], XJ[b * pitch + k], s);
-    const double rab = (I0 + a < n && J0 + b < n) ? s - (double)M[(int64_t)(I0 + a) * n + J0 + b] : 0.0;
-    lsum = fma(rab, rab, lsum);
-    Rt[a * (T + 1) + b] = rab;
-    __syncthreads();
+    // R micro-tile: rows ty + 16 a, columns tx + 16 b
+    double s[MT][MT];
 #pragma unroll
-    for (int m = 0; m < kMaxRank / T; ++m) {
-      const int k = b + T * m;
-      if (k < r) {
-        double t = acc[m];
-#pragma unroll 8
-        for (int bb = 0; bb < T; ++bb) t = fma(Rt[a * (T + 1) + bb], XJ[bb * pitch + k], t);
-        acc[m] = t;
+    for (int a = 0; a < MT; ++a)
+#pragma unroll
+      for (int b = 0; b < MT; ++b) s[a][b] = 0.0;
+    for (int k = 0; k < r; ++k) {
+      double xa[MT], xb[MT];
+#pragma unroll
+      for (int a = 0; a < MT; ++a) xa[a] = XI[(ty + TH * a) * pitch + k];
+#pragma unroll
+      for (int b = 0; b < MT; ++b) xb[b] = XJ[(tx + TH * b) * pitch + k];
+#pragma unroll
+      for (int a = 0; a < MT; ++a)
+#pragma unroll
+        for (int b = 0; b < MT; ++b) s[a][b] = fma(xa[a], xb[b], s[a][b]);
+    }
+#pragma unroll
+    for (int a = 0; a < MT; ++a)
+#pragma unroll
+      for (int b = 0; b < MT; ++b) {
+        const int ri = I0 + ty + TH * a, cj = J0 + tx + TH * b;
+        const double rab = (ri < n && cj < n) ? s[a][b] - (double)M[(int64_t)ri * n + cj] : 0.0;
+        lsum = fma(rab, rab, lsum);
+        Rt[(ty + TH * a) * (T + 1) + tx + TH * b] = rab;
+      }
+    __syncthreads();
+    // G rows ty + 16 a, columns tx + 16 m
+    for (int bb = 0; bb < T; ++bb) {
+      double ra[MT];
+#pragma unroll
+      for (int a = 0; a < MT; ++a) ra[a] = Rt[(ty + TH * a) * (T + 1) + bb];
+#pragma unroll
+      for (int m = 0; m < KM; ++m) {
+        const int k = tx + TH * m;
+        if (k < r) {
+          const double xj = XJ[bb * pitch + k];
+#pragma unroll
+          for (int a = 0; a < MT; ++a) acc[a][m] = fma(ra[a], xj, acc[a][m]);
+        }
       }
     }
     __syncthreads();
   }
-  if (write_g && I0 + a < n) {
-    float* gi = g + (int64_t)i * ld + (int64_t)(I0 + a) * r;
+  if (write_g) {
 #pragma unroll
-    for (int m = 0; m < kMaxRank / T; ++m) {
-      const int k = b + T * m;
-      if (k < r) gi[k] = (float)acc[m];
+    for (int a = 0; a < MT; ++a) {
+      const int ri = I0 + ty + TH * a;
+      if (ri < n) {
+        float* gi = g + (int64_t)i * ld + (int64_t)ri * r;
+#pragma unroll
+        for (int m = 0; m < KM; ++m) {
+          const int k = tx + TH * m;
+          if (k < r) gi[k] = (float)acc[a][m];
+        }
+      }
     }
   }
-  // block sum of R^2 in a fixed order: warp shuffles, then the 32 warp sums in index order
+  // block sum of R^2 in a fixed order: warp shuffles, then the 8 warp sums in index order
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
-  __shared__ double s_w[T];
-  if (b == 0) s_w[a] = lsum;
+  __shared__ double s_w[TH * TH / 32];
+  if ((tid & 31) == 0) s_w[tid >> 5] = lsum;
   __syncthreads();
   if (tid == 0) {
     double t = 0.0;
-    for (int w = 0; w < T; ++w) t += s_w[w];
+    for (int w = 0; w < TH * TH / 32; ++w) t += s_w[w];
     partials[(int64_t)i * n_partials + blockIdx.x] = t;
   }
 }
@@ -91,11 +131,11 @@ cudaError_t launch_psd_grad(const float* x, float* g, const float* M, int32_t n,
   const size_t smem = sizeof(double) * (size_t)(2 * T * pitch + T * (T + 1));
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(psd_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(psd_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid((unsigned)n_partials, (unsigned)P), block(T, T);
+  dim3 grid((unsigned)n_partials, (unsigned)P), block(TH, TH);
   psd_grad_kernel<<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, write_g ? 1 : 0);
   return cudaGetLastError();
 }
