@@ -118,6 +118,10 @@ typedef struct {
   const int32_t* held_y;     /* DEVICE int32[n_heldout]                                              */
   void* scratch;             /* DEVICE, lsgd_mlp_scratch_bytes() bytes, 1024-byte aligned            */
   uint64_t scratch_bytes;
+  int32_t loss_window;       /* 0: lsgd_elect(h, NULL) evaluates the held-out loss.  K in 1..64: it elects
+                                on the mean of each worker's minibatch losses over the last K lsgd_grad
+                                calls, the estimator of the paper's deep-network runs (Section 4.1: the
+                                last 10 / 64 batches); fewer than K are averaged until K have been seen */
 } lsgd_mlp_desc;
 
 typedef struct {

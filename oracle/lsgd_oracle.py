@@ -240,7 +240,13 @@ class Mlp(Objective):
     accumulated in float64; bias gradients are column sums of the *rounded* dz / dh; the relu mask
     is taken from the stored (rounded) activation."""
 
-    def __init__(self, segs, data_x, data_y, batch_idx, held_x, held_y, mode="bf16emu"):
+    def __init__(self, segs, data_x, data_y, batch_idx, held_x, held_y, mode="bf16emu", loss_window=0):
+        # loss_window K > 0: the election loss is the mean of the worker's minibatch losses over the last K
+        # gradient evaluations (Section 4.1: "the average of the training loss computed over the last 10 ...
+        # data batches"), kept in a ring of K slots and averaged in slot order
+        self.loss_window = int(loss_window)
+        self.ring = []
+        self.n_grads = 0
         self.segs = segs
         self.data_x, self.data_y, self.batch_idx = data_x, data_y, batch_idx
         self.held_x, self.held_y = held_x, held_y
@@ -297,9 +303,21 @@ class Mlp(Objective):
                     dh = (delta @ Ws[l]) * (hs[l] > 0.0)
                     delta = self.rd(dh.astype(F32)).astype(F64)
         self.last_train_loss = losses
+        if self.loss_window > 0:
+            slot = self.n_grads % self.loss_window
+            if slot == len(self.ring):
+                self.ring.append(losses.copy())
+            else:
+                self.ring[slot] = losses.copy()
+            self.n_grads += 1
         return g
 
     def loss(self, x, n):
+        if self.loss_window > 0:
+            acc = np.zeros(x.shape[0], dtype=F64)
+            for slot_losses in self.ring:
+                acc = acc + slot_losses.astype(F64)
+            return (acc / len(self.ring)).astype(F32)
         out = np.empty(x.shape[0], dtype=F32)
         for i in range(x.shape[0]):
             _, _, z = self._forward(x[i], self.held_x)

@@ -42,7 +42,7 @@ class PsdDesc(C.Structure):
 class MlpDesc(C.Structure):
     _fields_ = [("dims", C.c_int32 * 4), ("batch", C.c_int32), ("pool", C.c_int32), ("pool_x", C.c_void_p),
                 ("pool_y", C.c_void_p), ("n_heldout", C.c_int32), ("held_x", C.c_void_p), ("held_y", C.c_void_p),
-                ("scratch", C.c_void_p), ("scratch_bytes", C.c_uint64)]
+                ("scratch", C.c_void_p), ("scratch_bytes", C.c_uint64), ("loss_window", C.c_int32)]
 
 
 class BgemmDesc(C.Structure):

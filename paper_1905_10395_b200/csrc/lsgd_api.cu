@@ -292,8 +292,13 @@ lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
         e.partial_scale = 0.25;
         break;
       case LSGD_OBJ_MLP: {
-        if (h->fused_applied) return LSGD_ERR_STATE;   // x is between two steps: no loss at x_t any more
-        lsgd_status st = mlp_heldout_loss(h, h->d_loss);
+        lsgd_status st;
+        if (h->mlp.loss_window > 0) {
+          st = mlp_window_loss(h, h->d_loss);            // running mean of the training losses
+        } else {
+          if (h->fused_applied) return LSGD_ERR_STATE;   // x is between two steps: no loss at x_t any more
+          st = mlp_heldout_loss(h, h->d_loss);
+        }
         if (st != LSGD_OK) return st;
         e.loss_in = h->d_loss;
         break;

@@ -21,6 +21,7 @@ namespace lsgd {
 namespace {
 
 constexpr int kMaxClasses = 16;
+constexpr int kMaxLossWindow = 64;
 
 inline int64_t up32(int64_t n) { return (n + 31) / 32 * 32; }
 inline size_t up1k(size_t n) { return (n + 1023) & ~size_t(1023); }
@@ -42,7 +43,7 @@ Layout param_layout(const int32_t* dims) {
 }
 
 struct Scratch {
-  size_t wb, xb, h1, h2, dh2, dh1, dz, loss_b, xh, hh1, hh2, loss_h, total;
+  size_t wb, xb, h1, h2, dh2, dh1, dz, loss_b, xh, hh1, hh2, loss_h, ring, total;
 };
 Scratch scratch_layout(const int32_t* dims, int64_t ld, int32_t P, int32_t B, int32_t nH) {
   Scratch s{};
@@ -60,6 +61,7 @@ Scratch scratch_layout(const int32_t* dims, int64_t ld, int32_t P, int32_t B, in
   s.hh1 = take((size_t)P * nH * dims[1] * 2);
   s.hh2 = take((size_t)P * nH * dims[2] * 2);
   s.loss_h = take((size_t)P * nH * 4);
+  s.ring = take((size_t)kMaxLossWindow * P * 4);
   s.total = off;
   return s;
 }
@@ -71,7 +73,8 @@ struct MlpState {
   int32_t B, nH, P;
   int64_t ld;
   __nv_bfloat16 *wb, *xb, *h1, *h2, *dh2, *dh1, *xh, *hh1, *hh2;
-  float *dz, *loss_b, *loss_h;
+  float *dz, *loss_b, *loss_h, *ring;   // ring[slot][P]: mean minibatch loss of the last grads
+  int64_t n_grads;
   CUtensorMap m_xb, m_w1, m_w2, m_h1, m_dh2, m_dh1, m_xh, m_hh1;
 };
 
@@ -359,6 +362,15 @@ column_sum_kernel(const __nv_bfloat16* __restrict__ delta, float* __restrict__ g
   }
 }
 
+// out[i] = mean over the first n_slots rows of ring[slot][i], added in slot order in fp64
+__global__ void window_mean_kernel(const float* __restrict__ ring, float* __restrict__ out, int32_t P, int32_t n_slots) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= P) return;
+  double acc = 0.0;
+  for (int sl = 0; sl < n_slots; ++sl) acc += (double)ring[(int64_t)sl * P + i];
+  out[i] = (float)(acc / (double)n_slots);
+}
+
 // out[i] = mean_b v[i][b], summed in a fixed order by one warp per worker.
 __global__ void __launch_bounds__(32) row_mean_kernel(const float* __restrict__ v, float* __restrict__ out, int32_t n) {
   const int i = blockIdx.x, lane = threadIdx.x;
@@ -402,6 +414,7 @@ lsgd_status mlp_validate(const lsgd_config& c, const lsgd_mlp_desc& m) {
   for (int l = 0; l < 4; ++l)
     if (m.dims[l] < 1) return LSGD_ERR_INVALID_ARG;
   if (m.batch < 1 || m.pool < 1 || m.n_heldout < 1) return LSGD_ERR_INVALID_ARG;
+  if (m.loss_window < 0 || m.loss_window > kMaxLossWindow) return LSGD_ERR_INVALID_ARG;
   if (!m.pool_x || !m.pool_y || !m.held_x || !m.held_y || !m.scratch) return LSGD_ERR_INVALID_ARG;
   // TMA rows must be 16-byte multiples (8 bf16); the head kernels keep the class scores in registers
   if (m.dims[0] % 8 || m.dims[1] % 8 || m.dims[2] % 8 || m.dims[3] > kMaxClasses) return LSGD_ERR_UNSUPPORTED;
@@ -443,6 +456,8 @@ lsgd_status mlp_create(lsgd_ctx* h) {
   st->hh1 = reinterpret_cast<__nv_bfloat16*>(base + st->S.hh1);
   st->hh2 = reinterpret_cast<__nv_bfloat16*>(base + st->S.hh2);
   st->loss_h = reinterpret_cast<float*>(base + st->S.loss_h);
+  st->ring = reinterpret_cast<float*>(base + st->S.ring);
+  st->n_grads = 0;
 
   const int32_t* d = st->dims;
   const int64_t B = st->B, nH = st->nH, P = st->P, ld = st->ld;
@@ -490,6 +505,10 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
       return LSGD_ERR_CUDA;
     bwd_attr = true;
   }
+  if (m.loss_window > 0) {   // remember this step's mean minibatch losses for the running-mean election
+    row_mean_kernel<<<P, 32, 0, s>>>(st->loss_b, st->ring + (st->n_grads % m.loss_window) * P, B);
+    st->n_grads++;
+  }
   head_backward_kernel<<<dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdThreadsX, kBwdSlices), bwd_smem, s>>>(
       st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]);
   if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
@@ -533,6 +552,15 @@ lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss) {
       st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr, st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2], st->L.b[2], st->nH,
       kGroups, h->d_status);
   row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_h, loss, st->nH);
+  return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
+}
+
+lsgd_status mlp_window_loss(lsgd_ctx* h, float* loss) {
+  MlpState* st = state(h);
+  const int K = h->mlp.loss_window;
+  if (!st || K < 1 || st->n_grads < 1) return LSGD_ERR_STATE;   // nothing recorded yet
+  const int n_slots = st->n_grads < K ? (int)st->n_grads : K;
+  window_mean_kernel<<<(st->P + 127) / 128, 128, 0, h->stream>>>(st->ring, loss, st->P, n_slots);
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
 }
 

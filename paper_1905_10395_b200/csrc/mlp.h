@@ -11,6 +11,7 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd);
 // the parameter ranges lsgd_step still has to update after a fused lsgd_grad: {offset, length} pairs
 int mlp_unfused_ranges(lsgd_ctx* h, int64_t (*ranges)[2]);
 lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss);
+lsgd_status mlp_window_loss(lsgd_ctx* h, float* loss);  // mean of the recorded minibatch losses (loss_window)
 lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss);   // mean minibatch loss of the last lsgd_grad
 lsgd_status mlp_refresh_shadow(lsgd_ctx* h);             // bf16 copy of the weights <- x
 uint16_t* mlp_weight_shadow(lsgd_ctx* h);

@@ -75,7 +75,7 @@ class Population:
             sp = (self.scratch.data_ptr() + 1023) // 1024 * 1024
             desc = api.MlpDesc((C.c_int32 * 4)(*m["dims"]), m["batch"], len(A["pool_y"]), self.pool_x.data_ptr(),
                                self.pool_y.data_ptr(), len(A["held_y"]), self.held_x.data_ptr(),
-                               self.held_y.data_ptr(), sp, nbytes)
+                               self.held_y.data_ptr(), sp, nbytes, int(m.get("loss_window", 0)))
             self.batches = [torch.from_numpy(np.ascontiguousarray(p)).to(dev) for p in A["batch_idx"]]
             if self.g is None:
                 self.g = torch.empty_like(self.x)

@@ -21,7 +21,8 @@ def loss_close(got, ref):
 def _oracle(w):
     A = w.arrays
     segs, _ = inputs.mlp_layout(w.meta["dims"])
-    obj = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="bf16emu")
+    obj = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="bf16emu",
+                  loss_window=int(w.meta.get("loss_window", 0)))
     return orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
 
 
@@ -177,3 +178,20 @@ def test_fused_weight_step_is_bit_identical_to_the_materialised_gradient_path():
     a.lsgd.step()
     a.close()
     b.close()
+
+
+def test_election_on_the_running_mean_of_training_losses():
+    """loss_window = 3: leaders are elected on the mean of the last three minibatch losses of each worker."""
+    w = inputs.make_mlp(4, 2, dims=(40, 72, 136, 7), pool=256, heldout=40, batch=24, n_classes=7, steps=8, tau=2,
+                        config_id=83)
+    w.meta["loss_window"] = 3
+    pop, o, tg, tr, forced = _run_pair(w, 8)
+    _check(pop, o, w, tg, tr, forced)
+    for hg, ho in zip(pop.history, o.history):
+        assert loss_close(hg["loss"], ho["loss"])
+    # the elected-on loss is the window mean, not the held-out loss
+    k = len(pop.history) - 1
+    t_last = pop.history[k]["t"]
+    want = np.mean([tg[t] for t in range(max(0, t_last - 2), t_last + 1)], axis=0)
+    assert np.allclose(pop.history[k]["loss"], want, rtol=1e-5, atol=0)
+    pop.close()

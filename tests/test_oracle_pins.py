@@ -456,3 +456,16 @@ def test_psd_completion_gradient_and_monotone_descent():
     o.run(60)
     best = [float(h["loss"].min()) for h in o.history]
     assert all(b1 <= b0 for b0, b1 in zip(best, best[1:])) and best[-1] < 0.5 * best[0]
+
+
+# ---- running-mean election loss of the deep-network runs (Section 4.1) ------------------------------
+def test_mlp_running_mean_election_loss():
+    w, segs, _ = _tiny_mlp("fp32")
+    A = w.arrays
+    obj = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="fp32", loss_window=3)
+    seen = []
+    for t in range(5):
+        obj.grad(w.x0 * F32(1.0 + 0.1 * t), t)
+        seen.append(obj.last_train_loss.astype(F64))
+        want = np.mean(seen[-3:], axis=0)
+        assert np.allclose(obj.loss(w.x0, 0), want, rtol=1e-6, atol=0)
