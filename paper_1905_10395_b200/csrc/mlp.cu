@@ -43,7 +43,7 @@ Layout param_layout(const int32_t* dims) {
 }
 
 struct Scratch {
-  size_t wb, xb, h1, h2, dh2, dh1, dz, loss_b, xh, hh1, hh2, loss_h, ring, total;
+  size_t wb, xb, h1, h2, dh2, dh1, dz, loss_b, xh, hh1, hh2, loss_h, ring, logits, total;
 };
 Scratch scratch_layout(const int32_t* dims, int64_t ld, int32_t P, int32_t B, int32_t nH) {
   Scratch s{};
@@ -62,6 +62,7 @@ Scratch scratch_layout(const int32_t* dims, int64_t ld, int32_t P, int32_t B, in
   s.hh2 = take((size_t)P * nH * dims[2] * 2);
   s.loss_h = take((size_t)P * nH * 4);
   s.ring = take((size_t)kMaxLossWindow * P * 4);
+  s.logits = take((size_t)P * nH * kMaxClasses * 4);
   s.total = off;
   return s;
 }
@@ -73,9 +74,10 @@ struct MlpState {
   int32_t B, nH, P;
   int64_t ld;
   __nv_bfloat16 *wb, *xb, *h1, *h2, *dh2, *dh1, *xh, *hh1, *hh2;
+  float* logits;                         // held-out logits [P][nH][kMaxClasses] (fp32)
   float *dz, *loss_b, *loss_h, *ring;   // ring[slot][P]: mean minibatch loss of the last grads
   int64_t n_grads;
-  CUtensorMap m_xb, m_w1, m_w2, m_h1, m_dh2, m_dh1, m_xh, m_hh1;
+  CUtensorMap m_xb, m_w1, m_w2, m_w3, m_h1, m_dh2, m_dh1, m_xh, m_hh1, m_hh2;
 };
 
 // ------------------------------------------------------------------------------------ small kernels
@@ -362,6 +364,38 @@ column_sum_kernel(const __nv_bfloat16* __restrict__ delta, float* __restrict__ g
   }
 }
 
+// Per-sample softmax cross-entropy from stored logits (+ bias): one thread per sample.
+__global__ void __launch_bounds__(256)
+logits_loss_kernel(const float* __restrict__ logits, const float* __restrict__ x, const int32_t* __restrict__ labels,
+                   float* __restrict__ loss_b, int32_t n, int32_t C, int64_t ld, int64_t b3_off, uint32_t* status) {
+  const int i = blockIdx.y;
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= n) return;
+  const float* z = logits + ((int64_t)i * n + b) * kMaxClasses;
+  const float* b3 = x + (int64_t)i * ld + b3_off;
+  int cls = labels[b];
+  if (cls < 0 || cls >= C) {
+    atomicOr(status, FLAG_BAD_INDEX);
+    cls = 0;
+  }
+  float v[kMaxClasses];
+  float zmax = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < kMaxClasses; ++c)
+    if (c < C) {
+      v[c] = z[c] + b3[c];
+      zmax = fmaxf(zmax, v[c]);
+    }
+  float sum = 0.f, zy = 0.f;
+#pragma unroll
+  for (int c = 0; c < kMaxClasses; ++c)
+    if (c < C) {
+      sum += expf(v[c] - zmax);
+      if (c == cls) zy = v[c];
+    }
+  loss_b[(int64_t)i * n + b] = zmax + logf(sum) - zy;
+}
+
 // out[i] = mean over the first n_slots rows of ring[slot][i], added in slot order in fp64
 __global__ void window_mean_kernel(const float* __restrict__ ring, float* __restrict__ out, int32_t P, int32_t n_slots) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -457,6 +491,7 @@ lsgd_status mlp_create(lsgd_ctx* h) {
   st->hh2 = reinterpret_cast<__nv_bfloat16*>(base + st->S.hh2);
   st->loss_h = reinterpret_cast<float*>(base + st->S.loss_h);
   st->ring = reinterpret_cast<float*>(base + st->S.ring);
+  st->logits = reinterpret_cast<float*>(base + st->S.logits);
   st->n_grads = 0;
 
   const int32_t* d = st->dims;
@@ -470,6 +505,8 @@ lsgd_status mlp_create(lsgd_ctx* h) {
   ok = ok && make_operand_map(&st->m_dh1, st->dh1, d[1], B, d[1], P, B * d[1]);
   ok = ok && make_operand_map(&st->m_xh, st->xh, d[0], nH, d[0], 1, 0);
   ok = ok && make_operand_map(&st->m_hh1, st->hh1, d[1], nH, d[1], P, nH * d[1]);
+  ok = ok && make_operand_map(&st->m_hh2, st->hh2, d[2], nH, d[2], P, nH * d[2]);
+  ok = ok && make_operand_map(&st->m_w3, st->wb + st->L.w[2], d[2], d[3], d[2], P, ld);
   if (!ok) return LSGD_ERR_CUDA;
 
   // bf16 copies of the weights and of the held-out inputs; gradient padding cleared once
@@ -546,11 +583,21 @@ lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss) {
   const int32_t* d = st->dims;
   lsgd_status fs = forward_hidden(h, st->m_xh, 0, st->nH, st->hh1, st->m_hh1, st->hh2);
   if (fs != LSGD_OK) return fs;
-  constexpr int kS = 4, kGroups = 2;   // 8 warps x 2 groups x 4 samples = 64 samples per CTA
-  const int per_cta = kHeadWarps * kGroups * kS;
-  head_forward_kernel<kS><<<dim3((st->nH + per_cta - 1) / per_cta, st->P), kHeadWarps * 32, (size_t)d[3] * d[2] * 2, h->stream>>>(
-      st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr, st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2], st->L.b[2], st->nH,
-      kGroups, h->d_status);
+  if (st->nH >= 512) {
+    // large held-out batch: the logits are one more tensor-core product (N = n_classes, zero-filled to a
+    // tile by TMA), followed by a per-sample softmax
+    GemmShape g3 = shape(st->nH, d[3], d[2], st->P, 0, 0, 1, GEMM_EPI_F32, st->logits, kMaxClasses,
+                         (int64_t)st->nH * kMaxClasses, h->d_status);
+    if (launch_bgemm(st->m_hh2, st->m_w3, g3, h->stream) != cudaSuccess) return LSGD_ERR_CUDA;
+    logits_loss_kernel<<<dim3((st->nH + 255) / 256, st->P), 256, 0, h->stream>>>(st->logits, c.x, m.held_y, st->loss_h, st->nH,
+                                                                              d[3], st->ld, st->L.b[2], h->d_status);
+  } else {
+    constexpr int kS = 4, kGroups = 2;   // 8 warps x 2 groups x 4 samples = 64 samples per CTA
+    const int per_cta = kHeadWarps * kGroups * kS;
+    head_forward_kernel<kS><<<dim3((st->nH + per_cta - 1) / per_cta, st->P), kHeadWarps * 32, (size_t)d[3] * d[2] * 2, h->stream>>>(
+        st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr, st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2], st->L.b[2], st->nH,
+        kGroups, h->d_status);
+  }
   row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_h, loss, st->nH);
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
 }
