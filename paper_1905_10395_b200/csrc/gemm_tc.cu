@@ -34,20 +34,19 @@
 namespace lsgd {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64;
+constexpr int BM = 128, BK = 64;                            // tile rows, k-slice; the tile width BN (128 or 256) is a template parameter
 constexpr int kMaxStages = 6;
-constexpr int kStageBytes = (BM * BK + BN * BK) * 2;       // 32 KiB
 constexpr int kABytes = BM * BK * 2;                        // 16 KiB
-constexpr int kEpiF32Bytes = BM * BN * 4;                   // 64 KiB: fp32 tile, 4 boxes of [128][32 floats]
-constexpr int kEpiBf16Bytes = BM * BN * 2;                  // 32 KiB: bf16 tile, 2 boxes of [128][64 bf16]
 constexpr int kThreads = 192;                               // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
-// Shared memory is carved per epilogue kind (224 KiB + alignment slack in every case):
-//   bf16 outputs      : 6 operand stages + 1 bf16 tile
-//   fp32 output       : 5 operand stages + 1 fp32 tile
-//   fused SGD step    : 2 operand stages (these products have K <= 128) + 2 fp32 tiles (the x tile of the
-//                       next tile is loaded while the current one is updated) + 1 bf16 tile
+// Shared memory is carved per epilogue kind (at most 224 KiB + alignment slack):
+//   bf16 outputs, 128-wide tiles : 6 operand stages (32 KiB) + 1 bf16 tile (32 KiB)
+//   bf16 outputs, 256-wide tiles : 3 operand stages (48 KiB) + 1 bf16 tile (64 KiB); used when the product has
+//                                  enough tiles to fill the machine twice -- a quarter less operand traffic
+//                                  from L2 per flop, which is what bounds the M = 1024 forward products
+//   fp32 output                  : 5 operand stages + 1 fp32 tile (64 KiB)
+//   fused SGD step               : 2 operand stages (these products have K <= 128) + 2 fp32 tiles (the x tile of
+//                                  the next tile is loaded while the current one is updated) + 1 bf16 tile
 constexpr int kSmemBytes = 224 * 1024 + 1024;
-constexpr uint32_t kTmemCols = 256;                         // two accumulator tiles
 constexpr long long kWaitBudgetCycles = 2000000000LL;       // about one second
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -137,22 +136,27 @@ __device__ __forceinline__ uint32_t swz(int r, int u) { return (uint32_t)(r * 12
 struct Tile {
   int z, m0, n0;
 };
-__device__ __forceinline__ Tile tile_of(int t, int mt, int nt) {
+__device__ __forceinline__ Tile tile_of(int t, int mt, int nt, int bn) {
   Tile q;
-  q.n0 = (t % nt) * BN;
+  q.n0 = (t % nt) * bn;
   t /= nt;
   q.m0 = (t % mt) * BM;
   q.z = t / mt;
   return q;
 }
 
+template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_aux, GemmShape p) {
+  constexpr int kStageBytes = (BM * BK + BN * BK) * 2;     // 32 or 48 KiB
+  constexpr int kEpiF32Bytes = BM * BN * 4;                 // fp32 tile: BN / 32 boxes of [128][32 floats]
+  constexpr int kEpiBf16Bytes = BM * BN * 2;                // bf16 tile: BN / 64 boxes of [128][64 bf16]
+  constexpr uint32_t kTmemCols = 2 * BN;                    // two accumulator tiles
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const bool sgd = (p.epilogue == GEMM_EPI_SGD);
-  const int kStages = sgd ? 2 : (p.epilogue == GEMM_EPI_F32 ? 5 : 6);
+  const int kStages = BN == 256 ? 3 : (sgd ? 2 : (p.epilogue == GEMM_EPI_F32 ? 5 : 6));
   const int nx = sgd ? 2 : 1;                               // input-tile buffers (x is double-buffered)
   uint8_t* buf_f32_0 = smem + kStages * kStageBytes;        // fp32 tile(s): C out, or x in/out (SGD)
   uint8_t* buf_b16 = buf_f32_0 + (sgd ? 2 : (p.epilogue == GEMM_EPI_F32 ? 1 : 0)) * kEpiF32Bytes;   // bf16 tile: C out, mask in, bf16 x out
@@ -202,7 +206,7 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     int local = 0;          // tiles this CTA has started
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
-      const Tile q = tile_of(t, mt, nt);
+      const Tile q = tile_of(t, mt, nt, BN);
       const int za = p.a_batched ? q.z : 0, zb = p.b_batched ? q.z : 0;
       for (int kt = 0; kt < nk; ++kt, ++it) {
         const int s = it % kStages;
@@ -220,12 +224,10 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           tma_load_3d(sa, &map_a, &full_bar[s], k0, q.m0, za);
           tma_load_3d(sa + 8192, &map_a, &full_bar[s], k0, q.m0 + 64, za);
         }
-        if (p.b_mn) {
-          tma_load_3d(sb, &map_b, &full_bar[s], q.n0, k0, zb);
-          tma_load_3d(sb + 8192, &map_b, &full_bar[s], q.n0 + 64, k0, zb);
-        } else {
-          tma_load_3d(sb, &map_b, &full_bar[s], k0, q.n0, zb);
-          tma_load_3d(sb + 8192, &map_b, &full_bar[s], k0, q.n0 + 64, zb);
+#pragma unroll
+        for (int j = 0; j < BN / 64; ++j) {
+          if (p.b_mn) tma_load_3d(sb + j * 8192, &map_b, &full_bar[s], q.n0 + 64 * j, k0, zb);
+          else tma_load_3d(sb + j * 8192, &map_b, &full_bar[s], k0, q.n0 + 64 * j, zb);
         }
       }
       if (ok && reads_tile) {
@@ -242,7 +244,7 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         } else {
           mbar_expect_tx(&in_full[xb], kEpiBf16Bytes);
 #pragma unroll
-          for (int c = 0; c < 2; ++c) tma_load_3d(buf_b16 + c * 16384, &map_aux, &in_full[xb], q.n0 + c * 64, q.m0, q.z);
+          for (int c = 0; c < BN / 64; ++c) tma_load_3d(buf_b16 + c * 16384, &map_aux, &in_full[xb], q.n0 + c * 64, q.m0, q.z);
         }
       }
     }
@@ -283,7 +285,7 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     int local = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
-      const Tile q = tile_of(t, mt, nt);
+      const Tile q = tile_of(t, mt, nt, BN);
       const int b = local & 1;
       ok = mbar_wait(&acc_full[b], (local >> 1) & 1, abort_flag, p.status);
       const int xb = local % nx;
@@ -388,13 +390,13 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (leader) {
         if (p.epilogue == GEMM_EPI_F32 || p.epilogue == GEMM_EPI_SGD) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
+          for (int c = 0; c < BN / 32; ++c)
             if (q.n0 + c * 32 < p.N) tma_store_3d(buf_f32 + c * 16384, &map_c, q.n0 + c * 32, q.m0, q.z);
         }
         if (p.epilogue != GEMM_EPI_F32) {
           const CUtensorMap* mo = (p.epilogue == GEMM_EPI_SGD) ? &map_aux : &map_c;
 #pragma unroll
-          for (int c = 0; c < 2; ++c)
+          for (int c = 0; c < BN / 64; ++c)
             if (q.n0 + c * 64 < p.N) tma_store_3d(buf_b16 + c * 16384, mo, q.n0 + c * 64, q.m0, q.z);
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -468,7 +470,9 @@ cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, con
   static bool attr_set = false;
   static int sms = 0;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(bgemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(bgemm_bf16_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(bgemm_bf16_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -500,9 +504,17 @@ cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, con
       break;
   }
   if (!ok) return cudaErrorInvalidValue;
-  const int64_t tiles = (int64_t)((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM) * p.batch;
-  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-  bgemm_bf16_kernel<<<grid, kThreads, kSmemBytes, s>>>(map_a, map_b, map_c, map_aux, p);
+  const int64_t mtiles = (p.M + BM - 1) / BM;
+  const int64_t tiles256 = (int64_t)((p.N + 255) / 256) * mtiles * p.batch;
+  const bool bf16_out = p.epilogue != GEMM_EPI_F32 && p.epilogue != GEMM_EPI_SGD;
+  if (bf16_out && p.N >= 256 && tiles256 >= 2 * (int64_t)sms) {
+    const unsigned grid = (unsigned)(tiles256 < sms ? tiles256 : sms);
+    bgemm_bf16_kernel<256><<<grid, kThreads, kSmemBytes, s>>>(map_a, map_b, map_c, map_aux, p);
+  } else {
+    const int64_t tiles = (int64_t)((p.N + 127) / 128) * mtiles * p.batch;
+    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    bgemm_bf16_kernel<128><<<grid, kThreads, kSmemBytes, s>>>(map_a, map_b, map_c, map_aux, p);
+  }
   return cudaGetLastError();
 }
 

@@ -88,3 +88,21 @@ def test_bgemm_epilogues_and_shared_operand():
     assert torch.equal(got, want)
     got = _run(api, torch, A, B, M, N, K, batch, 0, 0, epilogue=3, share_a=True)
     assert torch.equal(got, ref.to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 1)])
+def test_bgemm_wide_tiles_on_large_products(a_mn, b_mn):
+    """Products with enough tiles use 256-wide tiles (bf16 outputs only): ragged M, N, K, every epilogue."""
+    import torch
+    from paper_1905_10395_b200 import api
+    gen = torch.Generator(device="cuda").manual_seed(31 + 2 * a_mn + b_mn)
+    M, N, K, batch = 1000, 1096, 200, 12                      # 8 x 5 x 12 = 480 wide tiles
+    A, B, ref = _operands(torch, gen, M, N, K, batch, a_mn, b_mn, integer=True)
+    got = _run(api, torch, A, B, M, N, K, batch, a_mn, b_mn, epilogue=3)
+    assert torch.equal(got, ref.to(torch.bfloat16))
+    bias = torch.randint(-3, 4, (batch, N), generator=gen, device="cuda").float()
+    got = _run(api, torch, A, B, M, N, K, batch, a_mn, b_mn, epilogue=1, bias=bias)
+    assert torch.equal(got, torch.relu(ref + bias[:, None, :].double()).to(torch.bfloat16))
+    mask = torch.randint(-1, 2, (batch, M, N), generator=gen, device="cuda").to(torch.bfloat16)
+    got = _run(api, torch, A, B, M, N, K, batch, a_mn, b_mn, epilogue=2, mask=mask)
+    assert torch.equal(got, torch.where(mask.double() > 0, ref, torch.zeros_like(ref)).to(torch.bfloat16))
