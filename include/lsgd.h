@@ -174,7 +174,9 @@ typedef struct {
 
 /* Validates the configuration on the host, copies the group map, builds the group tables and
  * allocates O(P + G) words of device state plus reduction scratch for the objective's election
- * loss.  Returns LSGD_ERR_CUDA if no CUDA device is usable.  *out is NULL on failure.            */
+ * loss (MATCOMP additionally 8 bytes per worker-parameter for its order-independent gradient
+ * accumulator).  Nothing is allocated after this call.  Returns LSGD_ERR_CUDA if no CUDA device is
+ * usable.  *out is NULL on failure.                                                              */
 LSGD_API lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out);
 
 /* Step 1: stochastic gradients of all workers at the current x (Eq. (1): g_t^{j,i}).

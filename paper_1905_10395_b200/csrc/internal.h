@@ -97,7 +97,8 @@ struct MatcompArgs {
   int32_t P;
   uint32_t* status;
 };
-cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, cudaStream_t s);
+// acc: DEVICE u64[P*ld] fixed-point accumulator, all zero on entry and again on exit
+cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, cudaStream_t s);
 int32_t matcomp_loss_blocks(int32_t n_heldout);
 cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials, int32_t n_partials,
                                          cudaStream_t s);
@@ -133,4 +134,5 @@ struct lsgd_ctx {
   bool fused_applied;        // MLP: the pending gradient has already stepped W1, W2 (plain step)
   const float* armed_noise;  // QUADRATIC with g == NULL: noise pointer for the next step
   void* mlp_state;           // opaque MLP pipeline state
+  unsigned long long* d_acc64;  // MATCOMP: fixed-point gradient accumulator [P*ld], kept all-zero between steps
 };

@@ -115,6 +115,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->armed_noise = nullptr;
   h->slab = nullptr;
   h->mlp_state = nullptr;
+  h->d_acc64 = nullptr;
   std::memset(&h->quad, 0, sizeof(h->quad));
   std::memset(&h->mc, 0, sizeof(h->mc));
   std::memset(&h->mlp, 0, sizeof(h->mlp));
@@ -183,10 +184,17 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   // the host vectors die at return: drain the copies now (creation is not on the hot path)
   ok = ok && cudaStreamSynchronize(h->stream) == cudaSuccess;
   if (ok && cfg->objective == LSGD_OBJ_MLP) ok = (mlp_create(h) == LSGD_OK);
+  if (ok && cfg->objective == LSGD_OBJ_MATCOMP) {
+    const size_t bytes = sizeof(unsigned long long) * (size_t)P * (size_t)cfg->ld;
+    ok = cudaMalloc(reinterpret_cast<void**>(&h->d_acc64), bytes) == cudaSuccess &&
+         cudaMemsetAsync(h->d_acc64, 0, bytes, h->stream) == cudaSuccess;
+  }
   // the gradient kernel of this objective writes columns < d only: clear the padding of g once
   if (ok && cfg->objective == LSGD_OBJ_PSD_COMPLETION && cfg->ld > cfg->d)
     ok = cudaMemsetAsync(cfg->g, 0, sizeof(float) * (size_t)P * (size_t)cfg->ld, h->stream) == cudaSuccess;
   if (!ok) {
+    if (h->mlp_state) mlp_destroy(h);
+    cudaFree(h->d_acc64);
     cudaFree(h->slab);
     delete h;
     return LSGD_ERR_CUDA;
@@ -214,7 +222,7 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
     case LSGD_OBJ_MATCOMP: {
       if (!batch) return LSGD_ERR_INVALID_ARG;
       MatcompArgs a{h->mc, c.x, c.g, c.ld, c.P, h->d_status};
-      LSGD_CUDA(launch_matcomp_grad(a, static_cast<const int32_t*>(batch), h->stream));
+      LSGD_CUDA(launch_matcomp_grad(a, static_cast<const int32_t*>(batch), h->d_acc64, h->stream));
       break;
     }
     case LSGD_OBJ_PSD_COMPLETION:
@@ -428,6 +436,7 @@ lsgd_status lsgd_destroy(lsgd_handle h) {
   if (!h) return LSGD_OK;
   cudaStreamSynchronize(h->stream);
   if (h->mlp_state) mlp_destroy(h);
+  cudaFree(h->d_acc64);
   cudaError_t e = cudaFree(h->slab);
   delete h;
   return e == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;

@@ -7,9 +7,12 @@
 //   election loss: (1/N) sum over the held-out list of e^2, fp64 partial sums in a fixed order.
 //
 // The whole state of this workload (a few MB per worker) lives in L2; the kernels are gather /
-// scatter bound, not HBM bound.  The gradient buffer is cleared and then accumulated with fp32
-// reductions in L2; rows hit once or twice in a batch are order-independent (fp addition commutes),
-// rows hit three or more times may differ in the last bit from run to run.
+// scatter bound, not HBM bound.  Duplicated rows and columns of a batch make the gradient a scatter-ADD.
+// To keep it independent of the order in which the adds land, every contribution e * y / B is evaluated
+// in fp64, converted to 2^-44 fixed point and added with 64-bit integer atomics (integer addition is
+// associative, so the sum is exact and the same on every run); a second kernel converts the sums to fp32
+// and clears the accumulator for the next step.  |contribution| < 2^4 and at most 2^15 of them meet in one
+// entry, so the 64-bit sum cannot overflow; the resolution is 5.7e-14.
 #include "internal.h"
 
 namespace lsgd {
@@ -19,8 +22,11 @@ constexpr int kThreads = 256;
 constexpr int kMaxRank = 32;
 constexpr int kLossPerThread = 4;
 
+constexpr double kFixScale = 17592186044416.0;        // 2^44
+constexpr double kFixInv = 1.0 / 17592186044416.0;
+
 __global__ void __launch_bounds__(kThreads)
-matcomp_grad_kernel(MatcompArgs a, const int32_t* __restrict__ pos) {
+matcomp_grad_kernel(MatcompArgs a, const int32_t* __restrict__ pos, unsigned long long* __restrict__ acc) {
   const int i = blockIdx.y;
   const int p = blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= a.m.batch) return;
@@ -38,22 +44,33 @@ matcomp_grad_kernel(MatcompArgs a, const int32_t* __restrict__ pos) {
   const int64_t xo = (int64_t)i * a.ld + (int64_t)r * rank;
   const int64_t yo = (int64_t)i * a.ld + ((int64_t)a.m.n_rows + c) * rank;
   float xr[kMaxRank], yc[kMaxRank];
-  float dot = 0.f;
+  double dot = 0.0;
 #pragma unroll
   for (int k = 0; k < kMaxRank; ++k) {
     if (k < rank) {
       xr[k] = a.x[xo + k];
       yc[k] = a.x[yo + k];
-      dot = fmaf(xr[k], yc[k], dot);
+      dot += (double)xr[k] * (double)yc[k];
     }
   }
-  const float e = (dot - a.m.obs_v[q]) / (float)a.m.batch;
+  const double e = (dot - (double)a.m.obs_v[q]) / (double)a.m.batch * kFixScale;
 #pragma unroll
   for (int k = 0; k < kMaxRank; ++k) {
     if (k < rank) {
-      atomicAdd(a.g + xo + k, e * yc[k]);
-      atomicAdd(a.g + yo + k, e * xr[k]);
+      atomicAdd(acc + xo + k, (unsigned long long)__double2ll_rn(e * (double)yc[k]));
+      atomicAdd(acc + yo + k, (unsigned long long)__double2ll_rn(e * (double)xr[k]));
     }
+  }
+}
+
+// g <- fixed-point sums as fp32; the accumulator is cleared on the way
+__global__ void __launch_bounds__(kThreads)
+matcomp_finish_kernel(unsigned long long* __restrict__ acc, float* __restrict__ g, int64_t total) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+    const long long v = (long long)acc[e];
+    if (v != 0) acc[e] = 0ull;
+    g[e] = (float)((double)v * kFixInv);
   }
 }
 
@@ -100,11 +117,13 @@ matcomp_loss_kernel(MatcompArgs a, double* __restrict__ partials, int32_t n_part
 
 }  // namespace
 
-cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, cudaStream_t s) {
-  cudaError_t e = cudaMemsetAsync(a.g, 0, sizeof(float) * (size_t)a.P * (size_t)a.ld, s);
-  if (e != cudaSuccess) return e;
+cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, cudaStream_t s) {
   dim3 grid((unsigned)((a.m.batch + kThreads - 1) / kThreads), (unsigned)a.P);
-  matcomp_grad_kernel<<<grid, kThreads, 0, s>>>(a, pos);
+  matcomp_grad_kernel<<<grid, kThreads, 0, s>>>(a, pos, acc);
+  const int64_t total = (int64_t)a.P * a.ld;
+  int64_t blocks = (total + kThreads - 1) / kThreads;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  matcomp_finish_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(acc, a.g, total);
   return cudaGetLastError();
 }
 

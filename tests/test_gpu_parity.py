@@ -325,3 +325,20 @@ def test_psd_completion_lgd(n, r):
     assert rel_err(pop.x_host(), o.x) <= TOL
     assert pop.lsgd.check_device() == 0
     pop.close()
+
+
+def test_matcomp_gradient_is_reproducible_bit_for_bit():
+    # heavy duplication (batch 3000 over 60 rows / 50 columns): the scatter-add must not depend on atomics order
+    w = inputs.make_matcomp(4, 2, n_rows=60, n_cols=50, rank=10, n_obs=2500, n_heldout=256, batch=3000, steps=4, tau=2,
+                            config_id=57)
+    runs = []
+    for _ in range(3):
+        pop = _pop(w)
+        pop.run(4)
+        runs.append(pop.x_host().copy())
+        pop.close()
+    assert np.array_equal(runs[0].view(np.uint32), runs[1].view(np.uint32))
+    assert np.array_equal(runs[0].view(np.uint32), runs[2].view(np.uint32))
+    o = _oracle(w)
+    o.run(4)
+    assert rel_err(runs[0], o.x) <= TOL
