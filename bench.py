@@ -258,6 +258,13 @@ def run_ours(args):
     P, G, d = spec["P"], spec["G"], spec["d"]
     steps, warmup = args.steps, max(args.warmup, 3)
 
+    # --graph: everything runs on a side stream so that whole periods can be captured into a CUDA graph
+    gstream = None
+    if args.graph:
+        import contextlib
+        gstream = torch.cuda.Stream(dev)
+        _stack = contextlib.ExitStack()
+        _stack.enter_context(torch.cuda.stream(gstream))
     # ---- inputs: generated on the host from the seed (C4: into pinned memory, also used by the e2e leg)
     hx = hg = None
     if spec["kind"] == "external":
@@ -271,10 +278,10 @@ def run_ours(args):
         pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith, algorithm1=alg1)
     elif spec["kind"] == "psd":
         w = inputs.make_psd(P=P, n=spec["n"], r=spec["r"], steps=steps)
-        pop = Population(w, device=str(dev), arithmetic=args.arith)
+        pop = Population(w, device=str(dev), arithmetic=args.arith, stream=gstream)
     else:
         w = inputs.config(spec["cfg"], tau=spec["tau"])
-        pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith,
+        pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith, stream=gstream,
                          flags=0 if args.mlp_unfused_step else api.FLAG_MLP_FUSED_STEP)
     launches_per_step = lambda t: spec["launches"][0] if t % spec["tau"] == 0 else spec["launches"][1]
     torch.cuda.synchronize(dev)
@@ -383,6 +390,28 @@ def run_ours(args):
         "gpu_launches": n_launch,
     }
 
+    # ---- the same steps replayed from a CUDA graph (whole periods and whole passes over the batch ring)
+    if args.graph and spec["kind"] in ("quadratic", "matcomp", "mlp") and world == 1:
+        import math
+        cap = spec["tau"] * (len(pop.batches) if pop.batches else 1) // math.gcd(spec["tau"], len(pop.batches) if pop.batches else 1)
+        while pop.t % cap:
+            pop.step()
+        pop.capture(cap)
+        pop.replay()                                # warm replay
+        reps = max(1, steps // cap)
+        torch.cuda.synchronize(dev)
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        q0.record()
+        for _ in range(reps):
+            pop.replay()
+        q1.record()
+        torch.cuda.synchronize(dev)
+        g_ms_step = q0.elapsed_time(q1) / (reps * cap)
+        line["graph"] = {"ms_per_step": g_ms_step, "steps_per_s": 1e3 / g_ms_step, "value": P * d / (g_ms_step * 1e-3),
+                         "steps": reps * cap, "steps_per_graph": cap}
+        if pop.lsgd.check_device() != 0:
+            raise SystemExit("device status word set during the graph replays")
+
     # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs, D2H of its result
     if rank == 0 and world == 1 and not args.no_e2e and hx is not None and not alg1_mode:
         e_steps = args.e2e_steps
@@ -442,6 +471,7 @@ def main():
     ap.add_argument("--schedule", default="fused", choices=["fused", "algorithm1"],
                     help="c4 only: algorithm1 = the paper's Algorithm 1 schedule (gamma 0.1 / 0.05, tau_G = 4 tau)")
     ap.add_argument("--mlp-unfused-step", action="store_true", help="c3: do not set LSGD_FLAG_MLP_FUSED_STEP")
+    ap.add_argument("--graph", action="store_true", help="c0-c3: also time the steps replayed from a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

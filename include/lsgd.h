@@ -227,6 +227,14 @@ LSGD_API lsgd_status lsgd_center(lsgd_handle h, float* center);
  * the library's internal copies of the parameters (the bf16 weight copy of the MLP objective) on the
  * stream.  The step counter and the leaders are kept.                                               */
 LSGD_API lsgd_status lsgd_sync_parameters(lsgd_handle h);
+/* CUDA-graph support.  grad / elect / step only enqueue kernels, so a sequence of whole steps can be
+ * captured from the stream (after at least one un-captured step has run, so that one-time kernel
+ * attributes are set) and replayed.  The pull / plain decision of every captured step is frozen into the
+ * graph, so capture a whole number of communication periods starting at t % tau == 0 (and t % tau_G == 0
+ * with LSGD_FLAG_ALGORITHM1) and replay from such a t.  The library counts steps on the host when they are
+ * enqueued, not when a graph replays them: after each replay call lsgd_advance_step with the number of
+ * steps the graph contains.                                                                        */
+LSGD_API lsgd_status lsgd_advance_step(lsgd_handle h, int64_t n_steps);
 /* Replaces eta (learning-rate schedules are the caller's, Section 4).                            */
 LSGD_API lsgd_status lsgd_set_eta(lsgd_handle h, float eta);
 

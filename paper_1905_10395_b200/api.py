@@ -85,6 +85,8 @@ def lib() -> C.CDLL:
         L.lsgd_get_train_loss.restype = C.c_int
         L.lsgd_center.argtypes = [H, C.c_void_p]
         L.lsgd_center.restype = C.c_int
+        L.lsgd_advance_step.argtypes = [H, C.c_int64]
+        L.lsgd_advance_step.restype = C.c_int
         L.lsgd_sync_parameters.argtypes = [H]
         L.lsgd_sync_parameters.restype = C.c_int
         L.lsgd_get_step.argtypes = [H, C.POINTER(C.c_int64)]
@@ -236,6 +238,9 @@ class Lsgd:
     def center(self, out):
         """out (device float[ld]) <- average of all workers' parameters (the paper's center variable)."""
         _check(lib().lsgd_center(self.h, _ptr(out)), "lsgd_center")
+
+    def advance_step(self, n: int):
+        _check(lib().lsgd_advance_step(self.h, int(n)), "lsgd_advance_step")
 
     def sync_parameters(self):
         _check(lib().lsgd_sync_parameters(self.h), "lsgd_sync_parameters")

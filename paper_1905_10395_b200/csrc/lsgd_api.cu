@@ -508,6 +508,13 @@ lsgd_status lsgd_sync_parameters(lsgd_handle h) {
   return LSGD_OK;
 }
 
+lsgd_status lsgd_advance_step(lsgd_handle h, int64_t n_steps) {
+  if (!h || n_steps < 0) return LSGD_ERR_INVALID_ARG;
+  h->t += n_steps;
+  h->loss_partials_valid = false;
+  return LSGD_OK;
+}
+
 lsgd_status lsgd_set_eta(lsgd_handle h, float eta) {
   if (!h || !std::isfinite(eta)) return LSGD_ERR_INVALID_ARG;
   h->cfg.eta = eta;

@@ -15,13 +15,14 @@ from .inputs import Workload
 class Population:
     def __init__(self, w: Workload, *, fused_quadratic: bool = False, arithmetic: int = api.ARITH_FP64,
                  device: str = "cuda:0", x: Optional[torch.Tensor] = None, g: Optional[torch.Tensor] = None,
-                 upload_noise: bool = True, flags: int = 0, algorithm1: Optional[dict] = None):
+                 upload_noise: bool = True, flags: int = 0, algorithm1: Optional[dict] = None,
+                 stream: Optional["torch.cuda.Stream"] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.w = w
         self.dev = torch.device(device)
         torch.cuda.set_device(self.dev)
-        self.stream = torch.cuda.current_stream(self.dev)
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.dev)
         dev = self.dev
         self.x = x if x is not None else torch.from_numpy(w.x0).to(dev)
         self.g = g
@@ -94,6 +95,7 @@ class Population:
                                     x=self.x, g=self.g, stream=self.stream.cuda_stream, arithmetic=arithmetic,
                                     flags=flags, **extra)
         self._keep.append(keep)
+        torch.cuda.synchronize(self.dev)          # uploads were made on torch's current stream
         self.lsgd = api.Lsgd(cfg, keep)
         self.t = 0
         self.n_elections = 0
@@ -146,6 +148,43 @@ class Population:
     def run(self, steps: int, record: bool = False) -> None:
         for _ in range(steps):
             self.step(record=record)
+
+    # ---- CUDA graphs: capture n whole steps once, replay them without per-launch host work
+    def capture(self, n_steps: int):
+        """Captures the next ``n_steps`` steps (a whole number of communication periods, starting at a
+        period boundary, and a whole number of passes over the batch ring) into a CUDA graph.  The captured
+        steps are not executed; ``replay`` runs them."""
+        if self.alg1 is not None:
+            raise ValueError("capture() drives the fused schedule only")
+        if self.t % self.w.tau or n_steps % self.w.tau:
+            raise ValueError("capture whole communication periods starting at t % tau == 0")
+        if self.batches and n_steps % len(self.batches):
+            raise ValueError("capture a whole number of passes over the batch ring")
+        if self.loss_ring is not None and (n_steps // self.w.tau) % self.loss_ring.shape[0]:
+            raise ValueError("capture a whole number of passes over the loss ring")
+        if self.stream.cuda_stream == 0:
+            raise ValueError("create the Population with stream=torch.cuda.Stream(): the default stream cannot be captured")
+        t0, e0 = self.t, self.n_elections
+        graph = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize(self.dev)
+        # the library enqueues on the stream it was created with: capture on that very stream
+        with torch.cuda.graph(graph, stream=self.stream):
+            for _ in range(n_steps):
+                self.step()
+        # nothing ran yet; the library has counted the captured steps as enqueued (see replay)
+        self._graph, self._graph_steps = graph, n_steps
+        self.t, self.n_elections = t0, e0
+        self._graph_lib_ahead = n_steps
+        return graph
+
+    def replay(self) -> None:
+        self._graph.replay()
+        if self._graph_lib_ahead:
+            self._graph_lib_ahead = 0       # the capture already advanced the library's counter once
+        else:
+            self.lsgd.advance_step(self._graph_steps)
+        self.t += self._graph_steps
+        self.n_elections += self._graph_steps // self.w.tau
 
     def x_host(self) -> np.ndarray:
         torch.cuda.synchronize(self.dev)

@@ -342,3 +342,34 @@ def test_matcomp_gradient_is_reproducible_bit_for_bit():
     o = _oracle(w)
     o.run(4)
     assert rel_err(runs[0], o.x) <= TOL
+
+
+@pytest.mark.parametrize("kind", ["quadratic", "matcomp"])
+def test_cuda_graph_replay_matches_the_oracle(kind):
+    """Whole communication periods captured into a CUDA graph and replayed (lsgd_advance_step keeps the
+    library's step counter in line) give the same trajectory as issuing the calls one by one."""
+    import torch
+    if kind == "quadratic":
+        w = inputs.config(0, d=3000, tau=2, steps=12, noise_ring=4)
+    else:
+        w = inputs.make_matcomp(4, 2, n_rows=300, n_cols=200, rank=7, n_obs=5000, n_heldout=512, batch=700, steps=4,
+                                tau=2, config_id=58)
+    stream = torch.cuda.Stream()
+    pop = _pop(w, fused_quadratic=(kind == "quadratic"), stream=stream)
+    with torch.cuda.stream(stream):
+        pop.run(4)                                   # un-captured warm-up: one pass over the batch ring
+        pop.capture(4)
+        pop.replay()
+        pop.replay()
+    stream.synchronize()
+    assert pop.lsgd.t() == 12
+    o = _oracle(w)
+    o.run(12)
+    x = pop.x_host()
+    if kind == "quadratic":
+        assert np.array_equal(x.view(np.uint32), o.x.view(np.uint32))
+    else:
+        assert rel_err(x, o.x) <= TOL
+    ll, gl = pop.lsgd.leaders()
+    assert gl == o.gl and np.array_equal(ll, o.ll)
+    pop.close()
