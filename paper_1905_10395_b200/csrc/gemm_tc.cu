@@ -10,7 +10,7 @@
 //   * warp 1 (one thread): issues tcgen05.mma (M = 128, N = 128, K = 16, cta_group::1) into one of TWO
 //     fp32 accumulator tiles in tensor memory (2 x 128 columns), so the products of tile i+1 overlap
 //     the epilogue of tile i.
-//   * warps 2..5: epilogue.  tcgen05.ld of the accumulator (thread = row), fused arithmetic, swizzled
+//   * warps 2..9: epilogue (two warps per tensor-memory lane quarter, each half of the columns).  tcgen05.ld of the accumulator (thread = row), fused arithmetic, swizzled
 //     st.shared into the epilogue buffers, then ONE thread issues TMA stores of the whole tile
 //     (cp.async.bulk.tensor shared -> global): all global traffic of the kernel goes through TMA, edge
 //     tiles are clipped by the tensor maps.
@@ -37,7 +37,8 @@ namespace {
 constexpr int BM = 128, BK = 64;                            // tile rows, k-slice; the tile width BN (128 or 256) is a template parameter
 constexpr int kMaxStages = 6;
 constexpr int kABytes = BM * BK * 2;                        // 16 KiB
-constexpr int kThreads = 192;                               // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kEpiWarps = 8;                                // two warps per tensor-memory lane quarter, half the columns each
+constexpr int kThreads = 64 + 32 * kEpiWarps;               // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
 // Shared memory is carved per epilogue kind (at most 224 KiB + alignment slack):
 //   bf16 outputs, 128-wide tiles : 6 operand stages (32 KiB) + 1 bf16 tile (32 KiB)
 //   bf16 outputs, 256-wide tiles : 3 operand stages (48 KiB) + 1 bf16 tile (64 KiB); used when the product has
@@ -127,7 +128,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory"); }
 
 // Byte offset of the 16-byte unit `u` (0..7) of row `r` inside a [rows][128 B] box written / read by TMA
 // with the 128-byte swizzle: the unit index is XORed with the row index modulo 8.
@@ -178,7 +179,7 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&acc_full[b], 1);
-      mbar_init(&acc_empty[b], 4);      // one arrival per epilogue warp
+      mbar_init(&acc_empty[b], kEpiWarps);   // one arrival per epilogue warp
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&in_full[b], 1);
@@ -278,8 +279,9 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (ok) mma_commit(&acc_full[b]);  // accumulator complete
     }
   } else if (warp >= 2) {
-    // ---------------------------------------------------------------- epilogue (128 threads)
+    // ---------------------------------------------------------------- epilogue (8 warps)
     const int q4 = warp & 3;                  // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;         // which half of the tile's columns this warp handles
     const int row = q4 * 32 + lane;           // row of the tile owned by this thread
     const bool leader = (threadIdx.x == 64);  // issues the bulk stores
     int local = 0;
@@ -304,7 +306,7 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t tacc = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * BN);
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
         uint32_t r[32];
         tmem_ld32(tacc + (uint32_t)(c * 32), r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
