@@ -37,7 +37,10 @@ namespace {
 constexpr int BM = 128, BK = 64;                            // tile rows, k-slice; the tile width BN (128 or 256) is a template parameter
 constexpr int kMaxStages = 6;
 constexpr int kABytes = BM * BK * 2;                        // 16 KiB
-constexpr int kEpiWarps = 8;                                // two warps per tensor-memory lane quarter, half the columns each
+#ifndef LSGD_GEMM_EPI_WARPS
+#define LSGD_GEMM_EPI_WARPS 8
+#endif
+constexpr int kEpiWarps = LSGD_GEMM_EPI_WARPS;              // kEpiWarps / 4 warps per tensor-memory lane quarter, sharing the columns
 constexpr int kThreads = 64 + 32 * kEpiWarps;               // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
 // Shared memory is carved per epilogue kind (at most 224 KiB + alignment slack):
 //   bf16 outputs, 128-wide tiles : 6 operand stages (32 KiB) + 1 bf16 tile (32 KiB)
@@ -281,7 +284,8 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   } else if (warp >= 2) {
     // ---------------------------------------------------------------- epilogue (8 warps)
     const int q4 = warp & 3;                  // TMEM lane quarter this warp may read
-    const int half = (warp - 2) >> 2;         // which half of the tile's columns this warp handles
+    const int part = (warp - 2) >> 2;         // which share of the tile's columns this warp handles
+    constexpr int kChunksPerPart = (BN / 32) / (kEpiWarps / 4);
     const int row = q4 * 32 + lane;           // row of the tile owned by this thread
     const bool leader = (threadIdx.x == 64);  // issues the bulk stores
     int local = 0;
@@ -306,7 +310,7 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t tacc = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * BN);
 #pragma unroll 1
-      for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
+      for (int c = part * kChunksPerPart; c < (part + 1) * kChunksPerPart; ++c) {
         uint32_t r[32];
         tmem_ld32(tacc + (uint32_t)(c * 32), r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
