@@ -42,6 +42,38 @@ def read_peaks():
     return 6650.0, "fallback"
 
 
+def read_tensor_peak():
+    """Dense bf16 tensor throughput for a kernel timed inside a long step (the sustained figure)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        if "bf16_tflops_sustained" in p:
+            return float(p["bf16_tflops_sustained"]), "measured (sustained)"
+    return 1400.0, "fallback (sustained)"
+
+
+def mlp_step_bytes_flops(dims, batch):
+    """Algorithmic HBM bytes and tensor-core flops of ONE worker's fused gradient + SGD step.
+
+    Every operand is counted once per kernel that must read or write it: bf16 activations and shadow weights
+    (2 B), the fp32 master weights read and rewritten by the step (4 + 4 B) plus their new bf16 shadow (2 B),
+    the fp32 pool rows gathered into the bf16 batch.  The 10-wide head is counted with its fp32 weights."""
+    d0, d1, d2, d3 = [int(v) for v in dims]
+    B = int(batch)
+    by = B * d0 * (4 + 2)                                    # gather
+    by += d0 * d1 * 2 + B * (d0 + d1) * 2                    # H1 = relu(X W1^T + b1)
+    by += d1 * d2 * 2 + B * (d1 + d2) * 2                    # H2
+    by += d2 * d3 * 4 + B * d2 * 2                           # head forward
+    by += d2 * d3 * (4 + 4 + 2) + 2 * B * d2 * 2             # head backward: dH2 out, H2 in, W3 stepped
+    by += d1 * d2 * 2 + B * (d2 + 2 * d1) * 2 + B * d1 * 2   # dH1 = (dH2 W2) masked by H1
+    by += B * (d1 + d2) * 2 + d1 * d2 * (4 + 4 + 2)          # dW2 with the step in its epilogue
+    by += B * (d1 + d2) * 2                                  # bias gradients (column sums)
+    by += B * (d0 + d1) * 2 + d0 * d1 * (4 + 4 + 2)          # dW1 with the step in its epilogue
+    fl = 2.0 * B * (2 * d0 * d1 + 3 * d1 * d2 + 2 * d2 * d3)
+    return float(by), fl
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -311,10 +343,10 @@ def run_ours(args):
     for s in range(steps):
         t = pop.t
         batch = pop.batches[t % len(pop.batches)] if pop.batches else None
-        if spec["kind"] == "psd":
+        if spec["kind"] in ("psd", "mlp"):
             g_ev[s][0].record()
         pop.lsgd.grad(batch)
-        if spec["kind"] == "psd":
+        if spec["kind"] in ("psd", "mlp"):
             g_ev[s][1].record()
         if alg1_mode:
             # Algorithm 1: step with small pulls towards the leader copies, then the communication when due
@@ -375,6 +407,18 @@ def run_ours(args):
                     "peak": fp64_peak, "peak_source": "148 SMs x 64 fp64 FMA/clk x 1.965 GHz", "unit": "TFLOP/s",
                     "frac": flops / (g_ms * 1e-3) / 1e12 / fp64_peak, "traffic": None, "ms_per_launch": g_ms,
                     "flops_per_launch": flops}
+    if spec["kind"] == "mlp" and not args.mlp_unfused_step and not all(pull_flags):
+        # plain steps: the gradient call holds every GEMM and, in their epilogues, the SGD step itself.  With a
+        # batch of 128 rows per worker each weight is used 2 x 128 times per pass, so the weight streams bound it.
+        g_ms = float(np.mean([a.elapsed_time(b) for (a, b), f in zip(g_ev, pull_flags) if not f]))
+        mb, mflops = mlp_step_bytes_flops(w.meta["dims"], int(w.meta["batch"]))
+        t_peak, t_src = read_tensor_peak()
+        roofline = {"bound": "hbm", "kernel": "bgemm_bf16_kernel inside the fused gradient + step call (plain steps)",
+                    "achieved": P * mb / (g_ms * 1e-3) / 1e9, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+                    "frac": P * mb / (g_ms * 1e-3) / 1e9 / peak, "traffic": None, "ms_per_launch": g_ms,
+                    "algorithmic_bytes_per_launch": P * mb, "tensor_tflops": P * mflops / (g_ms * 1e-3) / 1e12,
+                    "tensor_peak_tflops": t_peak, "tensor_peak_source": t_src,
+                    "tensor_frac": P * mflops / (g_ms * 1e-3) / 1e12 / t_peak}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": elapsed_ms / steps, "steps_per_s": steps * world / (elapsed_ms * 1e-3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

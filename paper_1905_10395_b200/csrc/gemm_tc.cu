@@ -203,6 +203,9 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_s;
   volatile int* abort_flag = &abort_s;
+  // everything above touched only this CTA's own state; the operands may come from the kernel before
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0 && lane == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -311,6 +314,7 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t tacc = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * BN);
 #pragma unroll 1
       for (int c = part * kChunksPerPart; c < (part + 1) * kChunksPerPart; ++c) {
+        if (q.n0 + c * 32 >= p.N) break;                        // ragged last tile: these columns do not exist
         uint32_t r[32];
         tmem_ld32(tacc + (uint32_t)(c * 32), r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -515,13 +519,12 @@ cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, con
   const bool bf16_out = p.epilogue != GEMM_EPI_F32 && p.epilogue != GEMM_EPI_SGD;
   if (bf16_out && p.N >= 256 && tiles256 >= 2 * (int64_t)sms) {
     const unsigned grid = (unsigned)(tiles256 < sms ? tiles256 : sms);
-    bgemm_bf16_kernel<256><<<grid, kThreads, kSmemBytes, s>>>(map_a, map_b, map_c, map_aux, p);
+    return launch_pdl(bgemm_bf16_kernel<256>, dim3(grid), dim3(kThreads), kSmemBytes, s, map_a, map_b, map_c, map_aux, p);
   } else {
     const int64_t tiles = (int64_t)((p.N + 127) / 128) * mtiles * p.batch;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    bgemm_bf16_kernel<128><<<grid, kThreads, kSmemBytes, s>>>(map_a, map_b, map_c, map_aux, p);
+    return launch_pdl(bgemm_bf16_kernel<128>, dim3(grid), dim3(kThreads), kSmemBytes, s, map_a, map_b, map_c, map_aux, p);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace lsgd

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
 #include <vector>
 
 #include "lsgd.h"
@@ -107,6 +108,36 @@ cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials,
 int32_t psd_loss_blocks(int32_t n);
 cudaError_t launch_psd_grad(const float* x, float* g, const float* M, int32_t n, int32_t r, int32_t P, int64_t ld,
                             double* partials, int32_t n_partials, bool write_g, cudaStream_t s);
+
+// Programmatic dependent launch.  A kernel started with launch_pdl() may become resident, and run its
+// prologue (barrier and tensor-memory set-up, descriptor prefetch), while the kernel before it in the stream
+// is still draining.  Such a kernel calls pdl_wait() before its first access to global memory that an earlier
+// kernel may have written or may still read: the wait returns once every earlier kernel has completed and its
+// writes are visible.  pdl_launch_dependents() lets the NEXT kernel in the stream become resident as soon as
+// resources free up; it says nothing about this kernel's data, which the next kernel obtains through its own
+// pdl_wait().  Building with -DLSGD_NO_PDL=1 turns every such launch into a plain one.
+#ifndef LSGD_NO_PDL
+#define LSGD_NO_PDL 0
+#endif
+#if defined(__CUDACC__)
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = LSGD_NO_PDL ? 0 : 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#endif
 
 }  // namespace lsgd
 

@@ -90,6 +90,8 @@ __global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16*
 __global__ void __launch_bounds__(128)
 gather_rows_kernel(const float* __restrict__ pool, const int32_t* __restrict__ idx, __nv_bfloat16* __restrict__ xb,
                    int32_t rows_total, int32_t d0, int32_t pool_rows, uint32_t* status) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int row = blockIdx.x;
   if (row >= rows_total) return;
   int src = idx[row];
@@ -134,6 +136,8 @@ head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* _
                     const int32_t* __restrict__ labels, const int32_t* __restrict__ label_idx, float* __restrict__ dz,
                     float* __restrict__ loss_b, int32_t n, int32_t d2, int32_t C, int64_t ld, int64_t w3_off, int64_t b3_off,
                     int32_t label_rows, int32_t groups_per_warp, uint32_t* status) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ uint4 s_w3[];   // [C][d2 / 8]
   const int i = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -232,6 +236,8 @@ __global__ void __launch_bounds__(kBwdThreadsX * kBwdSlices)
 head_backward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ dz,
                      __nv_bfloat16* __restrict__ dh2, float* __restrict__ g, int32_t n, int32_t d2, int32_t C, int64_t ld,
                      int64_t w3_off, int64_t b3_off, int64_t b2_off) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ __align__(16) float s_mem[];
   float* s_dz = s_mem;                              // [n][kDzPitch], zero beyond C
   float* s_red = s_mem + (size_t)n * kDzPitch;      // [kBwdSlices][C + 1][kBwdCols]
@@ -330,6 +336,8 @@ constexpr int kSumThreadsX = 64, kSumSlices = 8;
 // of columns 2k, 2k + 1 and the slices are combined in slice order.
 __global__ void __launch_bounds__(kSumThreadsX * kSumSlices)
 column_sum_kernel(const __nv_bfloat16* __restrict__ delta, float* __restrict__ g, int32_t n, int32_t dcols, int64_t ld, int64_t off) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ float s_part[kSumSlices][2 * kSumThreadsX];
   const int i = blockIdx.y, tx = threadIdx.x, ty = threadIdx.y;
   const int k = blockIdx.x * 2 * kSumThreadsX + 2 * tx;
@@ -407,6 +415,8 @@ __global__ void window_mean_kernel(const float* __restrict__ ring, float* __rest
 
 // out[i] = mean_b v[i][b], summed in a fixed order by one warp per worker.
 __global__ void __launch_bounds__(32) row_mean_kernel(const float* __restrict__ v, float* __restrict__ out, int32_t n) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int i = blockIdx.x, lane = threadIdx.x;
   double acc = 0.0;
   for (int b = lane; b < n; b += 32) acc += (double)v[(int64_t)i * n + b];
@@ -526,15 +536,17 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   const int64_t ld = st->ld;
   cudaStream_t s = h->stream;
 
-  gather_rows_kernel<<<P * B, 128, 0, s>>>(m.pool_x, batch_idx, st->xb, P * B, d[0], m.pool, h->d_status);
-  if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
+  if (launch_pdl(gather_rows_kernel, dim3(P * B), dim3(128), 0, s, m.pool_x, batch_idx, st->xb, P * B, d[0], m.pool,
+                 h->d_status) != cudaSuccess)
+    return LSGD_ERR_CUDA;
   lsgd_status fs = forward_hidden(h, st->m_xb, 1, B, st->h1, st->m_h1, st->h2);
   if (fs != LSGD_OK) return fs;
 
   const size_t w3_smem = (size_t)d[3] * d[2] * 2;
-  head_forward_kernel<1><<<dim3((B + kHeadWarps - 1) / kHeadWarps, P), kHeadWarps * 32, w3_smem, s>>>(
-      st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], m.pool, 1,
-      h->d_status);
+  if (launch_pdl(head_forward_kernel<1>, dim3((B + kHeadWarps - 1) / kHeadWarps, P), dim3(kHeadWarps * 32), w3_smem, s,
+                 st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2], d[3], ld, st->L.w[2], st->L.b[2],
+                 m.pool, 1, h->d_status) != cudaSuccess)
+    return LSGD_ERR_CUDA;
   const size_t bwd_smem = sizeof(float) * ((size_t)B * kDzPitch + (size_t)kBwdSlices * (d[3] + 1) * kBwdCols);
   static bool bwd_attr = false;
   if (!bwd_attr) {
@@ -543,12 +555,15 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
     bwd_attr = true;
   }
   if (m.loss_window > 0) {   // remember this step's mean minibatch losses for the running-mean election
-    row_mean_kernel<<<P, 32, 0, s>>>(st->loss_b, st->ring + (st->n_grads % m.loss_window) * P, B);
+    if (launch_pdl(row_mean_kernel, dim3(P), dim3(32), 0, s, st->loss_b, st->ring + (st->n_grads % m.loss_window) * P,
+                   B) != cudaSuccess)
+      return LSGD_ERR_CUDA;
     st->n_grads++;
   }
-  head_backward_kernel<<<dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdThreadsX, kBwdSlices), bwd_smem, s>>>(
-      st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]);
-  if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
+  if (launch_pdl(head_backward_kernel, dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdThreadsX, kBwdSlices), bwd_smem,
+                 s, st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]) !=
+      cudaSuccess)
+    return LSGD_ERR_CUDA;
 
   // dH1 = (dH2 . W2) masked by H1 > 0        [B x d1] = [B x d2] . [d2 x d1]
   GemmShape gd = shape(B, d[1], d[2], P, 0, 1, 1, GEMM_EPI_MASK_BF16, st->dh1, d[1], (int64_t)B * d[1], h->d_status);
@@ -563,9 +578,9 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   g2.eta = (double)c.eta;
   g2.arith = c.arithmetic;
   if (launch_bgemm(st->m_dh2, st->m_h1, g2, s) != cudaSuccess) return LSGD_ERR_CUDA;
-  column_sum_kernel<<<dim3((d[1] + 2 * kSumThreadsX - 1) / (2 * kSumThreadsX), P), dim3(kSumThreadsX, kSumSlices), 0, s>>>(
-      st->dh1, c.g, B, d[1], ld, st->L.b[0]);
-  if (cudaGetLastError() != cudaSuccess) return LSGD_ERR_CUDA;
+  if (launch_pdl(column_sum_kernel, dim3((d[1] + 2 * kSumThreadsX - 1) / (2 * kSumThreadsX), P),
+                 dim3(kSumThreadsX, kSumSlices), 0, s, st->dh1, c.g, B, d[1], ld, st->L.b[0]) != cudaSuccess)
+    return LSGD_ERR_CUDA;
   // dW1 = dH1^T . X                           [d1 x d0]
   GemmShape g1 = shape(d[1], d[0], B, P, 1, 1, 1, fuse_sgd ? GEMM_EPI_SGD : GEMM_EPI_F32, c.g + st->L.w[0], d[0], ld, h->d_status);
   g1.x_upd = c.x + st->L.w[0];

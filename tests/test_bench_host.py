@@ -50,3 +50,15 @@ def test_single_process_defaults():
     assert bench.dist_env() == (0, 1, 0) or "RANK" in os.environ
     assert bench.max_over_ranks(3.5, 1) == 3.5
     assert bench.aggregate(100.0, 50.0, 4) == 100.0 * 4 / 0.05
+
+
+def test_mlp_step_bytes_and_flops_count_each_operand_once():
+    """The fused MLP step's algorithmic figures: weights dominate, and the flops are five GEMMs plus the head."""
+    sys.path.insert(0, ROOT)
+    import bench
+    by, fl = bench.mlp_step_bytes_flops((784, 1024, 1024, 10), 128)
+    n_w = 784 * 1024 + 1024 * 1024
+    # every big weight: two bf16 reads (forward, and W2 once more for dH1) plus the 10-byte stepped rewrite
+    assert by > n_w * 12 + 1024 * 1024 * 2
+    assert by < n_w * 12 + 1024 * 1024 * 2 + 6e6           # activations and the head add a few MB at most
+    assert fl == 2.0 * 128 * (2 * 784 * 1024 + 3 * 1024 * 1024 + 2 * 1024 * 10)
