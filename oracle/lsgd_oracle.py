@@ -23,6 +23,8 @@ Readings of the paper taken here (each is also exercised by a pin in tests/test_
     right-hand term carries subscript t), i.e. a simultaneous (Jacobi) update of all workers.
   * argmin ties go to the lowest worker index; the order on losses is
     -inf < finite < +inf < NaN, and -0.0 == +0.0.
+  * Nesterov momentum and weight decay (Section 4.1) act on the gradient step only; the pulls stay outside
+    the momentum buffer (momentum_update).
 
 Pins: see tests/test_oracle_pins.py.  Parity unpinned (self-consistent definitions only, no
 external fact fixes them): the placement of bf16 roundings in the MLP objective's "bf16emu" mode,
@@ -93,6 +95,42 @@ def update(x: np.ndarray, g: np.ndarray, group_of: Sequence[int], ll: Sequence[i
             zl = snap_l[int(ll[int(group_of[i])])]
             new = new - eta * lambda_l * (xi - zl) - eta * lambda_g * (xi - snap_g)
         x[i] = new.astype(F32)
+
+
+def momentum_update(x: np.ndarray, v: np.ndarray, g: np.ndarray, group_of: Sequence[int], ll: Sequence[int],
+                    gl: int, eta: float, lambda_l: float, lambda_g: float, pull: bool, mu: float,
+                    wd: float) -> None:
+    """The optimiser of the deep-network runs (Section 4.1: Nesterov momentum 0.9 and weight decay 1e-4 for
+    every method), in place on x and on the momentum buffer v (both float32 [P, ld]):
+
+        d  = g + wd x            weight decay enters as the gradient of (wd / 2) |x|^2
+        v+ = mu v + d            momentum buffer, v_0 = 0
+        u  = d + mu v+           Nesterov look-ahead direction
+        x+ = x - eta u  [ - eta lambda_l (x - x_ll) - eta lambda_g (x - x_gl)  on a pull step ]
+
+    The paper does not say how the pulls and the momentum buffer combine; the reading here keeps the pulls
+    out of the buffer, so that with mu = wd = 0 the step is Eq. (1) again.  Every stored value is evaluated
+    in float64 in the order written and rounded once; u uses the unrounded v+."""
+    eta = float(F32(eta))
+    lambda_l = float(F32(lambda_l))
+    lambda_g = float(F32(lambda_g))
+    mu = float(F32(mu))
+    wd = float(F32(wd))
+    P = x.shape[0]
+    if pull:
+        snap_l = {int(r): x[int(r)].astype(F64) for r in set(int(q) for q in ll)}
+        snap_g = x[int(gl)].astype(F64)
+    for i in range(P):
+        xi = x[i].astype(F64)
+        d = g[i].astype(F64) + wd * xi
+        vn = mu * v[i].astype(F64) + d
+        u = d + mu * vn
+        new = xi - eta * u
+        if pull:
+            zl = snap_l[int(ll[int(group_of[i])])]
+            new = new - eta * lambda_l * (xi - zl) - eta * lambda_g * (xi - snap_g)
+        x[i] = new.astype(F32)
+        v[i] = vn.astype(F32)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -361,9 +399,13 @@ class LsgdOracle:
     """
 
     def __init__(self, x0: np.ndarray, objective: Objective, group_of: Sequence[int], G: int,
-                 eta: float, lambda_l: float, lambda_g: float, tau: int):
+                 eta: float, lambda_l: float, lambda_g: float, tau: int, momentum: Optional[float] = None,
+                 weight_decay: float = 0.0):
         assert tau >= 1
         self.x = np.array(x0, dtype=F32, copy=True)
+        # momentum is None: the step of Eq. (1); a number (0 included): the Section 4.1 optimiser
+        self.mu, self.wd = momentum, weight_decay
+        self.v = None if momentum is None else np.zeros_like(self.x)
         self.obj = objective
         self.group_of = np.asarray(group_of, dtype=np.int32)
         self.G = int(G)
@@ -385,8 +427,12 @@ class LsgdOracle:
             self.history.append({"t": self.t, "loss": self.loss.copy(), "ll": self.ll.copy(),
                                  "gl": self.gl})
             self.n_elections += 1
-        update(self.x, g, self.group_of, self.ll if pull else (), self.gl if pull else -1,
-               self.eta, self.lambda_l, self.lambda_g, pull)
+        if self.v is None:
+            update(self.x, g, self.group_of, self.ll if pull else (), self.gl if pull else -1,
+                   self.eta, self.lambda_l, self.lambda_g, pull)
+        else:
+            momentum_update(self.x, self.v, g, self.group_of, self.ll if pull else (), self.gl if pull else -1,
+                            self.eta, self.lambda_l, self.lambda_g, pull, self.mu, self.wd)
         self.t += 1
 
     def run(self, steps: int) -> np.ndarray:

@@ -141,3 +141,57 @@ def test_gradient_mistakes_are_caught(monkeypatch):
     monkeypatch.setattr(orc, "bf16_round", lambda a: (np.asarray(a, F32).view(np.uint32) & 0xFFFF0000).view(F32))  # truncation
     assert _fails(pins.test_mlp_bf16emu_is_close_to_fp32_and_rounding_matches_library)
     monkeypatch.setattr(orc, "bf16_round", good_round)
+
+
+# ---- the Section 4.1 optimiser ------------------------------------------------------------------------
+from tests import test_oracle_momentum as mpins  # noqa: E402
+
+
+def _momentum_variant(kind):
+    def momentum_update(x, v, g, group_of, ll, gl, eta, lambda_l, lambda_g, pull, mu, wd):
+        eta, lambda_l, lambda_g, mu, wd = (float(F32(q)) for q in (eta, lambda_l, lambda_g, mu, wd))
+        snap = x.astype(F64)
+        for i in range(x.shape[0]):
+            xi = snap[i]
+            d = g[i].astype(F64) + (-wd if kind == "decay_sign" else wd) * xi
+            pulls = 0.0
+            if pull:
+                pulls = lambda_l * (xi - snap[int(ll[int(group_of[i])])]) + lambda_g * (xi - snap[int(gl)])
+            if kind == "pull_in_buffer":                       # the pulls treated as part of the gradient
+                d = d + pulls
+                pulls = 0.0
+            vn = mu * v[i].astype(F64) + d
+            if kind == "classical":                            # heavy ball: step along the buffer itself
+                u = vn
+            elif kind == "lookahead_on_old_buffer":
+                u = d + mu * v[i].astype(F64)
+            else:
+                u = d + mu * vn
+            x[i] = (xi - eta * u - eta * pulls).astype(F32)
+            v[i] = vn.astype(F32)
+    return momentum_update
+
+
+MOMENTUM_CASES = {
+    "classical": [mpins.test_without_pulls_it_is_the_library_nesterov_sgd,
+                  mpins.test_closed_form_on_the_quadratic_is_a_two_by_two_recurrence],
+    "lookahead_on_old_buffer": [mpins.test_closed_form_on_the_quadratic_is_a_two_by_two_recurrence],
+    "decay_sign": [mpins.test_weight_decay_moves_the_fixed_point, mpins.test_without_pulls_it_is_the_library_nesterov_sgd],
+    "pull_in_buffer": [mpins.test_pulls_stay_outside_the_momentum_buffer],
+}
+
+
+@pytest.mark.filterwarnings("ignore::RuntimeWarning")      # a planted sign error may diverge
+@pytest.mark.parametrize("kind", sorted(MOMENTUM_CASES))
+def test_momentum_mistakes_are_caught(kind, monkeypatch):
+    monkeypatch.setattr(orc, "momentum_update", _momentum_variant(kind))
+    for fn in MOMENTUM_CASES[kind]:
+        assert _fails(fn), (kind, fn.__name__)
+
+
+def test_correct_momentum_variant_passes(monkeypatch):
+    monkeypatch.setattr(orc, "momentum_update", _momentum_variant("none"))
+    for fns in MOMENTUM_CASES.values():
+        for fn in fns:
+            fn()
+    mpins.test_zero_momentum_and_decay_is_eq1()
