@@ -163,7 +163,8 @@ def workload_spec(args):
     if wl == "c4":
         return dict(kind="external", cfg=4, P=16, G=4, d=args.d or (1 << 26), eta=0.01, lambda_l=0.1, lambda_g=0.05,
                     tau=args.tau or 1, name="C4 fused-update stress: P=16 G=4 d=2^26 fp32, supplied g and losses",
-                    launches=(2, 1))
+                    launches=(2, 1), momentum=getattr(args, "momentum", None),
+                    weight_decay=getattr(args, "weight_decay", 0.0))
     if wl == "c1":
         return dict(kind="quadratic", cfg=1, P=64, G=8, d=1 << 20, eta=0.05, lambda_l=0.1, lambda_g=0.05,
                     tau=args.tau or 4, name="C1 multi-leader quadratic: P=64 G=8 d=2^20 fp32, noise sigma=0.01, "
@@ -239,7 +240,9 @@ def oracle_sample_run(spec, steps, warmup, sample_cols):
         segs, _ = inputs.mlp_layout(w.meta["dims"])
         obj = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="bf16emu")
         what = f"{P} of {spec['P']} workers (one group)"
-    o = orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
+    mom = spec.get("momentum") if spec["kind"] == "external" else None
+    o = orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau, momentum=mom,
+                       weight_decay=spec.get("weight_decay", 0.0))
     for _ in range(warmup):
         o.step()
     t0 = time.perf_counter()
@@ -307,7 +310,8 @@ def run_ours(args):
         x = hx.to(dev, non_blocking=True)
         g = hg.to(dev, non_blocking=True)
         alg1 = dict(gamma_l=0.1, gamma_g=0.05, tau_g=4 * spec["tau"]) if args.schedule == "algorithm1" else None
-        pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith, algorithm1=alg1)
+        pop = Population(w, device=str(dev), x=x, g=g, arithmetic=args.arith, algorithm1=alg1,
+                         momentum=args.momentum, weight_decay=args.weight_decay)
     elif spec["kind"] == "psd":
         w = inputs.make_psd(P=P, n=spec["n"], r=spec["r"], steps=steps)
         pop = Population(w, device=str(dev), arithmetic=args.arith, stream=gstream)
@@ -380,19 +384,23 @@ def run_ours(args):
     k_ms = [a.elapsed_time(b) for a, b in k_ev]
     upd_ms = float(np.mean(k_ms))
     alg_bytes = bytes_per_worker_param(spec) * P * d
+    with_momentum = spec["kind"] == "external" and args.momentum is not None
+    if with_momentum:
+        alg_bytes += 8.0 * P * d                # the momentum buffer is read and rewritten
     if alg1_mode:
         alg_bytes += 4.0 * (G + 1) * d          # the G + 1 leader copies are read once per step
     peak, peak_src = read_peaks()
     achieved = alg_bytes / (upd_ms * 1e-3) / 1e9
     traffic = None
-    if spec["kind"] == "external" and args.arith == 0 and not alg1_mode:
+    if spec["kind"] == "external" and args.arith == 0 and not alg1_mode and not with_momentum:
         n_pull = sum(pull_flags)
         traffic = P * d * (n_pull * MEASURED_TRAFFIC_PER_WORKER_PARAM["pull"] +
                            (steps - n_pull) * MEASURED_TRAFFIC_PER_WORKER_PARAM["plain"]) / steps
     if pop.lsgd.check_device() != 0:
         raise SystemExit("device status word set during the bench")
 
-    roofline = {"bound": "hbm", "kernel": "pull_update_staged_kernel / plain_update_kernel", "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": "momentum_update_kernel" if with_momentum else
+                "pull_update_staged_kernel / plain_update_kernel", "achieved": achieved,
                 "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
                 "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags)),
@@ -428,6 +436,7 @@ def run_ours(args):
                    "l2": ("per-step inputs exceed the 126 MB L2; no flush between steps" if P * d * 8 > 3e8 else
                           "working set fits in L2; steps run back to back as in training (no flush)"),
                    "multi_gpu": "replicas only", "schedule": args.schedule,
+                   **({"momentum": args.momentum, "weight_decay": args.weight_decay} if with_momentum else {}),
                    **({"mlp_fused_step": not args.mlp_unfused_step} if spec["kind"] == "mlp" else {})},
         "clocks": clocks,
         "roofline": roofline,
@@ -516,6 +525,9 @@ def main():
                     help="c4 only: algorithm1 = the paper's Algorithm 1 schedule (gamma 0.1 / 0.05, tau_G = 4 tau)")
     ap.add_argument("--mlp-unfused-step", action="store_true", help="c3: do not set LSGD_FLAG_MLP_FUSED_STEP")
     ap.add_argument("--graph", action="store_true", help="c0-c3: also time the steps replayed from a CUDA graph")
+    ap.add_argument("--momentum", type=float, default=None,
+                    help="c4: Nesterov momentum of the Section 4.1 optimiser (adds the buffer v: 20 B per worker-param)")
+    ap.add_argument("--weight-decay", type=float, default=0.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -149,6 +149,19 @@ typedef struct {
   int32_t tau_g;             /* global communication period tau_G >= 1                               */
   float* leader_copies;      /* DEVICE float[(G+1)*ld], 16-byte aligned: the leaders' parameters as of
                                 their last election (rows 0..G-1 local, row G global); library-written */
+  /* --- the optimiser of the paper's deep-network runs (Section 4.1); only read when v != NULL --- */
+  float* v;                  /* DEVICE float[P*ld] momentum buffers, 16-byte aligned, caller-owned and
+                                caller-initialised (zeros for a fresh run), updated in place by lsgd_step.
+                                NULL: the step of Eq. (1), momentum and weight_decay are ignored.
+                                Non-NULL: with d = g + weight_decay x,  v <- momentum v + d,
+                                x <- x - eta (d + momentum v) - [the two pulls of Eq. (1) on a pull step]:
+                                Nesterov momentum with the decay inside the gradient; the pulls stay
+                                outside the buffer (the paper does not say how they combine), so that
+                                momentum = weight_decay = 0 gives Eq. (1) again.  Needs cfg.g; not
+                                combined with LSGD_FLAG_MLP_FUSED_STEP or LSGD_FLAG_ALGORITHM1
+                                (LSGD_ERR_UNSUPPORTED).                                              */
+  float momentum;            /* Nesterov momentum mu, finite (the paper uses 0.9)                    */
+  float weight_decay;        /* L2 decay coefficient, finite (the paper uses 1e-4)                   */
 } lsgd_config;
 
 /* MLP objective: on steps that are not pull steps, let lsgd_grad apply x <- x - eta g for W1 and W2

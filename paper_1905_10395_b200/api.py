@@ -59,7 +59,8 @@ class Config(C.Structure):
                 ("lambda_g", C.c_float), ("tau", C.c_int32), ("objective", C.c_int32),
                 ("objective_desc", C.c_void_p), ("x", C.c_void_p), ("g", C.c_void_p), ("stream", C.c_void_p),
                 ("arithmetic", C.c_int32), ("flags", C.c_uint32), ("gamma_l", C.c_float), ("gamma_g", C.c_float),
-                ("tau_g", C.c_int32), ("leader_copies", C.c_void_p)]
+                ("tau_g", C.c_int32), ("leader_copies", C.c_void_p), ("v", C.c_void_p), ("momentum", C.c_float),
+                ("weight_decay", C.c_float)]
 
 
 _lib = None
@@ -180,7 +181,7 @@ def mlp_scratch_bytes(dims: Sequence[int], P: int, batch: int, n_heldout: int) -
 def make_config(*, P: int, G: int, group_of: np.ndarray, d: int, ld: int, eta: float, lambda_l: float,
                 lambda_g: float, tau: int, objective: int, desc=None, x=None, g=None, stream: int = 0,
                 arithmetic: int = ARITH_FP64, flags: int = 0, gamma_l: float = 0.0, gamma_g: float = 0.0,
-                tau_g: int = 1, leader_copies=None):
+                tau_g: int = 1, leader_copies=None, v=None, momentum: float = 0.0, weight_decay: float = 0.0):
     """Returns (Config, keepalive) -- keepalive holds the host arrays the struct points to."""
     go = np.ascontiguousarray(group_of, dtype=np.int32)
     cfg = Config()
@@ -199,6 +200,8 @@ def make_config(*, P: int, G: int, group_of: np.ndarray, d: int, ld: int, eta: f
     cfg.flags = int(flags)
     cfg.gamma_l, cfg.gamma_g, cfg.tau_g = float(gamma_l), float(gamma_g), int(tau_g)
     cfg.leader_copies = _ptr(leader_copies)
+    cfg.v = _ptr(v)
+    cfg.momentum, cfg.weight_decay = float(momentum), float(weight_decay)
     return cfg, (go, desc)
 
 

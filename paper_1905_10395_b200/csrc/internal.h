@@ -36,6 +36,8 @@ struct QuadInline {
 struct Coef {
   double eta, cl, cg, sigma;
   float eta_f, cl_f, cg_f, sigma_f;
+  double mu, wd;            // Nesterov momentum and weight decay (momentum kernel only)
+  float mu_f, wd_f;
 };
 
 struct UpdateArgs {
@@ -55,8 +57,11 @@ struct UpdateArgs {
   int arith;                // 0 fp64 unfused, 1 fp64 fma, 2 fp32 fma (see update.cu)
   uint32_t* status;
   bool pull;
+  float* v;                 // momentum buffers [P][ld], or nullptr = the step of Eq. (1)
 };
 cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s);
+// Section 4.1 optimiser (a.v != nullptr): Nesterov momentum + weight decay around the same step.
+cudaError_t launch_momentum_update(const UpdateArgs& a, cudaStream_t s);
 cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, int64_t ld, cudaStream_t s);
 
 struct ElectArgs {

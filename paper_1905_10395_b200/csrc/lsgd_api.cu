@@ -44,6 +44,12 @@ lsgd_status validate(const lsgd_config* c) {
     if (!c->leader_copies) return LSGD_ERR_INVALID_ARG;
     if (!aligned16(c->leader_copies)) return LSGD_ERR_ALIGNMENT;
   }
+  if (c->v) {
+    if (!std::isfinite(c->momentum) || !std::isfinite(c->weight_decay)) return LSGD_ERR_INVALID_ARG;
+    if (!c->g) return LSGD_ERR_INVALID_ARG;
+    if (!aligned16(c->v)) return LSGD_ERR_ALIGNMENT;
+    if (c->flags & (LSGD_FLAG_MLP_FUSED_STEP | LSGD_FLAG_ALGORITHM1)) return LSGD_ERR_UNSUPPORTED;
+  }
   if (c->P > kMaxWorkers) return LSGD_ERR_UNSUPPORTED;
   if (c->ld % 32 != 0) return LSGD_ERR_ALIGNMENT;
   if (!c->x) return LSGD_ERR_INVALID_ARG;
@@ -353,9 +359,14 @@ UpdateArgs base_update_args(lsgd_ctx* h) {
   a.k.cl_f = (float)a.k.cl;
   a.k.cg_f = (float)a.k.cg;
   a.k.sigma_f = h->quad.sigma;
+  a.k.mu = (double)c.momentum;
+  a.k.wd = (double)c.weight_decay;
+  a.k.mu_f = c.momentum;
+  a.k.wd_f = c.weight_decay;
   a.arith = c.arithmetic;
   a.status = h->d_status;
   a.pull = false;
+  a.v = c.v;
   return a;
 }
 
@@ -419,6 +430,8 @@ extern "C" lsgd_status lsgd_step(lsgd_handle h) {
       b.d = ranges[r][1];
       LSGD_CUDA(launch_update(b, h->stream));
     }
+  } else if (a.v) {
+    LSGD_CUDA(launch_momentum_update(a, h->stream));
   } else {
     LSGD_CUDA(launch_update(a, h->stream));
   }

@@ -16,7 +16,8 @@ class Population:
     def __init__(self, w: Workload, *, fused_quadratic: bool = False, arithmetic: int = api.ARITH_FP64,
                  device: str = "cuda:0", x: Optional[torch.Tensor] = None, g: Optional[torch.Tensor] = None,
                  upload_noise: bool = True, flags: int = 0, algorithm1: Optional[dict] = None,
-                 stream: Optional["torch.cuda.Stream"] = None):
+                 stream: Optional["torch.cuda.Stream"] = None, momentum: Optional[float] = None,
+                 weight_decay: float = 0.0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.w = w
@@ -90,6 +91,11 @@ class Population:
             flags |= api.FLAG_ALGORITHM1
             extra = dict(gamma_l=algorithm1["gamma_l"], gamma_g=algorithm1["gamma_g"], tau_g=algorithm1["tau_g"],
                          leader_copies=self.leader_copies)
+        self.v = None
+        if momentum is not None:
+            # Section 4.1 optimiser: Nesterov momentum + weight decay; the buffers start at zero
+            self.v = torch.zeros_like(self.x)
+            extra.update(v=self.v, momentum=momentum, weight_decay=weight_decay)
         cfg, keep = api.make_config(P=w.P, G=w.G, group_of=w.group_of, d=w.d, ld=w.ld, eta=w.eta,
                                     lambda_l=w.lambda_l, lambda_g=w.lambda_g, tau=w.tau, objective=obj, desc=desc,
                                     x=self.x, g=self.g, stream=self.stream.cuda_stream, arithmetic=arithmetic,
