@@ -455,6 +455,270 @@ inline int staged_tile_width(const UpdateArgs& a) {
   return 0;
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Chunked staged form: the same bulk-copy pipeline for any population size, and for the inline quadratic
+// gradient.
+//
+// A tile's rows no longer have to fit in shared memory together.  What every row of the tile needs -- the
+// leaders' pieces (one slot per group's local leader, one for the global leader when it is not among them, or
+// the G + 1 leader copies) and, for the quadratic, the pieces of a and b -- goes into a double-buffered
+// "leader block" first; the workers' rows (x and g / noise) then stream through a ring of chunks of R workers.
+// The consumers start on a tile only after its leader block has landed, so every leader value is x at time t
+// although the leader's own row is rewritten while the tile is processed.  A worker that is its group's
+// leader takes its x from the leader block and its row is not fetched again: every byte of x and g is still
+// read once.
+#ifndef LSGD_K1_CHUNK_SHAPES
+#define LSGD_K1_CHUNK_SHAPES {768, 8, 3}, {768, 8, 2}, {768, 4, 3}, {768, 4, 2}, {512, 12, 2}, {512, 6, 3}, {512, 6, 2}
+#endif
+constexpr int kChunkMaxStages = 4;
+constexpr int kChunkSmemBudget = 224 * 1024;
+
+struct ChunkShape {
+  int W, R, S;      // tile width (floats), workers per chunk, ring stages; W == 0: the shape does not fit
+  size_t smem;
+};
+
+template <int MODE, bool PULL, bool QUAD, bool NOISE, bool SHADOW>
+__global__ void __launch_bounds__(kTmaThreads, 1)
+update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
+  extern __shared__ __align__(128) uint8_t s_raw[];
+  __shared__ uint64_t full_bar[kChunkMaxStages], empty_bar[kChunkMaxStages], lfull_bar[2], lempty_bar[2];
+  __shared__ int s_abort, s_bad, s_gslot;
+  const int P = p.P, G = p.G;
+  const bool snap = PULL && p.snap != nullptr;
+  const bool has_g = (QUAD ? NOISE : true) && p.use_g;      // a pure pull drops the gradient term
+  const int pull_slots = PULL ? G + 1 : 0;                  // slots 0..G-1: local leaders, slot G: global leader
+  const int nlead = pull_slots + (QUAD ? 2 : 0);            // then a, b
+  const int stage_rows = R * (has_g ? 2 : 1);
+  float* lead0 = reinterpret_cast<float*>(s_raw);                                   // [2][nlead][W]
+  float* ring0 = lead0 + (size_t)2 * nlead * W;                                     // [S][stage_rows][W]
+  int32_t* s_lead = reinterpret_cast<int32_t*>(ring0 + (size_t)S * stage_rows * W); // [P] slot of worker i's local leader
+  int32_t* s_self = s_lead + P;                                                     // [P] worker i is that leader: x comes from the slot
+  int32_t* s_slot_row = s_self + P;                                                 // [G+1] row of x behind a slot
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    s_bad = 0;
+    for (int s = 0; s < S; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&full_bar[s])), "r"(1) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&empty_bar[s])), "r"(kTmaConsumers / 32) : "memory");
+    }
+    for (int b = 0; b < 2; ++b) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&lfull_bar[b])), "r"(1) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&lempty_bar[b])), "r"(kTmaConsumers / 32) : "memory");
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_gslot = G;
+    if (PULL && !snap) {
+      const int gl = *p.gl;
+      if (gl < 0 || gl >= P) {
+        s_bad = 1;
+      } else {
+        const int grp = p.tab.group_of[gl];
+        s_slot_row[G] = gl;
+        if (p.ll[grp] == gl) s_gslot = grp;     // the global leader is its group's leader: one slot serves both
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < P; i += blockDim.x) {
+    int slot = 0, self = 0;
+    if (PULL) {
+      slot = p.tab.group_of[i];
+      if (!snap) {
+        const int l = p.ll[slot];
+        if (l < 0 || l >= P) s_bad = 1;
+        self = (l == i);
+      }
+    }
+    s_lead[i] = slot;
+    s_self[i] = self;
+  }
+  if (PULL && !snap)
+    for (int j = threadIdx.x; j < G; j += blockDim.x) s_slot_row[j] = p.ll[j];
+  __syncthreads();
+  if (s_bad) {   // never dereference a leader index that is out of range
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(p.status, FLAG_BAD_LEADER);
+    return;
+  }
+  volatile int* abort_flag = &s_abort;
+  const int gslot = s_gslot;
+  const int64_t total_floats = n_cols4 * 4;
+  const int64_t n_tiles = (total_floats + W - 1) / W;
+  const int n_chunks = (P + R - 1) / R;
+  const float* gsrc = QUAD ? p.quad.noise : p.g;
+  if (warp == kTmaConsumers / 32) {
+    // ------------------------------------------------------------------ producer warp
+    uint32_t tit = 0, cit = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tit) {
+      const int b = tit & 1;
+      ok = bar_wait(&lempty_bar[b], ((tit >> 1) & 1) ^ 1, abort_flag, p.status);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      const int64_t c0 = t * W;
+      const int wt = (int)((total_floats - c0) < W ? (total_floats - c0) : W);   // floats in this tile (multiple of 4)
+      const uint32_t bytes = (uint32_t)wt * 4u;
+      float* lead = lead0 + (size_t)b * nlead * W;
+      // the leader block: leaders' pieces (slot G only when it is a row of its own), then a and b
+      const int n_fetch = nlead - ((PULL && gslot != G) ? 1 : 0);
+      if (lane == 0)
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&lfull_bar[b])), "r"(bytes * (uint32_t)n_fetch) : "memory");
+      __syncwarp();
+      for (int r = lane; r < nlead; r += 32) {
+        const float* src;
+        if (r < pull_slots) {
+          if (r == G && gslot != G) continue;
+          src = snap ? p.snap + (int64_t)r * p.ld : p.x + (int64_t)s_slot_row[r] * p.ld;
+        } else {
+          src = (r == pull_slots) ? p.quad.a : p.quad.b;
+        }
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_addr(lead + (size_t)r * W)), "l"(src + c0), "r"(bytes), "r"(smem_addr(&lfull_bar[b])) : "memory");
+      }
+      for (int c = 0; c < n_chunks && ok; ++c, ++cit) {
+        const int s = cit % S;
+        ok = bar_wait(&empty_bar[s], ((cit / S) & 1) ^ 1, abort_flag, p.status);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        const int i0 = c * R;
+        const int nr = (P - i0) < R ? (P - i0) : R;
+        float* sx = ring0 + (size_t)s * stage_rows * W;
+        // rows q < nr: worker (i0 + q)'s x unless it sits in the leader block; rows R + q: its g / noise
+        int mine = 0;
+        for (int q = lane; q < nr; q += 32) mine += (s_self[i0 + q] ? 0 : 1) + (has_g ? 1 : 0);
+        const int n_copies = __reduce_add_sync(0xFFFFFFFFu, mine);
+        if (lane == 0)
+          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&full_bar[s])), "r"(bytes * (uint32_t)n_copies) : "memory");
+        __syncwarp();
+        for (int q = lane; q < nr; q += 32) {
+          const int i = i0 + q;
+          if (!s_self[i])
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(sx + (size_t)q * W)), "l"(p.x + (int64_t)i * p.ld + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
+          if (has_g)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(sx + (size_t)(R + q) * W)), "l"(gsrc + (int64_t)i * p.ld + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
+        }
+      }
+    }
+    if (*abort_flag && lane == 0) {
+      // a wait ran out somewhere: let the copies already issued land before the CTA exits
+      const uint32_t cfirst = cit > (uint32_t)S ? cit - S : 0;
+      for (uint32_t j = cfirst; j < cit; ++j) {
+        const long long t0 = clock64();
+        while (!bar_try(&full_bar[j % S], (j / S) & 1) && clock64() - t0 < kTmaWaitCycles) {}
+      }
+      const uint32_t tfirst = tit > 1 ? tit - 1 : 0;
+      for (uint32_t j = tfirst; j <= tit; ++j) {
+        const long long t0 = clock64();
+        while (!bar_try(&lfull_bar[j & 1], (j >> 1) & 1) && clock64() - t0 < kTmaWaitCycles) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers
+    const Coef k = p.k;
+    const int w4 = W >> 2;                          // 16-byte columns per tile row
+    const int c4 = threadIdx.x % w4;                // this thread's column
+    const int r0 = threadIdx.x / w4, rstep = kTmaConsumers / w4;
+    uint32_t tit = 0, cit = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tit) {
+      const int b = tit & 1;
+      ok = bar_wait(&lfull_bar[b], (tit >> 1) & 1, abort_flag, p.status);
+      if (!ok) break;
+      const int64_t c0 = t * W;
+      const int wt4 = (int)(((total_floats - c0) < W ? (total_floats - c0) : W) >> 2);
+      const bool live = c4 < wt4;
+      const float* lead = lead0 + (size_t)b * nlead * W + c4 * 4;
+      float4 xg = make_float4(0.f, 0.f, 0.f, 0.f), av = xg, bv = xg;
+      if (live) {
+        if (PULL) xg = *reinterpret_cast<const float4*>(lead + (size_t)gslot * W);
+        if (QUAD) {
+          av = *reinterpret_cast<const float4*>(lead + (size_t)pull_slots * W);
+          bv = *reinterpret_cast<const float4*>(lead + (size_t)(pull_slots + 1) * W);
+        }
+      }
+      for (int c = 0; c < n_chunks; ++c, ++cit) {
+        const int s = cit % S;
+        ok = bar_wait(&full_bar[s], (cit / S) & 1, abort_flag, p.status);
+        if (!ok) break;
+        const int i0 = c * R;
+        const int nr = (P - i0) < R ? (P - i0) : R;
+        const float* sx = ring0 + (size_t)s * stage_rows * W + c4 * 4;
+        const float* sg = sx + (size_t)R * W;
+        if (live) {
+          for (int q = r0; q < nr; q += rstep) {
+            const int i = i0 + q;
+            float4 xl = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (PULL) xl = *reinterpret_cast<const float4*>(lead + (size_t)s_lead[i] * W);
+            const float4 x = (PULL && s_self[i]) ? xl : *reinterpret_cast<const float4*>(sx + (size_t)q * W);
+            float4 g = has_g ? *reinterpret_cast<const float4*>(sg + (size_t)q * W) : make_float4(0.f, 0.f, 0.f, 0.f);
+            if (QUAD && p.use_g) {
+              g.x = quad_g<MODE>(x.x, av.x, bv.x, g.x, k, NOISE);
+              g.y = quad_g<MODE>(x.y, av.y, bv.y, g.y, k, NOISE);
+              g.z = quad_g<MODE>(x.z, av.z, bv.z, g.z, k, NOISE);
+              g.w = quad_g<MODE>(x.w, av.w, bv.w, g.w, k, NOISE);
+            }
+            float4 r;
+            if (PULL) {
+              r.x = pull1<MODE>(x.x, g.x, xl.x, xg.x, k);
+              r.y = pull1<MODE>(x.y, g.y, xl.y, xg.y, k);
+              r.z = pull1<MODE>(x.z, g.z, xl.z, xg.z, k);
+              r.w = pull1<MODE>(x.w, g.w, xl.w, xg.w, k);
+            } else {
+              r.x = plain1<MODE>(x.x, g.x, k);
+              r.y = plain1<MODE>(x.y, g.y, k);
+              r.z = plain1<MODE>(x.z, g.z, k);
+              r.w = plain1<MODE>(x.w, g.w, k);
+            }
+            const int64_t off = (int64_t)i * p.ld + c0 + c4 * 4;
+            st4(p.x + off, r);
+            if (SHADOW) st4_bf16(p.x_bf16 + off, r);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&empty_bar[s])) : "memory");
+      }
+      if (!ok) break;
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&lempty_bar[b])) : "memory");
+    }
+  }
+}
+
+// Shape for the chunked kernel: the widest tile and deepest ring whose leader block (twice) and ring fit.
+inline ChunkShape chunk_shape(const UpdateArgs& a, bool quad, bool noise) {
+  ChunkShape none{0, 0, 0, 0};
+  if (!a.pull && !quad) return none;
+  const bool has_g = (quad ? noise : true) && a.use_g;
+  if (!quad && a.use_g && a.g == nullptr) return none;
+  const int nlead = (a.pull ? a.G + 1 : 0) + (quad ? 2 : 0);
+  static const int shapes[][3] = {LSGD_K1_CHUNK_SHAPES};
+  for (const auto& sh : shapes) {
+    const int W = sh[0], R = sh[1], S = sh[2];
+    if (S > kChunkMaxStages || (kTmaConsumers % (W / 4)) != 0) continue;
+    const size_t bytes = ((size_t)2 * nlead + (size_t)S * R * (has_g ? 2 : 1)) * W * 4 + (size_t)(2 * a.P + a.G + 1) * 4;
+    if (bytes <= (size_t)kChunkSmemBudget) return ChunkShape{W, R, S, bytes};
+  }
+  return none;
+}
+
+template <int MODE, bool PULL, bool QUAD, bool NOISE, bool SHADOW>
+cudaError_t launch_chunked(const UpdateArgs& a, const ChunkShape& cs, int64_t n4, int sms, cudaStream_t s) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kChunkSmemBudget);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const int64_t tiles = (n4 * 4 + cs.W - 1) / cs.W;
+  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+  update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW><<<grid, kTmaThreads, cs.smem, s>>>(a, n4, cs.W, cs.R, cs.S);
+  return cudaGetLastError();
+}
+
 template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
 cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
   static int sms = 0;
@@ -479,6 +743,10 @@ cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
     const int64_t tiles = (n4 * 4 + W - 1) / (W > 0 ? W : 1);
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     pull_update_staged_kernel<MODE, SHADOW><<<grid, kTmaThreads, smem, s>>>(a, n4, W);
+  } else if (!LSGD_K1_NO_STAGED && (a.pull || (QUAD && !SHADOW)) && chunk_shape(a, QUAD, NOISE).W > 0) {
+    const ChunkShape cs = chunk_shape(a, QUAD, NOISE);
+    if (a.pull) return launch_chunked<MODE, true, QUAD, NOISE, SHADOW>(a, cs, n4, sms, s);
+    if constexpr (QUAD && !SHADOW) return launch_chunked<MODE, false, QUAD, NOISE, false>(a, cs, n4, sms, s);
   } else if (a.pull) {
     int64_t blocks = (n4 + kThreads - 1) / kThreads;
     if (blocks > cap) blocks = cap;

@@ -30,6 +30,15 @@ def test_tiny_and_boundary_populations(P, G, d):
     _check(w, 5)
 
 
+@pytest.mark.parametrize("P,G,d", [(33, 1, 777), (64, 8, 3001), (40, 40, 1100), (100, 7, 2500), (60, 30, 600),
+                                   (28, 2, 148 * 768 * 2 + 4)])
+def test_populations_streamed_in_chunks(P, G, d):
+    # populations too large to stage whole: the rows of a column tile pass through shared memory in chunks
+    # (ragged last chunk, ragged last tile, leader blocks of 2 .. 41 slots, several tiles per CTA)
+    w = inputs.make_external(P, G, d, eta=0.05, lambda_l=0.3, lambda_g=0.2, tau=2, steps=5, loss_ring=3, config_id=115)
+    _check(w, 5)
+
+
 def test_single_worker_is_plain_sgd():
     w = inputs.make_external(1, 1, 257, eta=0.05, lambda_l=0.3, lambda_g=0.2, tau=1, steps=4, config_id=111)
     from paper_1905_10395_b200.runner import Population
