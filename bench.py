@@ -399,8 +399,13 @@ def run_ours(args):
     if pop.lsgd.check_device() != 0:
         raise SystemExit("device status word set during the bench")
 
-    roofline = {"bound": "hbm", "kernel": "momentum_update_kernel" if with_momentum else
-                "pull_update_staged_kernel / plain_update_kernel", "achieved": achieved,
+    if with_momentum:
+        k1_name = "momentum_update_kernel"
+    elif spec["kind"] == "quadratic" or spec["P"] > 26:
+        k1_name = "update_chunked_kernel"
+    else:
+        k1_name = "pull_update_staged_kernel / plain_update_kernel"
+    roofline = {"bound": "hbm", "kernel": k1_name, "achieved": achieved,
                 "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
                 "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags)),

@@ -9,14 +9,14 @@
 // number of workers, at most a few thousand); the work is latency, not bandwidth.
 //
 // Optionally the kernel first finishes a two-stage loss reduction: loss_i = scale * sum_b
-// partials[i][b], summed in fp64 in index order by one lane per worker, so the value does not depend
+// partials[i][b], summed in fp64 by one warp per worker in a fixed order, so the value does not depend
 // on scheduling.
 #include "internal.h"
 
 namespace lsgd {
 namespace {
 
-constexpr int kElectThreads = 256;
+constexpr int kElectThreads = 1024;
 
 __device__ __forceinline__ uint32_t orderable(float v) {
   if (v != v) return 0xFFFFFFFFu;            // NaN: after +inf
@@ -36,11 +36,9 @@ __device__ __forceinline__ unsigned long long warp_min(unsigned long long k) {
 __global__ void __launch_bounds__(kElectThreads) elect_kernel(ElectArgs p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   if (p.partials != nullptr) {
-    for (int i = threadIdx.x; i < p.P; i += blockDim.x) {
-      const double* row = p.partials + (int64_t)i * p.n_partials;
-      double acc = 0.0;
-      for (int b = 0; b < p.n_partials; ++b) acc += row[b];
-      p.loss_out[i] = (float)(acc * p.partial_scale);
+    for (int i = warp; i < p.P; i += nwarps) {
+      const double acc = warp_sum_fixed(p.partials + (int64_t)i * p.n_partials, p.n_partials);
+      if (lane == 0) p.loss_out[i] = (float)(acc * p.partial_scale);
     }
   } else if (p.loss_in != p.loss_out) {
     for (int i = threadIdx.x; i < p.P; i += blockDim.x) p.loss_out[i] = p.loss_in[i];

@@ -128,6 +128,16 @@ cudaError_t launch_psd_grad(const float* x, float* g, const float* M, int32_t n,
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Sum of n doubles by one warp in a fixed order (lane-strided partial sums, then a butterfly), so the value
+// does not depend on timing.  All 32 lanes call it and all get the result.
+__device__ __forceinline__ double warp_sum_fixed(const double* __restrict__ v, int n) {
+  double acc = 0.0;
+  for (int b = threadIdx.x & 31; b < n; b += 32) acc += v[b];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+  return acc;
+}
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
   cudaLaunchConfig_t cfg = {};

@@ -2,7 +2,7 @@
 // Section 3.3 with a diagonal Hessian): materialised stochastic gradient g = a (x - b) + sigma eps
 // and the first stage of the exact election loss f(x_i).
 //
-// Loss: CTA (blk, row group) sums the terms of up to 8 workers over a fixed chunk of columns, every term
+// Loss: CTA (blk, row group) sums the terms of up to 4 workers over a fixed chunk of columns, every term
 // evaluated and accumulated in fp64, and writes one partial per worker; the election kernel adds the
 // partials in index order.
 // Chunking and tree shape depend only on d, so the result is reproducible run to run.
@@ -51,14 +51,16 @@ quadratic_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const 
   }
 }
 
-constexpr int kLossRows = 8;   // workers per CTA: a and b are loaded and converted once for all of them
+// Workers per CTA: a and b are loaded and converted once for all of them.  4 rather than 8: the CTAs of the
+// 64 x 2^20 problem then fill 2.8 waves instead of 1.4, and the partial sums stay the same bit for bit.
+constexpr int kLossRows = 4;
 
 __device__ __forceinline__ double term(double x, double a, double b) {
   const double r = x - b;
   return a * r * r;
 }
 
-// CTA (chunk, row group): partial sums of f over 8192 columns for up to 8 workers.
+// CTA (chunk, row group): partial sums of f over 8192 columns for up to kLossRows workers.
 __global__ void __launch_bounds__(kThreads)
 quadratic_loss_kernel(const float* __restrict__ x, const float* __restrict__ a, const float* __restrict__ b, int32_t P,
                       int64_t d, int64_t ld, double* __restrict__ partials, int32_t n_partials) {

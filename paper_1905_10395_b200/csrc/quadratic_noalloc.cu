@@ -24,15 +24,14 @@ constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) double g_noalloc_partials[kNoAllocMaxPartials];
 
-// loss[i] = 1/2 * (partials[i][0] + partials[i][1] + ...), added in index order in fp64 -- the same
-// order and rounding as the election kernel's own second stage.  Device code names the array directly.
+// loss[i] = 1/2 * (partials[i][0] + partials[i][1] + ...), one warp per worker, added in fp64 in the same
+// fixed order and with the same rounding as the election kernel's own second stage.  Device code names the
+// array directly.
 __global__ void __launch_bounds__(128) noalloc_finish_kernel(float* __restrict__ loss, int32_t P, int32_t n_partials) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= P) return;
-  const double* row = g_noalloc_partials + (int64_t)i * n_partials;
-  double acc = 0.0;
-  for (int b = 0; b < n_partials; ++b) acc += row[b];
-  loss[i] = (float)(acc * 0.5);
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (i >= P) return;      // whole warps leave together
+  const double acc = warp_sum_fixed(g_noalloc_partials + (int64_t)i * n_partials, n_partials);
+  if ((threadIdx.x & 31) == 0) loss[i] = (float)(acc * 0.5);
 }
 
 double* scratch_address_for_current_device(cudaError_t* err) {
@@ -73,6 +72,6 @@ extern "C" lsgd_status lsgd_quadratic_loss_noalloc(const float* x, const float* 
   // Every partial [i][blk] is written by exactly one CTA before it is read, so nothing has to be
   // cleared although the array still holds the previous call's values.
   if (launch_quadratic_loss_partials(x, a, b, P, d, ld, scratch, (int32_t)n_partials, s) != cudaSuccess) return LSGD_ERR_CUDA;
-  noalloc_finish_kernel<<<(P + 127) / 128, 128, 0, s>>>(loss, P, (int32_t)n_partials);
+  noalloc_finish_kernel<<<(P + 3) / 4, 128, 0, s>>>(loss, P, (int32_t)n_partials);
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
 }

@@ -112,6 +112,56 @@ __device__ __forceinline__ float pull1(float x, float g, float xl, float xg, con
   }
 }
 
+// The same three formulas on operands already held in the evaluation precision (double for modes 0 and 1,
+// float for mode 2).  float -> double is exact, so converting an operand once and reusing it gives the same
+// bits as converting it at every use.
+template <int MODE> struct Eval { using T = double; };
+template <> struct Eval<2> { using T = float; };
+
+template <int MODE>
+__device__ __forceinline__ float quad_g_t(typename Eval<MODE>::T X, typename Eval<MODE>::T A, typename Eval<MODE>::T B,
+                                          float n, const Coef& k, bool noise) {
+  if (MODE == 0) {
+    double r = __dmul_rn((double)A, __dsub_rn((double)X, (double)B));
+    if (noise) r = __dadd_rn(r, __dmul_rn(k.sigma, (double)n));
+    return (float)r;
+  } else if (MODE == 1) {
+    double r = (double)A * ((double)X - (double)B);
+    if (noise) r = fma(k.sigma, (double)n, r);
+    return (float)r;
+  } else {
+    return fmaf((float)A, (float)X - (float)B, noise ? k.sigma_f * n : 0.f);
+  }
+}
+
+template <int MODE>
+__device__ __forceinline__ float plain1_t(typename Eval<MODE>::T X, float g, const Coef& k) {
+  if (MODE == 0) return (float)__dsub_rn((double)X, __dmul_rn(k.eta, (double)g));
+  if (MODE == 1) return (float)fma(-k.eta, (double)g, (double)X);
+  return fmaf(-k.eta_f, g, (float)X);
+}
+
+template <int MODE>
+__device__ __forceinline__ float pull1_t(typename Eval<MODE>::T X, float g, typename Eval<MODE>::T XL,
+                                         typename Eval<MODE>::T XG, const Coef& k) {
+  if (MODE == 0) {
+    double acc = __dsub_rn((double)X, __dmul_rn(k.eta, (double)g));
+    acc = __dsub_rn(acc, __dmul_rn(k.cl, __dsub_rn((double)X, (double)XL)));
+    acc = __dsub_rn(acc, __dmul_rn(k.cg, __dsub_rn((double)X, (double)XG)));
+    return (float)acc;
+  } else if (MODE == 1) {
+    double acc = fma(-k.eta, (double)g, (double)X);
+    acc = fma(-k.cl, (double)X - (double)XL, acc);
+    acc = fma(-k.cg, (double)X - (double)XG, acc);
+    return (float)acc;
+  } else {
+    float acc = fmaf(-k.eta_f, g, (float)X);
+    acc = fmaf(-k.cl_f, (float)X - (float)XL, acc);
+    acc = fmaf(-k.cg_f, (float)X - (float)XG, acc);
+    return acc;
+  }
+}
+
 template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
 __global__ void __launch_bounds__(kThreads, LSGD_K1_PULL_MIN_BLOCKS)
 pull_update_kernel(UpdateArgs p, int64_t n4) {
@@ -617,6 +667,7 @@ update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
     }
   } else {
     // ------------------------------------------------------------------ consumers
+    using T = typename Eval<MODE>::T;
     const Coef k = p.k;
     const int w4 = W >> 2;                          // 16-byte columns per tile row
     const int c4 = threadIdx.x % w4;                // this thread's column
@@ -631,12 +682,21 @@ update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
       const int wt4 = (int)(((total_floats - c0) < W ? (total_floats - c0) : W) >> 2);
       const bool live = c4 < wt4;
       const float* lead = lead0 + (size_t)b * nlead * W + c4 * 4;
-      float4 xg = make_float4(0.f, 0.f, 0.f, 0.f), av = xg, bv = xg;
+      // a, b and the global leader's values are converted to the evaluation precision once per tile, a local
+      // leader's once per run of rows that share it: with fp64 evaluation the float <-> double conversions
+      // (16 per clock per SM) are what bounds this kernel, not the arithmetic or the memory system
+      T XG[4] = {0, 0, 0, 0}, A[4] = {0, 0, 0, 0}, B[4] = {0, 0, 0, 0}, XL[4] = {0, 0, 0, 0};
+      int cur_slot = -1;
       if (live) {
-        if (PULL) xg = *reinterpret_cast<const float4*>(lead + (size_t)gslot * W);
+        if (PULL) {
+          const float4 v = *reinterpret_cast<const float4*>(lead + (size_t)gslot * W);
+          XG[0] = (T)v.x; XG[1] = (T)v.y; XG[2] = (T)v.z; XG[3] = (T)v.w;
+        }
         if (QUAD) {
-          av = *reinterpret_cast<const float4*>(lead + (size_t)pull_slots * W);
-          bv = *reinterpret_cast<const float4*>(lead + (size_t)(pull_slots + 1) * W);
+          const float4 av = *reinterpret_cast<const float4*>(lead + (size_t)pull_slots * W);
+          const float4 bv = *reinterpret_cast<const float4*>(lead + (size_t)(pull_slots + 1) * W);
+          A[0] = (T)av.x; A[1] = (T)av.y; A[2] = (T)av.z; A[3] = (T)av.w;
+          B[0] = (T)bv.x; B[1] = (T)bv.y; B[2] = (T)bv.z; B[3] = (T)bv.w;
         }
       }
       for (int c = 0; c < n_chunks; ++c, ++cit) {
@@ -647,34 +707,35 @@ update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
         const int nr = (P - i0) < R ? (P - i0) : R;
         const float* sx = ring0 + (size_t)s * stage_rows * W + c4 * 4;
         const float* sg = sx + (size_t)R * W;
-        if (live) {
-          for (int q = r0; q < nr; q += rstep) {
-            const int i = i0 + q;
-            float4 xl = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (PULL) xl = *reinterpret_cast<const float4*>(lead + (size_t)s_lead[i] * W);
-            const float4 x = (PULL && s_self[i]) ? xl : *reinterpret_cast<const float4*>(sx + (size_t)q * W);
-            float4 g = has_g ? *reinterpret_cast<const float4*>(sg + (size_t)q * W) : make_float4(0.f, 0.f, 0.f, 0.f);
-            if (QUAD && p.use_g) {
-              g.x = quad_g<MODE>(x.x, av.x, bv.x, g.x, k, NOISE);
-              g.y = quad_g<MODE>(x.y, av.y, bv.y, g.y, k, NOISE);
-              g.z = quad_g<MODE>(x.z, av.z, bv.z, g.z, k, NOISE);
-              g.w = quad_g<MODE>(x.w, av.w, bv.w, g.w, k, NOISE);
-            }
-            float4 r;
+        for (int q = r0; q < nr; q += rstep) {
+          const int i = i0 + q;
+          if (live) {
             if (PULL) {
-              r.x = pull1<MODE>(x.x, g.x, xl.x, xg.x, k);
-              r.y = pull1<MODE>(x.y, g.y, xl.y, xg.y, k);
-              r.z = pull1<MODE>(x.z, g.z, xl.z, xg.z, k);
-              r.w = pull1<MODE>(x.w, g.w, xl.w, xg.w, k);
-            } else {
-              r.x = plain1<MODE>(x.x, g.x, k);
-              r.y = plain1<MODE>(x.y, g.y, k);
-              r.z = plain1<MODE>(x.z, g.z, k);
-              r.w = plain1<MODE>(x.w, g.w, k);
+              const int slot = s_lead[i];
+              if (slot != cur_slot) {
+                cur_slot = slot;
+                const float4 v = *reinterpret_cast<const float4*>(lead + (size_t)slot * W);
+                XL[0] = (T)v.x; XL[1] = (T)v.y; XL[2] = (T)v.z; XL[3] = (T)v.w;
+              }
             }
+            T X[4];
+            if (PULL && s_self[i]) {
+              X[0] = XL[0]; X[1] = XL[1]; X[2] = XL[2]; X[3] = XL[3];
+            } else {
+              const float4 v = *reinterpret_cast<const float4*>(sx + (size_t)q * W);
+              X[0] = (T)v.x; X[1] = (T)v.y; X[2] = (T)v.z; X[3] = (T)v.w;
+            }
+            const float4 gv = has_g ? *reinterpret_cast<const float4*>(sg + (size_t)q * W) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float g[4] = {gv.x, gv.y, gv.z, gv.w}, r[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              if (QUAD && p.use_g) g[e] = quad_g_t<MODE>(X[e], A[e], B[e], g[e], k, NOISE);
+              r[e] = PULL ? pull1_t<MODE>(X[e], g[e], XL[e], XG[e], k) : plain1_t<MODE>(X[e], g[e], k);
+            }
+            const float4 rv = make_float4(r[0], r[1], r[2], r[3]);
             const int64_t off = (int64_t)i * p.ld + c0 + c4 * 4;
-            st4(p.x + off, r);
-            if (SHADOW) st4_bf16(p.x_bf16 + off, r);
+            st4(p.x + off, rv);
+            if (SHADOW) st4_bf16(p.x_bf16 + off, rv);
           }
         }
         __syncwarp();
