@@ -5,7 +5,7 @@
 // Parameter row = [W1 | b1 | W2 | b2 | W3 | b3], W_l stored [n_out][n_in].  All matrix products take
 // bf16 operands and accumulate in fp32:
 //   forward   H1 = relu(X W1^T + b1), H2 = relu(H1 W2^T + b2)            tensor cores (gemm_tc.cu)
-//   head      Z = H2 W3^T + b3, loss, dZ, dW3, db3, dH2, db2             CUDA cores (n_classes is tiny)
+//   head      Z = H2 W3^T + b3, loss, dZ, dH2; dW3, db3, db2, db1        CUDA cores (n_classes is tiny)
 //   backward  dH1 = (dH2 W2) * [H1 > 0], dW2 = dH2^T H1, dW1 = dH1^T X   tensor cores
 // Stored activations and back-propagated deltas are rounded to bf16 once, when they are written.
 // The bf16 copy of the weights is refreshed by the update kernel itself when it writes x.
@@ -134,8 +134,8 @@ template <int S>
 __global__ void __launch_bounds__(kHeadWarps * 32)
 head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ x,
                     const int32_t* __restrict__ labels, const int32_t* __restrict__ label_idx, float* __restrict__ dz,
-                    float* __restrict__ loss_b, int32_t n, int32_t d2, int32_t C, int64_t ld, int64_t w3_off, int64_t b3_off,
-                    int32_t label_rows, int32_t groups_per_warp, uint32_t* status) {
+                    __nv_bfloat16* __restrict__ dh2, float* __restrict__ loss_b, int32_t n, int32_t d2, int32_t C, int64_t ld,
+                    int64_t w3_off, int64_t b3_off, int32_t label_rows, int32_t groups_per_warp, uint32_t* status) {
   pdl_wait();
   pdl_launch_dependents();
   extern __shared__ uint4 s_w3[];   // [C][d2 / 8]
@@ -178,19 +178,22 @@ head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* _
       for (int c = 0; c < kMaxClasses; ++c)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc[sx][c] += __shfl_xor_sync(0xFFFFFFFFu, acc[sx][c], o);
-    // lane sx finishes sample b0 + sx (every lane holds all the reduced sums)
+    // Every lane holds all the reduced sums.  Held-out batch: lane sx finishes sample b0 + sx.  Training batch:
+    // all lanes finish the sample together (the same arithmetic in every lane), lane sx stores the loss and dZ,
+    // and the warp goes on to this sample's row of dH2 = [H2 > 0] * (dZ W3) while W3 is still in shared memory.
 #pragma unroll
     for (int sx = 0; sx < S; ++sx) {
       const int b = b0 + sx;
-      if (lane == sx && b < n) {
+      const bool writer = lane == sx;
+      if ((writer || dh2 != nullptr) && b < n) {
         int y = label_idx ? label_idx[(int64_t)i * n + b] : b;   // training: pool row of this sample
         if (y < 0 || y >= label_rows) {
-          atomicOr(status, FLAG_BAD_INDEX);
+          if (writer) atomicOr(status, FLAG_BAD_INDEX);
           y = 0;
         }
         int cls = labels[y];
         if (cls < 0 || cls >= C) {
-          atomicOr(status, FLAG_BAD_INDEX);
+          if (writer) atomicOr(status, FLAG_BAD_INDEX);
           cls = 0;
         }
         float zmax = -INFINITY;
@@ -208,166 +211,192 @@ head_forward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* _
             if (c == cls) zy = acc[sx][c];
           }
         const float lse = zmax + logf(sum);
-        loss_b[(int64_t)i * n + b] = lse - zy;
+        if (writer) loss_b[(int64_t)i * n + b] = lse - zy;
         if (dz) {
           const float inv_n = 1.f / (float)n;
+          float zr[kMaxClasses];          // dZ of this sample, rounded to bf16 as every back-propagated delta is
 #pragma unroll
-          for (int c = 0; c < kMaxClasses; ++c)
+          for (int c = 0; c < kMaxClasses; ++c) {
+            zr[c] = 0.f;
             if (c < C) {
               const float pc = expf(acc[sx][c] - lse);
               const float v = (pc - (c == cls ? 1.f : 0.f)) * inv_n;
-              dz[((int64_t)i * n + b) * C + c] = __bfloat162float(__float2bfloat16_rn(v));
+              zr[c] = __bfloat162float(__float2bfloat16_rn(v));
+              if (writer) dz[((int64_t)i * n + b) * C + c] = zr[c];
             }
+          }
+          if (dh2) {
+            const uint4* hrow = reinterpret_cast<const uint4*>(h2 + ((int64_t)i * n + b) * d2);
+            uint4* drow = reinterpret_cast<uint4*>(dh2 + ((int64_t)i * n + b) * d2);
+            for (int ch = lane; ch < chunks; ch += 32) {
+              float hv[8], dh[8];
+              unpack8(hrow[ch], hv);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) dh[j] = 0.f;
+#pragma unroll
+              for (int c = 0; c < kMaxClasses; ++c)
+                if (c < C) {
+                  float wv[8];
+                  unpack8(s_w3[c * chunks + ch], wv);
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) dh[j] = fmaf(zr[c], wv[j], dh[j]);
+                }
+              uint4 o;
+              uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const __nv_bfloat162 r = __floats2bfloat162_rn(hv[2 * j] > 0.f ? dh[2 * j] : 0.f, hv[2 * j + 1] > 0.f ? dh[2 * j + 1] : 0.f);
+                ow[j] = *reinterpret_cast<const uint32_t*>(&r);
+              }
+              drow[ch] = o;
+            }
+          }
         }
       }
     }
   }
 }
 
-constexpr int kBwdThreadsX = 64;   // each thread owns two adjacent hidden units (one bf16x2)
-constexpr int kBwdCols = 2 * kBwdThreadsX;
-constexpr int kBwdSlices = 8;      // batch slices per CTA (blockDim.y), combined in a fixed order
 constexpr int kDzPitch = kMaxClasses;
 
-// Last layer backward.  Thread (k, s) walks the samples b = s, s + 8, ... of hidden units 2k, 2k + 1:
-// dH2[b][k] = [H2 > 0] * sum_c dZ[b][c] W3[c][k] (rounded to bf16 and stored), and its share of
-// dW3[:, k] and db2[k]; the slices are added in slice order.  Block 0 of each worker also writes db3.
-__global__ void __launch_bounds__(kBwdThreadsX * kBwdSlices)
-head_backward_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ wb, const float* __restrict__ dz,
-                     __nv_bfloat16* __restrict__ dh2, float* __restrict__ g, int32_t n, int32_t d2, int32_t C, int64_t ld,
-                     int64_t w3_off, int64_t b3_off, int64_t b2_off) {
+// Plain step of one parameter, the arithmetic of the update kernels (fp64 unfused / fp64 fused / fp32 fused).
+__device__ __forceinline__ float sgd1(float x, float g, double eta, int arith) {
+  if (arith == 0) return (float)__dsub_rn((double)x, __dmul_rn(eta, (double)g));
+  if (arith == 1) return (float)fma(-eta, (double)g, (double)x);
+  return fmaf(-(float)eta, g, x);
+}
+
+// Every gradient that is a sum over the batch of stored quantities, in one launch.  A CTA takes 128 columns of
+// one worker and one of three jobs:
+//   blocks [0, nb2)              : dW3[c][k] = sum_b dZ[b][c] H2[b][k]; block 0 also db3[c] = sum_b dZ[b][c];
+//   blocks [nb2, 2 nb2)          : db2[k] = sum_b dH2[b][k];
+//   blocks [2 nb2, 2 nb2 + nb1)  : db1[k] = sum_b dH1[b][k].
+// Thread (k, s) owns columns 2k, 2k + 1 and the samples b = s, s + 8, ...; the slices are added in slice order.
+// The kernel is all memory latency; two CTAs per SM with four loads in flight per thread measured best (more
+// loads in flight cost registers, and spills or a single CTA per SM cost more than they gain).
+// With sgd set the plain step x <- x - eta g of these parameters is taken here as well (x and its bf16 copy),
+// so that nothing is left for a separate update launch.
+constexpr int kBwdThreadsX = 64;   // each thread owns two adjacent columns (one bf16x2)
+constexpr int kBwdCols = 2 * kBwdThreadsX;
+constexpr int kBwdSlices = 8;      // batch slices per CTA (blockDim.y), combined in a fixed order
+constexpr int kSumBatch = 4;       // samples whose loads a thread has in flight
+__global__ void __launch_bounds__(kBwdThreadsX * kBwdSlices, 2)
+batch_sums_kernel(const __nv_bfloat16* __restrict__ h2, const __nv_bfloat16* __restrict__ dh2, const __nv_bfloat16* __restrict__ dh1,
+                  const float* __restrict__ dz, float* __restrict__ g, float* __restrict__ x, __nv_bfloat16* __restrict__ wb,
+                  int32_t n, int32_t d1, int32_t d2, int32_t C, int64_t ld, int64_t w3_off, int64_t b3_off, int64_t b2_off,
+                  int64_t b1_off, int32_t nb2, bool sgd, double eta, int arith) {
   pdl_wait();
   pdl_launch_dependents();
   extern __shared__ __align__(16) float s_mem[];
-  float* s_dz = s_mem;                              // [n][kDzPitch], zero beyond C
-  float* s_red = s_mem + (size_t)n * kDzPitch;      // [kBwdSlices][C + 1][kBwdCols]
+  float* s_dz = s_mem;                              // [n][kDzPitch], zero beyond C (job 0 only)
+  float* s_red = s_mem + (size_t)n * kDzPitch;      // [kBwdSlices][rows][kBwdCols]
   const int i = blockIdx.y;
   const int tx = threadIdx.x, ty = threadIdx.y;
   const int tid = ty * kBwdThreadsX + tx;
-  const float* dzi = dz + (int64_t)i * n * C;
-  for (int t = tid; t < n * kDzPitch; t += kBwdThreadsX * kBwdSlices) {
-    const int b = t / kDzPitch, c = t - b * kDzPitch;
-    s_dz[t] = c < C ? dzi[b * C + c] : 0.f;
-  }
-  __syncthreads();
+  constexpr int kThreads = kBwdThreadsX * kBwdSlices;
   float* gi = g + (int64_t)i * ld;
-  if (blockIdx.x == 0 && tid < C) {
-    float s = 0.f;
-    for (int b = 0; b < n; ++b) s += s_dz[b * kDzPitch + tid];
-    gi[b3_off + tid] = s;
+  float* xi = x + (int64_t)i * ld;
+  __nv_bfloat16* wi = wb + (int64_t)i * ld;
+  const int job = (int)blockIdx.x < nb2 ? 0 : ((int)blockIdx.x < 2 * nb2 ? 1 : 2);
+  const int blk = blockIdx.x - (job == 0 ? 0 : (job == 1 ? nb2 : 2 * nb2));
+  const int dcols = job == 2 ? d1 : d2;
+  const int rows = job == 0 ? C : 1;                // accumulator rows per column
+  const __nv_bfloat16* src = (job == 0 ? h2 : (job == 1 ? dh2 : dh1)) + (int64_t)i * n * dcols;
+  // where output (row c, column kcol) lives in the parameter row
+  auto out_off = [&](int c, int kcol) -> int64_t {
+    return job == 0 ? w3_off + (int64_t)c * d2 + kcol : (job == 1 ? b2_off : b1_off) + kcol;
+  };
+  // the x values the plain step will need: fetched now, used at the very end
+  constexpr int kMaxOut = (kMaxClasses * kBwdCols + kThreads - 1) / kThreads;
+  float x_old[kMaxOut];
+#pragma unroll
+  for (int u = 0; u < kMaxOut; ++u) {
+    const int t = tid + u * kThreads;
+    const int c = t / kBwdCols, kcol = blk * kBwdCols + (t - c * kBwdCols);
+    x_old[u] = (sgd && c < rows && kcol < dcols) ? xi[out_off(c, kcol)] : 0.f;
   }
-  const int k = blockIdx.x * kBwdCols + 2 * tx;     // d2 is even: k and k + 1 are both valid or both not
-  const bool live = k < d2;
-  const __nv_bfloat16* w3 = wb + (int64_t)i * ld + w3_off;
-  float w0[kMaxClasses], w1[kMaxClasses], a0[kMaxClasses], a1[kMaxClasses];
+  if (job == 0) {
+    const float* dzi = dz + (int64_t)i * n * C;
+    for (int t = tid; t < n * kDzPitch; t += kThreads) {
+      const int b = t / kDzPitch, c = t - b * kDzPitch;
+      s_dz[t] = c < C ? dzi[b * C + c] : 0.f;
+    }
+    __syncthreads();
+    if (blk == 0 && tid < C) {
+      float sum = 0.f;
+      for (int b = 0; b < n; ++b) sum += s_dz[b * kDzPitch + tid];
+      gi[b3_off + tid] = sum;
+      if (sgd) {
+        const float xn = sgd1(xi[b3_off + tid], sum, eta, arith);
+        xi[b3_off + tid] = xn;
+        wi[b3_off + tid] = __float2bfloat16_rn(xn);
+      }
+    }
+  }
+  const int k = blk * kBwdCols + 2 * tx;            // layer widths are even: k and k + 1 are both valid or both not
+  const bool live = k < dcols;
+  float a0[kMaxClasses], a1[kMaxClasses];
 #pragma unroll
   for (int c = 0; c < kMaxClasses; ++c) {
-    float2 wv = make_float2(0.f, 0.f);
-    if (live && c < C) wv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(w3 + (int64_t)c * d2 + k));
-    w0[c] = wv.x;
-    w1[c] = wv.y;
     a0[c] = 0.f;
     a1[c] = 0.f;
   }
-  float ab0 = 0.f, ab1 = 0.f;
   if (live) {
-    const __nv_bfloat16* hcol = h2 + (int64_t)i * n * d2 + k;
-    __nv_bfloat16* dcol = dh2 + (int64_t)i * n * d2 + k;
-    for (int b0 = ty; b0 < n; b0 += 4 * kBwdSlices) {
-      float2 hv[4];
+    const __nv_bfloat16* col = src + k;
+    for (int b0 = ty; b0 < n; b0 += kSumBatch * kBwdSlices) {
+      uint32_t raw[kSumBatch];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < kSumBatch; ++u) {
         const int b = b0 + u * kBwdSlices;
-        hv[u] = b < n ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hcol + (int64_t)b * d2)) : make_float2(0.f, 0.f);
+        raw[u] = b < n ? *reinterpret_cast<const uint32_t*>(col + (int64_t)b * dcols) : 0u;
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < kSumBatch; ++u) {
         const int b = b0 + u * kBwdSlices;
         if (b < n) {
-          float z[kMaxClasses];
+          const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw[u]));
+          if (job == 0) {
 #pragma unroll
-          for (int q = 0; q < kMaxClasses / 4; ++q) {
-            const float4 t = *reinterpret_cast<const float4*>(s_dz + b * kDzPitch + 4 * q);
-            z[4 * q] = t.x; z[4 * q + 1] = t.y; z[4 * q + 2] = t.z; z[4 * q + 3] = t.w;
-          }
-          float dh0 = 0.f, dh1 = 0.f;
-#pragma unroll
-          for (int c = 0; c < kMaxClasses; ++c)
-            if (c < C) {
-              a0[c] = fmaf(z[c], hv[u].x, a0[c]);
-              a1[c] = fmaf(z[c], hv[u].y, a1[c]);
-              dh0 = fmaf(z[c], w0[c], dh0);
-              dh1 = fmaf(z[c], w1[c], dh1);
+            for (int q = 0; q < kMaxClasses / 4; ++q) {
+              if (4 * q < C) {      // entries beyond C are zero in s_dz
+                const float4 t = *reinterpret_cast<const float4*>(s_dz + b * kDzPitch + 4 * q);
+                a0[4 * q] = fmaf(t.x, v.x, a0[4 * q]);         a1[4 * q] = fmaf(t.x, v.y, a1[4 * q]);
+                a0[4 * q + 1] = fmaf(t.y, v.x, a0[4 * q + 1]); a1[4 * q + 1] = fmaf(t.y, v.y, a1[4 * q + 1]);
+                a0[4 * q + 2] = fmaf(t.z, v.x, a0[4 * q + 2]); a1[4 * q + 2] = fmaf(t.z, v.y, a1[4 * q + 2]);
+                a0[4 * q + 3] = fmaf(t.w, v.x, a0[4 * q + 3]); a1[4 * q + 3] = fmaf(t.w, v.y, a1[4 * q + 3]);
+              }
             }
-          const __nv_bfloat162 r = __floats2bfloat162_rn(hv[u].x > 0.f ? dh0 : 0.f, hv[u].y > 0.f ? dh1 : 0.f);
-          *reinterpret_cast<__nv_bfloat162*>(dcol + (int64_t)b * d2) = r;
-          const float2 rf = __bfloat1622float2(r);
-          ab0 += rf.x;
-          ab1 += rf.y;
+          } else {
+            a0[0] += v.x;
+            a1[0] += v.y;
+          }
         }
       }
     }
   }
-  float* red = s_red + (size_t)ty * (C + 1) * kBwdCols;
+  float* red = s_red + (size_t)ty * rows * kBwdCols;
 #pragma unroll
   for (int c = 0; c < kMaxClasses; ++c)
-    if (c < C) {
+    if (c < rows) {
       red[c * kBwdCols + 2 * tx] = a0[c];
       red[c * kBwdCols + 2 * tx + 1] = a1[c];
     }
-  red[C * kBwdCols + 2 * tx] = ab0;
-  red[C * kBwdCols + 2 * tx + 1] = ab1;
   __syncthreads();
-  // (C + 1) x kBwdCols sums over the slices, in slice order
-  for (int t = tid; t < (C + 1) * kBwdCols; t += kBwdThreadsX * kBwdSlices) {
+  // rows x kBwdCols sums over the slices, in slice order
+#pragma unroll
+  for (int u = 0; u < kMaxOut; ++u) {
+    const int t = tid + u * kThreads;
     const int c = t / kBwdCols, kk = t - c * kBwdCols;
-    const int kcol = blockIdx.x * kBwdCols + kk;
-    if (kcol >= d2) continue;
+    const int kcol = blk * kBwdCols + kk;
+    if (c >= rows || kcol >= dcols) continue;
     float acc = 0.f;
-    for (int sl = 0; sl < kBwdSlices; ++sl) acc += s_red[((size_t)sl * (C + 1) + c) * kBwdCols + kk];
-    if (c < C) gi[w3_off + (int64_t)c * d2 + kcol] = acc;
-    else gi[b2_off + kcol] = acc;
-  }
-}
-
-constexpr int kSumThreadsX = 64, kSumSlices = 8;
-
-// db[k] = sum_b delta[b][k] for a stored (bf16) delta matrix; thread (k, s) adds the samples s, s + 8, ...
-// of columns 2k, 2k + 1 and the slices are combined in slice order.
-__global__ void __launch_bounds__(kSumThreadsX * kSumSlices)
-column_sum_kernel(const __nv_bfloat16* __restrict__ delta, float* __restrict__ g, int32_t n, int32_t dcols, int64_t ld, int64_t off) {
-  pdl_wait();
-  pdl_launch_dependents();
-  __shared__ float s_part[kSumSlices][2 * kSumThreadsX];
-  const int i = blockIdx.y, tx = threadIdx.x, ty = threadIdx.y;
-  const int k = blockIdx.x * 2 * kSumThreadsX + 2 * tx;
-  float s0 = 0.f, s1 = 0.f;
-  if (k < dcols) {
-    const __nv_bfloat16* col = delta + (int64_t)i * n * dcols + k;
-    for (int b0 = ty; b0 < n; b0 += 4 * kSumSlices) {
-      float2 v[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int b = b0 + u * kSumSlices;
-        v[u] = b < n ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(col + (int64_t)b * dcols)) : make_float2(0.f, 0.f);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        s0 += v[u].x;
-        s1 += v[u].y;
-      }
-    }
-  }
-  s_part[ty][2 * tx] = s0;
-  s_part[ty][2 * tx + 1] = s1;
-  __syncthreads();
-  const int t = ty * kSumThreadsX + tx;
-  if (t < 2 * kSumThreadsX) {
-    const int kcol = blockIdx.x * 2 * kSumThreadsX + t;
-    if (kcol < dcols) {
-      float acc = 0.f;
-      for (int sl = 0; sl < kSumSlices; ++sl) acc += s_part[sl][t];
-      g[(int64_t)i * ld + off + kcol] = acc;
+    for (int sl = 0; sl < kBwdSlices; ++sl) acc += s_red[((size_t)sl * rows + c) * kBwdCols + kk];
+    const int64_t off = out_off(c, kcol);
+    gi[off] = acc;
+    if (sgd) {
+      const float xn = sgd1(x_old[u], acc, eta, arith);
+      xi[off] = xn;
+      wi[off] = __float2bfloat16_rn(xn);
     }
   }
 }
@@ -465,8 +494,7 @@ lsgd_status mlp_validate(const lsgd_config& c, const lsgd_mlp_desc& m) {
   if (m.batch % 8 || m.n_heldout % 8 || m.batch > 1024) return LSGD_ERR_UNSUPPORTED;
   // shared-memory budgets of the last-layer kernels (48 KB without opting in)
   if ((size_t)m.dims[3] * m.dims[2] * 2 > 48 * 1024) return LSGD_ERR_UNSUPPORTED;
-  if (sizeof(float) * ((size_t)m.batch * kDzPitch + (size_t)kBwdSlices * (m.dims[3] + 1) * kBwdCols) > 160 * 1024)
-    return LSGD_ERR_UNSUPPORTED;
+  if (sizeof(float) * ((size_t)m.batch * kDzPitch + (size_t)8 * m.dims[3] * 128) > 160 * 1024) return LSGD_ERR_UNSUPPORTED;
   const Layout L = param_layout(m.dims);
   if (L.d != c.d || c.ld != c.d) return LSGD_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(m.scratch) & 1023u) return LSGD_ERR_ALIGNMENT;
@@ -544,26 +572,15 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
 
   const size_t w3_smem = (size_t)d[3] * d[2] * 2;
   if (launch_pdl(head_forward_kernel<1>, dim3((B + kHeadWarps - 1) / kHeadWarps, P), dim3(kHeadWarps * 32), w3_smem, s,
-                 st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->loss_b, B, d[2], d[3], ld, st->L.w[2], st->L.b[2],
-                 m.pool, 1, h->d_status) != cudaSuccess)
+                 st->h2, st->wb, c.x, m.pool_y, batch_idx, st->dz, st->dh2, st->loss_b, B, d[2], d[3], ld, st->L.w[2],
+                 st->L.b[2], m.pool, 1, h->d_status) != cudaSuccess)
     return LSGD_ERR_CUDA;
-  const size_t bwd_smem = sizeof(float) * ((size_t)B * kDzPitch + (size_t)kBwdSlices * (d[3] + 1) * kBwdCols);
-  static bool bwd_attr = false;
-  if (!bwd_attr) {
-    if (cudaFuncSetAttribute(head_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
-      return LSGD_ERR_CUDA;
-    bwd_attr = true;
-  }
   if (m.loss_window > 0) {   // remember this step's mean minibatch losses for the running-mean election
     if (launch_pdl(row_mean_kernel, dim3(P), dim3(32), 0, s, st->loss_b, st->ring + (st->n_grads % m.loss_window) * P,
                    B) != cudaSuccess)
       return LSGD_ERR_CUDA;
     st->n_grads++;
   }
-  if (launch_pdl(head_backward_kernel, dim3((d[2] + kBwdCols - 1) / kBwdCols, P), dim3(kBwdThreadsX, kBwdSlices), bwd_smem,
-                 s, st->h2, st->wb, st->dz, st->dh2, c.g, B, d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1]) !=
-      cudaSuccess)
-    return LSGD_ERR_CUDA;
 
   // dH1 = (dH2 . W2) masked by H1 > 0        [B x d1] = [B x d2] . [d2 x d1]
   GemmShape gd = shape(B, d[1], d[2], P, 0, 1, 1, GEMM_EPI_MASK_BF16, st->dh1, d[1], (int64_t)B * d[1], h->d_status);
@@ -571,6 +588,23 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   gd.ld_mask = d[1];
   gd.stride_mask = (int64_t)B * d[1];
   if (launch_bgemm(st->m_dh2, st->m_w2, gd, s) != cudaSuccess) return LSGD_ERR_CUDA;
+  // dW3, db3, db2, db1: the sums over the batch (and, fused, the plain step of those parameters)
+  const size_t sums_smem = sizeof(float) * ((size_t)B * kDzPitch + (size_t)kBwdSlices * d[3] * kBwdCols);
+  static bool sums_attr = false;
+  if (!sums_attr) {
+    if (cudaFuncSetAttribute(batch_sums_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
+      return LSGD_ERR_CUDA;
+    // two CTAs per SM: ask for the largest shared-memory carve-out (the default fits one CTA only)
+    if (cudaFuncSetAttribute(batch_sums_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) !=
+        cudaSuccess)
+      return LSGD_ERR_CUDA;
+    sums_attr = true;
+  }
+  const int nb2 = (d[2] + kBwdCols - 1) / kBwdCols, nb1 = (d[1] + kBwdCols - 1) / kBwdCols;
+  if (launch_pdl(batch_sums_kernel, dim3(2 * nb2 + nb1, P), dim3(kBwdThreadsX, kBwdSlices), sums_smem, s, st->h2, st->dh2, st->dh1,
+                 st->dz, c.g, c.x, st->wb, B, d[1], d[2], d[3], ld, st->L.w[2], st->L.b[2], st->L.b[1], st->L.b[0], nb2, fuse_sgd,
+                 (double)c.eta, (int)c.arithmetic) != cudaSuccess)
+    return LSGD_ERR_CUDA;
   // dW2 = dH2^T . H1                          [d2 x d1], contraction over the batch
   GemmShape g2 = shape(d[2], d[1], B, P, 1, 1, 1, fuse_sgd ? GEMM_EPI_SGD : GEMM_EPI_F32, c.g + st->L.w[1], d[1], ld, h->d_status);
   g2.x_upd = c.x + st->L.w[1];
@@ -578,9 +612,6 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   g2.eta = (double)c.eta;
   g2.arith = c.arithmetic;
   if (launch_bgemm(st->m_dh2, st->m_h1, g2, s) != cudaSuccess) return LSGD_ERR_CUDA;
-  if (launch_pdl(column_sum_kernel, dim3((d[1] + 2 * kSumThreadsX - 1) / (2 * kSumThreadsX), P),
-                 dim3(kSumThreadsX, kSumSlices), 0, s, st->dh1, c.g, B, d[1], ld, st->L.b[0]) != cudaSuccess)
-    return LSGD_ERR_CUDA;
   // dW1 = dH1^T . X                           [d1 x d0]
   GemmShape g1 = shape(d[1], d[0], B, P, 1, 1, 1, fuse_sgd ? GEMM_EPI_SGD : GEMM_EPI_F32, c.g + st->L.w[0], d[0], ld, h->d_status);
   g1.x_upd = c.x + st->L.w[0];
@@ -610,8 +641,8 @@ lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss) {
     constexpr int kS = 4, kGroups = 2;   // 8 warps x 2 groups x 4 samples = 64 samples per CTA
     const int per_cta = kHeadWarps * kGroups * kS;
     head_forward_kernel<kS><<<dim3((st->nH + per_cta - 1) / per_cta, st->P), kHeadWarps * 32, (size_t)d[3] * d[2] * 2, h->stream>>>(
-        st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr, st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2], st->L.b[2], st->nH,
-        kGroups, h->d_status);
+        st->hh2, st->wb, c.x, m.held_y, nullptr, nullptr, nullptr, st->loss_h, st->nH, d[2], d[3], st->ld, st->L.w[2], st->L.b[2],
+        st->nH, kGroups, h->d_status);
   }
   row_mean_kernel<<<st->P, 32, 0, h->stream>>>(st->loss_h, loss, st->nH);
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
@@ -634,13 +665,10 @@ lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss) {
 }
 
 int mlp_unfused_ranges(lsgd_ctx* h, int64_t (*ranges)[2]) {
-  MlpState* st = state(h);
-  // everything except W1 and W2: b1, then b2 | W3 | b3 (contiguous)
-  ranges[0][0] = st->L.b[0];
-  ranges[0][1] = st->L.w[1] - st->L.b[0];
-  ranges[1][0] = st->L.b[1];
-  ranges[1][1] = st->L.d - st->L.b[1];
-  return 2;
+  // none: W1, W2 are stepped in the weight-gradient products, the biases and W3 in the batch-sum kernel
+  (void)h;
+  (void)ranges;
+  return 0;
 }
 
 lsgd_status mlp_refresh_shadow(lsgd_ctx* h) {
