@@ -164,13 +164,20 @@ typedef struct {
   float weight_decay;        /* L2 decay coefficient, finite (the paper uses 1e-4)                   */
 } lsgd_config;
 
-/* MLP objective: on steps that are not pull steps, let lsgd_grad apply x <- x - eta g for W1 and W2
- * inside the epilogue of the weight-gradient products (same arithmetic, bit-identical result; g is then
- * not written for those two blocks and lsgd_step only finishes the biases and W3).  With this flag,
- * lsgd_grad may be called once per step and lsgd_elect(h, NULL) must not be called between lsgd_grad
- * and lsgd_step on a non-pull step (LSGD_ERR_STATE): the parameters are already partly advanced.
- * Off by default: the separate update kernel is currently the faster path.                          */
+/* MLP objective: on steps that are not pull steps, let lsgd_grad apply x <- x - eta g itself: for W1 and
+ * W2 inside the epilogue of the weight-gradient products (g is then not written for those two blocks), for
+ * the biases and W3 in the kernel that sums their gradients over the batch.  Same arithmetic as the update
+ * kernel, bit-identical result; lsgd_step then only advances the step counter.  With this flag, lsgd_grad
+ * may be called once per step and lsgd_elect(h, NULL) must not be called between lsgd_grad and lsgd_step on
+ * a non-pull step (LSGD_ERR_STATE): the parameters are already advanced.  Off by default.            */
 #define LSGD_FLAG_MLP_FUSED_STEP 1u
+
+/* MATCOMP objective: on steps that are not pull steps, lsgd_grad leaves the gradient as exact fixed-point
+ * sums in the library's accumulator and does not write g; lsgd_step takes x <- x - eta g straight from those
+ * sums, touching only the entries the minibatch reached (same arithmetic, bit-identical x).  lsgd_grad may
+ * then be called once per step (a second call before lsgd_step: LSGD_ERR_STATE).  Ignored with a momentum
+ * buffer or LSGD_FLAG_ALGORITHM1.  Off by default.                                                  */
+#define LSGD_FLAG_MATCOMP_FUSED_STEP 4u
 
 /* The schedule of the paper's Algorithm 1, run synchronously, instead of the fused Eq. (1) step:
  *   lsgd_elect at t = 0          initialisation: both elections, leader parameters copied, no pull;

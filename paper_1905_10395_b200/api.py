@@ -17,6 +17,7 @@ OBJ_EXTERNAL, OBJ_QUADRATIC, OBJ_MATCOMP, OBJ_MLP, OBJ_PSD_COMPLETION = range(5)
 ARITH_FP64, ARITH_FP64_FMA, ARITH_FP32 = range(3)
 FLAG_MLP_FUSED_STEP = 1
 FLAG_ALGORITHM1 = 2
+FLAG_MATCOMP_FUSED_STEP = 4
 
 
 class LsgdError(RuntimeError):

@@ -104,7 +104,11 @@ struct MatcompArgs {
   uint32_t* status;
 };
 // acc: DEVICE u64[P*ld] fixed-point accumulator, all zero on entry and again on exit
-cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, cudaStream_t s);
+// finish: also convert the sums to fp32 in a.g and clear acc; otherwise the sums stay in acc for
+// launch_matcomp_finish_step, which takes the plain step x <- x - eta g from them and clears acc
+cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, bool finish, cudaStream_t s);
+cudaError_t launch_matcomp_finish_step(unsigned long long* acc, float* x, int32_t P, int64_t ld, double eta, int arith,
+                                       cudaStream_t s);
 int32_t matcomp_loss_blocks(int32_t n_heldout);
 cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials, int32_t n_partials,
                                          cudaStream_t s);
@@ -181,4 +185,5 @@ struct lsgd_ctx {
   const float* armed_noise;  // QUADRATIC with g == NULL: noise pointer for the next step
   void* mlp_state;           // opaque MLP pipeline state
   unsigned long long* d_acc64;  // MATCOMP: fixed-point gradient accumulator [P*ld], kept all-zero between steps
+  bool mc_step_pending;         // MATCOMP fused step: the gradient sums wait in d_acc64 for lsgd_step
 };

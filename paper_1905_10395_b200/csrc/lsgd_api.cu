@@ -118,6 +118,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->n_elections = 0;
   h->grad_ready = false;
   h->fused_applied = false;
+  h->mc_step_pending = false;
   h->armed_noise = nullptr;
   h->slab = nullptr;
   h->mlp_state = nullptr;
@@ -227,8 +228,12 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
       break;
     case LSGD_OBJ_MATCOMP: {
       if (!batch) return LSGD_ERR_INVALID_ARG;
+      if (h->mc_step_pending) return LSGD_ERR_STATE;   // the previous gradient still waits for its lsgd_step
       MatcompArgs a{h->mc, c.x, c.g, c.ld, c.P, h->d_status};
-      LSGD_CUDA(launch_matcomp_grad(a, static_cast<const int32_t*>(batch), h->d_acc64, h->stream));
+      const bool fuse = (c.flags & LSGD_FLAG_MATCOMP_FUSED_STEP) && !(c.flags & LSGD_FLAG_ALGORITHM1) && !c.v &&
+                        (h->t % c.tau) != 0;
+      LSGD_CUDA(launch_matcomp_grad(a, static_cast<const int32_t*>(batch), h->d_acc64, !fuse, h->stream));
+      h->mc_step_pending = fuse;
       break;
     }
     case LSGD_OBJ_PSD_COMPLETION:
@@ -430,6 +435,9 @@ extern "C" lsgd_status lsgd_step(lsgd_handle h) {
       b.d = ranges[r][1];
       LSGD_CUDA(launch_update(b, h->stream));
     }
+  } else if (h->mc_step_pending) {
+    // plain step straight from the fixed-point gradient sums (only the entries the batch touched move)
+    LSGD_CUDA(launch_matcomp_finish_step(h->d_acc64, c.x, c.P, c.ld, (double)c.eta, (int)c.arithmetic, h->stream));
   } else if (a.v) {
     LSGD_CUDA(launch_momentum_update(a, h->stream));
   } else {
@@ -438,6 +446,7 @@ extern "C" lsgd_status lsgd_step(lsgd_handle h) {
   h->t++;
   h->loss_partials_valid = false;
   h->fused_applied = false;
+  h->mc_step_pending = false;
   h->grad_ready = false;
   h->armed_noise = nullptr;
   return LSGD_OK;

@@ -238,6 +238,34 @@ def test_matcomp_small_with_duplicates():
     pop.close()
 
 
+@pytest.mark.parametrize("rank", [3, 10, 20])
+def test_matcomp_fused_step_is_bit_identical_to_the_materialised_gradient_path(rank):
+    """With LSGD_FLAG_MATCOMP_FUSED_STEP a plain step is taken straight from the fixed-point gradient sums
+    (g is not written): same x, bit for bit, as gradient kernel + update kernel, and within tolerance of the
+    oracle.  Ranks on all three lane-group widths of the sparse kernels."""
+    from paper_1905_10395_b200 import api
+    w = inputs.make_matcomp(6, 2, n_rows=257, n_cols=190, rank=rank, n_obs=6000, n_heldout=1500, batch=900,
+                            steps=9, tau=4, config_id=54)
+    a = _pop(w, flags=api.FLAG_MATCOMP_FUSED_STEP)
+    b = _pop(w)
+    a.run(9, record=True)
+    b.run(9, record=True)
+    assert np.array_equal(a.x_host().view(np.uint32), b.x_host().view(np.uint32))
+    o = _oracle(w)
+    o.run(9)
+    _leaders_equal(a, o)
+    assert rel_err(a.x_host(), o.x) <= TOL
+    # protocol: a second gradient while the sums of the first wait for lsgd_step is refused (t = 9: not a pull step)
+    a.lsgd.grad(a.batches[9 % len(a.batches)])
+    with pytest.raises(api.LsgdError) as e:
+        a.lsgd.grad(a.batches[9 % len(a.batches)])
+    assert e.value.status == api.ERR_STATE
+    a.lsgd.step()
+    assert a.lsgd.check_device() == 0
+    a.close()
+    b.close()
+
+
 def test_config2_matrix_completion():
     w = inputs.config(2, steps=10)
     pop = _pop(w)
