@@ -523,6 +523,77 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------- groups sharded over ranks (optional mode) ----
+def run_sharded(args):
+    """--sharded: the paper's own mapping, groups on ranks (paper_1905_10395_b200/sharded.py).  The C4 shape
+    (P = 16, G = 4; d = 2^22 unless --d is given, since every rank generates the whole seeded population on its
+    host) split by groups over the N ranks; per pull step the ranks exchange their best loss and the owner
+    broadcasts the global leader's row over NCCL.  Total work is fixed ("strong").  Not the default: the
+    default multi-GPU mode is independent replicas."""
+    import torch
+    from paper_1905_10395_b200 import api, inputs, sharded
+
+    rank, world, local = dist_env()
+    dev = torch.device("cuda", local if world > 1 else 0)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    api.lib()
+    P, G, d = 16, 4, args.d or (1 << 22)
+    tau = args.tau or 1
+    steps, warmup = args.steps, max(args.warmup, 3)
+    w = inputs.make_external(P, G, d, eta=0.01, lambda_l=0.1, lambda_g=0.05, tau=tau, steps=steps, config_id=4)
+    eng = sharded.CudaShardEngine(w, rank, world, device=str(dev), arithmetic=args.arith)
+
+    def one_step():
+        if world > 1:
+            sharded.distributed_step(eng)
+        else:
+            sharded.run_lockstep([eng], 1)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    for _ in range(warmup):
+        one_step()
+    sampler = ClockSampler(local if world > 1 else 0)
+    sampler.start()
+    barrier()
+    torch.cuda.synchronize(dev)
+    wall0 = time.time()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        one_step()
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    wall1 = time.time()
+    barrier()
+    clocks = sampler.stop(wall0, wall1)
+    elapsed_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+    if eng.lsgd.check_device() != 0:
+        raise SystemExit("device status word set during the bench")
+    if rank == 0:
+        n_pull = len([t for t in range(warmup, warmup + steps) if t % tau == 0])
+        line = {"metric": METRIC, "value": P * d * steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
+                "warmup": warmup, "ms_per_step": elapsed_ms / steps, "higher_is_better": True, "scaling": "strong",
+                "vs_baseline": None, "dtype": "f64" if args.arith < 2 else "f32", "data": "synthetic",
+                "config": {"workload": f"C4 shape sharded by groups: P=16 G=4 d={d} over {world} rank(s)", "tau": tau,
+                           "multi_gpu": "groups on ranks; per pull step an all-gather of the ranks' best losses and a "
+                                        "broadcast of the global leader's row into every rank's own memory",
+                           "l2": "per-step inputs exceed the 126 MB L2" if P * d * 8 / world > 126e6 else "working set fits in L2"},
+                "clocks": clocks, "roofline": None, "e2e": None,
+                "gpu_launches": steps * 1 + n_pull * 1}
+        print(json.dumps(line), flush=True)
+    eng.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -544,11 +615,15 @@ def main():
     ap.add_argument("--momentum", type=float, default=None,
                     help="c4: Nesterov momentum of the Section 4.1 optimiser (adds the buffer v: 20 B per worker-param)")
     ap.add_argument("--weight-decay", type=float, default=0.0)
+    ap.add_argument("--sharded", action="store_true",
+                    help="groups sharded over the ranks with a leader broadcast per pull step (see run_sharded)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.sharded:
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -227,6 +227,15 @@ LSGD_API lsgd_status lsgd_destroy(lsgd_handle h);
 /* Accessors.  They synchronise the stream and are not part of the step.                          */
 LSGD_API lsgd_status lsgd_get_leaders(lsgd_handle h, int32_t* local_leaders /* HOST int32[G] */,
                              int32_t* global_leader /* HOST int32[1] */);
+/* Overrides the elected leaders (enqueued on the stream; the next pull step uses them).  local_leaders: HOST
+ * int32[G] with local_leaders[j] a member of group j, or NULL to keep the elected ones; global_leader: a worker
+ * index, or -1 to keep the elected one.  The global leader need not be one of the local leaders.  Uses: a
+ * population whose groups live on several devices (Section 2.2 maps a group to a node: the global leader may
+ * then be a row received from another device, see paper_1905_10395_b200/sharded.py), re-running a step with
+ * the leaders of a reference run when two losses are within rounding of each other, restoring a checkpoint.
+ * Counts as an election for the step protocol; the leader statistics are not changed.
+ * LSGD_ERR_BAD_GROUPS if an index is out of range or not in its group.                              */
+LSGD_API lsgd_status lsgd_set_leaders(lsgd_handle h, const int32_t* local_leaders, int32_t global_leader);
 LSGD_API lsgd_status lsgd_get_loss(lsgd_handle h, float* loss /* HOST float[P]: losses of the last election */);
 LSGD_API lsgd_status lsgd_get_step(lsgd_handle h, int64_t* t);
 /* Mean minibatch loss of every worker from the last lsgd_grad (MLP objective only; LSGD_ERR_UNSUPPORTED

@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
         L.lsgd_destroy.argtypes = [H]
         L.lsgd_get_leaders.argtypes = [H, C.c_void_p, C.c_void_p]
         L.lsgd_get_loss.argtypes = [H, C.c_void_p]
+        L.lsgd_set_leaders.argtypes = [H, C.c_void_p, C.c_int32]
+        L.lsgd_set_leaders.restype = C.c_int
         L.lsgd_get_train_loss.argtypes = [H, C.c_void_p]
         L.lsgd_get_train_loss.restype = C.c_int
         L.lsgd_center.argtypes = [H, C.c_void_p]
@@ -228,6 +230,11 @@ class Lsgd:
         gl = np.empty(1, dtype=np.int32)
         _check(lib().lsgd_get_leaders(self.h, ll.ctypes.data, gl.ctypes.data), "lsgd_get_leaders")
         return ll, int(gl[0])
+
+    def set_leaders(self, local_leaders=None, global_leader: int = -1):
+        ll = None if local_leaders is None else np.ascontiguousarray(local_leaders, dtype=np.int32)
+        _check(lib().lsgd_set_leaders(self.h, None if ll is None else ll.ctypes.data, int(global_leader)),
+               "lsgd_set_leaders")
 
     def loss(self):
         out = np.empty(self.P, dtype=np.float32)

@@ -473,6 +473,23 @@ lsgd_status lsgd_get_leaders(lsgd_handle h, int32_t* local_leaders, int32_t* glo
   return LSGD_OK;
 }
 
+lsgd_status lsgd_set_leaders(lsgd_handle h, const int32_t* local_leaders, int32_t global_leader) {
+  if (!h) return LSGD_ERR_INVALID_ARG;
+  const lsgd_config& c = h->cfg;
+  if (global_leader < -1 || global_leader >= c.P) return LSGD_ERR_BAD_GROUPS;
+  if (local_leaders)
+    for (int j = 0; j < c.G; ++j)
+      if (local_leaders[j] < 0 || local_leaders[j] >= c.P || h->group_of[local_leaders[j]] != j) return LSGD_ERR_BAD_GROUPS;
+  if ((!local_leaders || global_leader < 0) && h->n_elections == 0) return LSGD_ERR_STATE;   // nothing to keep yet
+  // pageable host memory: the copies are staged before the calls return, so the caller's array may go away
+  if (local_leaders)
+    LSGD_CUDA(cudaMemcpyAsync(h->d_ll, local_leaders, sizeof(int32_t) * c.G, cudaMemcpyHostToDevice, h->stream));
+  if (global_leader >= 0)
+    LSGD_CUDA(cudaMemcpyAsync(h->d_gl, &global_leader, sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+  h->n_elections++;
+  return LSGD_OK;
+}
+
 lsgd_status lsgd_get_loss(lsgd_handle h, float* loss) {
   if (!h || !loss) return LSGD_ERR_INVALID_ARG;
   LSGD_CUDA(cudaStreamSynchronize(h->stream));
