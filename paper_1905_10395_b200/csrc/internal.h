@@ -62,6 +62,7 @@ struct UpdateArgs {
 cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s);
 // Section 4.1 optimiser (a.v != nullptr): Nesterov momentum + weight decay around the same step.
 cudaError_t launch_momentum_update(const UpdateArgs& a, cudaStream_t s);
+cudaError_t launch_momentum_update_chunked(const UpdateArgs& a, cudaStream_t s);   // cudaErrorNotSupported: shape does not fit
 cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, int64_t ld, cudaStream_t s);
 
 struct ElectArgs {

@@ -179,6 +179,9 @@ cudaError_t launch_m(const UpdateArgs& a, cudaStream_t s) {
 
 cudaError_t launch_momentum_update(const UpdateArgs& a, cudaStream_t s) {
   if (!a.v || !a.g || a.snap || !a.use_g) return cudaErrorInvalidValue;
+  // first choice: the chunked staged pipeline of update.cu with the momentum buffer as a third row per worker
+  const cudaError_t e = launch_momentum_update_chunked(a, s);
+  if (e != cudaErrorNotSupported) return e;
   switch (a.arith) {
     case 0: return launch_m<0>(a, s);
     case 1: return launch_m<1>(a, s);

@@ -162,6 +162,47 @@ __device__ __forceinline__ float pull1_t(typename Eval<MODE>::T X, float g, type
   }
 }
 
+// The step with the Section 4.1 optimiser around it (the formulas of momentum.cu, same operation order):
+//   d = g + wd x,  v+ = mu v + d,  u = d + mu v+,  x+ = x - eta u [- pulls].
+template <int MODE, bool PULL>
+__device__ __forceinline__ void momentum1_t(typename Eval<MODE>::T X, float g, float v, typename Eval<MODE>::T XL,
+                                            typename Eval<MODE>::T XG, const Coef& k, float& x_new, float& v_new) {
+  if (MODE == 0) {
+    const double D = __dadd_rn((double)g, __dmul_rn(k.wd, (double)X));
+    const double VN = __dadd_rn(__dmul_rn(k.mu, (double)v), D);
+    const double U = __dadd_rn(D, __dmul_rn(k.mu, VN));
+    double acc = __dsub_rn((double)X, __dmul_rn(k.eta, U));
+    if (PULL) {
+      acc = __dsub_rn(acc, __dmul_rn(k.cl, __dsub_rn((double)X, (double)XL)));
+      acc = __dsub_rn(acc, __dmul_rn(k.cg, __dsub_rn((double)X, (double)XG)));
+    }
+    x_new = (float)acc;
+    v_new = (float)VN;
+  } else if (MODE == 1) {
+    const double D = fma(k.wd, (double)X, (double)g);
+    const double VN = fma(k.mu, (double)v, D);
+    const double U = fma(k.mu, VN, D);
+    double acc = fma(-k.eta, U, (double)X);
+    if (PULL) {
+      acc = fma(-k.cl, (double)X - (double)XL, acc);
+      acc = fma(-k.cg, (double)X - (double)XG, acc);
+    }
+    x_new = (float)acc;
+    v_new = (float)VN;
+  } else {
+    const float D = fmaf(k.wd_f, (float)X, g);
+    const float VN = fmaf(k.mu_f, v, D);
+    const float U = fmaf(k.mu_f, VN, D);
+    float acc = fmaf(-k.eta_f, U, (float)X);
+    if (PULL) {
+      acc = fmaf(-k.cl_f, (float)X - (float)XL, acc);
+      acc = fmaf(-k.cg_f, (float)X - (float)XG, acc);
+    }
+    x_new = acc;
+    v_new = VN;
+  }
+}
+
 template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
 __global__ void __launch_bounds__(kThreads, LSGD_K1_PULL_MIN_BLOCKS)
 pull_update_kernel(UpdateArgs p, int64_t n4) {
@@ -520,6 +561,9 @@ inline int staged_tile_width(const UpdateArgs& a) {
 #ifndef LSGD_K1_CHUNK_SHAPES
 #define LSGD_K1_CHUNK_SHAPES {768, 8, 3}, {768, 8, 2}, {768, 4, 3}, {768, 4, 2}, {512, 12, 2}, {512, 6, 3}, {512, 6, 2}
 #endif
+#ifndef LSGD_K1_MOM_SHAPES
+#define LSGD_K1_MOM_SHAPES {768, 8, 2}, {768, 4, 3}, {768, 4, 2}, {512, 12, 2}, {512, 6, 3}, {512, 6, 2}
+#endif
 constexpr int kChunkMaxStages = 4;
 constexpr int kChunkSmemBudget = 224 * 1024;
 
@@ -528,7 +572,7 @@ struct ChunkShape {
   size_t smem;
 };
 
-template <int MODE, bool PULL, bool QUAD, bool NOISE, bool SHADOW>
+template <int MODE, bool PULL, bool QUAD, bool NOISE, bool SHADOW, bool MOM>
 __global__ void __launch_bounds__(kTmaThreads, 1)
 update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
   extern __shared__ __align__(128) uint8_t s_raw[];
@@ -539,7 +583,7 @@ update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
   const bool has_g = (QUAD ? NOISE : true) && p.use_g;      // a pure pull drops the gradient term
   const int pull_slots = PULL ? G + 1 : 0;                  // slots 0..G-1: local leaders, slot G: global leader
   const int nlead = pull_slots + (QUAD ? 2 : 0);            // then a, b
-  const int stage_rows = R * (has_g ? 2 : 1);
+  const int stage_rows = R * ((has_g ? 2 : 1) + (MOM ? 1 : 0));   // per worker: x, g / noise, momentum buffer
   float* lead0 = reinterpret_cast<float*>(s_raw);                                   // [2][nlead][W]
   float* ring0 = lead0 + (size_t)2 * nlead * W;                                     // [S][stage_rows][W]
   int32_t* s_lead = reinterpret_cast<int32_t*>(ring0 + (size_t)S * stage_rows * W); // [P] slot of worker i's local leader
@@ -636,7 +680,7 @@ update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
         float* sx = ring0 + (size_t)s * stage_rows * W;
         // rows q < nr: worker (i0 + q)'s x unless it sits in the leader block; rows R + q: its g / noise
         int mine = 0;
-        for (int q = lane; q < nr; q += 32) mine += (s_self[i0 + q] ? 0 : 1) + (has_g ? 1 : 0);
+        for (int q = lane; q < nr; q += 32) mine += (s_self[i0 + q] ? 0 : 1) + (has_g ? 1 : 0) + (MOM ? 1 : 0);
         const int n_copies = __reduce_add_sync(0xFFFFFFFFu, mine);
         if (lane == 0)
           asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&full_bar[s])), "r"(bytes * (uint32_t)n_copies) : "memory");
@@ -649,6 +693,9 @@ update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
           if (has_g)
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                          ::"r"(smem_addr(sx + (size_t)(R + q) * W)), "l"(gsrc + (int64_t)i * p.ld + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
+          if (MOM)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(sx + (size_t)(2 * R + q) * W)), "l"(p.v + (int64_t)i * p.ld + c0), "r"(bytes), "r"(smem_addr(&full_bar[s])) : "memory");
         }
       }
     }
@@ -727,13 +774,22 @@ update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
             }
             const float4 gv = has_g ? *reinterpret_cast<const float4*>(sg + (size_t)q * W) : make_float4(0.f, 0.f, 0.f, 0.f);
             float g[4] = {gv.x, gv.y, gv.z, gv.w}, r[4];
+            const int64_t off = (int64_t)i * p.ld + c0 + c4 * 4;
+            if (MOM) {
+              const float4 vv = *reinterpret_cast<const float4*>(sx + (size_t)(2 * R + q) * W);
+              const float vo[4] = {vv.x, vv.y, vv.z, vv.w};
+              float vn[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              if (QUAD && p.use_g) g[e] = quad_g_t<MODE>(X[e], A[e], B[e], g[e], k, NOISE);
-              r[e] = PULL ? pull1_t<MODE>(X[e], g[e], XL[e], XG[e], k) : plain1_t<MODE>(X[e], g[e], k);
+              for (int e = 0; e < 4; ++e) momentum1_t<MODE, PULL>(X[e], g[e], vo[e], XL[e], XG[e], k, r[e], vn[e]);
+              st4(p.v + off, make_float4(vn[0], vn[1], vn[2], vn[3]));
+            } else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                if (QUAD && p.use_g) g[e] = quad_g_t<MODE>(X[e], A[e], B[e], g[e], k, NOISE);
+                r[e] = PULL ? pull1_t<MODE>(X[e], g[e], XL[e], XG[e], k) : plain1_t<MODE>(X[e], g[e], k);
+              }
             }
             const float4 rv = make_float4(r[0], r[1], r[2], r[3]);
-            const int64_t off = (int64_t)i * p.ld + c0 + c4 * 4;
             st4(p.x + off, rv);
             if (SHADOW) st4_bf16(p.x_bf16 + off, rv);
           }
@@ -749,34 +805,40 @@ update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
 }
 
 // Shape for the chunked kernel: the widest tile and deepest ring whose leader block (twice) and ring fit.
-inline ChunkShape chunk_shape(const UpdateArgs& a, bool quad, bool noise) {
+inline ChunkShape chunk_shape(const UpdateArgs& a, bool quad, bool noise, bool mom = false) {
   ChunkShape none{0, 0, 0, 0};
-  if (!a.pull && !quad) return none;
+  if (!a.pull && !quad && !mom) return none;
   const bool has_g = (quad ? noise : true) && a.use_g;
   if (!quad && a.use_g && a.g == nullptr) return none;
   const int nlead = (a.pull ? a.G + 1 : 0) + (quad ? 2 : 0);
-  static const int shapes[][3] = {LSGD_K1_CHUNK_SHAPES};
-  for (const auto& sh : shapes) {
+  // the momentum step streams three rows per worker over very long rows: two deep stages beat three there
+  static const int shapes_plain[][3] = {LSGD_K1_CHUNK_SHAPES};
+  static const int shapes_mom[][3] = {LSGD_K1_MOM_SHAPES};
+  const int (*shapes)[3] = mom ? shapes_mom : shapes_plain;
+  const int n_shapes = mom ? (int)(sizeof(shapes_mom) / sizeof(shapes_mom[0])) : (int)(sizeof(shapes_plain) / sizeof(shapes_plain[0]));
+  for (int q = 0; q < n_shapes; ++q) {
+    const int* sh = shapes[q];
     const int W = sh[0], R = sh[1], S = sh[2];
     if (S > kChunkMaxStages || (kTmaConsumers % (W / 4)) != 0) continue;
-    const size_t bytes = ((size_t)2 * nlead + (size_t)S * R * (has_g ? 2 : 1)) * W * 4 + (size_t)(2 * a.P + a.G + 1) * 4;
+    const size_t bytes = ((size_t)2 * nlead + (size_t)S * R * ((has_g ? 2 : 1) + (mom ? 1 : 0))) * W * 4 +
+                         (size_t)(2 * a.P + a.G + 1) * 4;
     if (bytes <= (size_t)kChunkSmemBudget) return ChunkShape{W, R, S, bytes};
   }
   return none;
 }
 
-template <int MODE, bool PULL, bool QUAD, bool NOISE, bool SHADOW>
+template <int MODE, bool PULL, bool QUAD, bool NOISE, bool SHADOW, bool MOM = false>
 cudaError_t launch_chunked(const UpdateArgs& a, const ChunkShape& cs, int64_t n4, int sms, cudaStream_t s) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW>,
+    cudaError_t e = cudaFuncSetAttribute(update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW, MOM>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kChunkSmemBudget);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
   const int64_t tiles = (n4 * 4 + cs.W - 1) / cs.W;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-  update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW><<<grid, kTmaThreads, cs.smem, s>>>(a, n4, cs.W, cs.R, cs.S);
+  update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW, MOM><<<grid, kTmaThreads, cs.smem, s>>>(a, n4, cs.W, cs.R, cs.S);
   return cudaGetLastError();
 }
 
@@ -867,6 +929,35 @@ cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, i
   if (blocks > 148 * 16) blocks = 148 * 16;
   center_kernel<<<(unsigned)blocks, 256, 0, s>>>(x, center, P, n4, ld);
   return cudaGetLastError();
+}
+
+namespace {
+template <int MODE>
+cudaError_t launch_momentum_chunked_m(const UpdateArgs& a, const ChunkShape& cs, cudaStream_t s) {
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (sms <= 0) sms = 148;
+  const int64_t n4 = (a.d + 3) / 4;
+  const bool shadow = a.x_bf16 != nullptr;
+  if (a.pull) return shadow ? launch_chunked<MODE, true, false, false, true, true>(a, cs, n4, sms, s)
+                            : launch_chunked<MODE, true, false, false, false, true>(a, cs, n4, sms, s);
+  return shadow ? launch_chunked<MODE, false, false, false, true, true>(a, cs, n4, sms, s)
+                : launch_chunked<MODE, false, false, false, false, true>(a, cs, n4, sms, s);
+}
+}  // namespace
+
+// The momentum step through the chunked staged pipeline (x, g and v rows in the ring).  cudaErrorNotSupported
+// when the shape does not fit: the caller then uses the register-staged momentum kernel.
+cudaError_t launch_momentum_update_chunked(const UpdateArgs& a, cudaStream_t s) {
+  if (LSGD_K1_NO_STAGED || !a.v || !a.g || a.snap || !a.use_g) return cudaErrorNotSupported;
+  const ChunkShape cs = chunk_shape(a, false, false, true);
+  if (cs.W == 0) return cudaErrorNotSupported;
+  switch (a.arith) {
+    case 0: return launch_momentum_chunked_m<0>(a, cs, s);
+    case 1: return launch_momentum_chunked_m<1>(a, cs, s);
+    default: return launch_momentum_chunked_m<2>(a, cs, s);
+  }
 }
 
 cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s) {
