@@ -39,6 +39,24 @@ def test_populations_streamed_in_chunks(P, G, d):
     _check(w, 5)
 
 
+@pytest.mark.parametrize("P,G,d", [(1, 1, 1), (3, 3, 5), (9, 2, 769), (70, 7, 1537)])
+def test_fused_quadratic_degenerate_shapes(P, G, d):
+    # the inline-gradient forms of the chunked kernel: one worker, every worker its own group, d below one
+    # 16-byte column, one column past a tile, a ragged last chunk of workers
+    w = inputs.make_quadratic(P, G, d, eta=0.05, lambda_l=0.1, lambda_g=0.05, tau=2, steps=5, noise_ring=3, config_id=116)
+    from paper_1905_10395_b200.runner import Population
+    pop = Population(w, fused_quadratic=True)
+    pop.run(5, record=True)
+    o = orc.LsgdOracle(w.x0, orc.Quadratic(w.arrays["a"], w.arrays["b"], w.meta["sigma"], w.arrays["noise"]), w.group_of,
+                       w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
+    o.run(5)
+    for hg, ho in zip(pop.history, o.history):
+        assert hg["gl"] == ho["gl"] and np.array_equal(hg["ll"], ho["ll"])
+    assert np.array_equal(pop.x_host().view(np.uint32), o.x.view(np.uint32))
+    assert pop.lsgd.check_device() == 0
+    pop.close()
+
+
 def test_single_worker_is_plain_sgd():
     w = inputs.make_external(1, 1, 257, eta=0.05, lambda_l=0.3, lambda_g=0.2, tau=1, steps=4, config_id=111)
     from paper_1905_10395_b200.runner import Population

@@ -63,6 +63,25 @@ def test_quadratic_with_noise_bit_exact_and_single_worker():
         pop.close()
 
 
+@pytest.mark.parametrize("P,G,d", [(1, 1, 3), (20, 4, 2311), (64, 8, 148 * 768 + 8), (150, 75, 260)])
+def test_momentum_shapes_on_both_kernels(P, G, d):
+    # one worker and d below a 16-byte column; a ragged last chunk of workers; more tiles than CTAs with a ragged
+    # last tile; and so many groups that the leader block does not fit (register-staged fallback kernel)
+    w = inputs.make_external(P, G, d, eta=0.05, lambda_l=0.1, lambda_g=0.05, tau=2, steps=5, loss_ring=3, config_id=96)
+    from paper_1905_10395_b200.runner import Population
+    pop = Population(w, momentum=0.9, weight_decay=1e-4)
+    pop.run(5, record=True)
+    o = orc.LsgdOracle(w.x0, orc.External(w.arrays["g"], w.arrays["loss_ring"]), w.group_of, w.G, w.eta, w.lambda_l,
+                       w.lambda_g, w.tau, momentum=0.9, weight_decay=1e-4)
+    o.run(5)
+    for hg, ho in zip(pop.history, o.history):
+        assert hg["gl"] == ho["gl"] and np.array_equal(hg["ll"], ho["ll"])
+    assert np.array_equal(pop.x_host().view(np.uint32), o.x.view(np.uint32))
+    assert np.array_equal(pop.v.cpu().numpy().view(np.uint32), o.v.view(np.uint32))
+    assert pop.lsgd.check_device() == 0
+    pop.close()
+
+
 def test_zero_momentum_and_decay_equals_the_plain_path():
     w = inputs.make_external(5, 2, 9000, eta=0.05, lambda_l=0.1, lambda_g=0.05, tau=2, steps=6, loss_ring=3,
                              config_id=54)
