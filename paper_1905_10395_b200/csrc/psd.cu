@@ -20,9 +20,11 @@ namespace {
 constexpr int T = 64;            // tile edge
 constexpr int TH = 16;           // threads per tile edge
 constexpr int MT = T / TH;       // micro-tile edge (4)
-constexpr int kMaxRank = 128;
-constexpr int KM = kMaxRank / TH;  // output columns per thread (8)
 
+// KM = output columns of G per thread = ceil(r / 16) rounded up to 1, 2, 4 or 8: a compile-time bound, so a
+// small rank neither issues the fp64 operations of absent columns (predicated off, they still occupy the pipe:
+// at r = 10 they were seven eighths of its work) nor holds their accumulators in registers.
+template <int KM>
 __global__ void __launch_bounds__(TH * TH)
 psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float* __restrict__ M, int32_t n, int32_t r,
                 int64_t ld, double* __restrict__ partials, int32_t n_partials, int write_g) {
@@ -44,12 +46,40 @@ psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float*
 #pragma unroll
     for (int m = 0; m < KM; ++m) acc[a][m] = 0.0;
   double lsum = 0.0;
-  for (int J0 = 0; J0 < n; J0 += T) {
-    for (int idx = tid; idx < T * r; idx += TH * TH) {
+  // The next block's operands -- this thread's 16 entries of M and its share of X_J -- are fetched into
+  // registers while the current block is being worked on, so their latency is off the critical path.
+  constexpr int NX = (T * 16 * KM + TH * TH - 1) / (TH * TH);   // X_J values per thread (r <= 16 KM)
+  float m_next[MT][MT], xj_next[NX];
+  auto fetch = [&](int J0) {
+#pragma unroll
+    for (int a = 0; a < MT; ++a)
+#pragma unroll
+      for (int b = 0; b < MT; ++b) {
+        const int ri = I0 + ty + TH * a, cj = J0 + tx + TH * b;
+        m_next[a][b] = (ri < n && cj < n) ? M[(int64_t)ri * n + cj] : 0.f;
+      }
+#pragma unroll
+    for (int q = 0; q < NX; ++q) {
+      const int idx = tid + q * TH * TH;
       const int row = idx / r, k = idx - row * r;
-      XJ[row * pitch + k] = (J0 + row < n) ? (double)xi[(int64_t)(J0 + row) * r + k] : 0.0;
+      xj_next[q] = (idx < T * r && J0 + row < n) ? xi[(int64_t)(J0 + row) * r + k] : 0.f;
+    }
+  };
+  fetch(0);
+  for (int J0 = 0; J0 < n; J0 += T) {
+    float m_cur[MT][MT];
+#pragma unroll
+    for (int a = 0; a < MT; ++a)
+#pragma unroll
+      for (int b = 0; b < MT; ++b) m_cur[a][b] = m_next[a][b];
+#pragma unroll
+    for (int q = 0; q < NX; ++q) {
+      const int idx = tid + q * TH * TH;
+      const int row = idx / r, k = idx - row * r;
+      if (idx < T * r) XJ[row * pitch + k] = (double)xj_next[q];
     }
     __syncthreads();
+    if (J0 + T < n) fetch(J0 + T);
     // R micro-tile: rows ty + 16 a, columns tx + 16 b
     double s[MT][MT];
 #pragma unroll
@@ -72,7 +102,7 @@ psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float*
 #pragma unroll
       for (int b = 0; b < MT; ++b) {
         const int ri = I0 + ty + TH * a, cj = J0 + tx + TH * b;
-        const double rab = (ri < n && cj < n) ? s[a][b] - (double)M[(int64_t)ri * n + cj] : 0.0;
+        const double rab = (ri < n && cj < n) ? s[a][b] - (double)m_cur[a][b] : 0.0;
         lsum = fma(rab, rab, lsum);
         Rt[(ty + TH * a) * (T + 1) + tx + TH * b] = rab;
       }
@@ -131,12 +161,19 @@ cudaError_t launch_psd_grad(const float* x, float* g, const float* M, int32_t n,
   const size_t smem = sizeof(double) * (size_t)(2 * T * pitch + T * (T + 1));
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(psd_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(psd_grad_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(psd_grad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(psd_grad_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(psd_grad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   dim3 grid((unsigned)n_partials, (unsigned)P), block(TH, TH);
-  psd_grad_kernel<<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, write_g ? 1 : 0);
+  const int wg = write_g ? 1 : 0;
+  if (r <= 16) psd_grad_kernel<1><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg);
+  else if (r <= 32) psd_grad_kernel<2><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg);
+  else if (r <= 64) psd_grad_kernel<4><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg);
+  else psd_grad_kernel<8><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg);
   return cudaGetLastError();
 }
 
