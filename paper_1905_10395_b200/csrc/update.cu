@@ -1,7 +1,16 @@
 // Fused LSGD update (Eq. (1) with eta-scaled pulls, Section 3.1.1) and the plain (S)GD step used
 // between communications (Section 3.1.2).
 //
-// Pull form.  A thread owns one 16-byte column (4 consecutive parameters) for ALL P workers.  It
+// Ownership rule of every form below: a CTA owns a column tile for ALL P workers, so whoever reads a leader's
+// values does so before anyone rewrites them, and every right-hand side is x at time t although x is updated
+// in place.  Three realisations, chosen in launch_t() / launch_momentum_update_chunked():
+//   staged   (pull_update_staged_kernel): all rows of a 3 KiB-wide tile brought into shared memory by bulk
+//            copies, for populations small enough that they fit twice (P <= 26);
+//   chunked  (update_chunked_kernel): a leader block, then the rows streamed through a ring of chunks of 8
+//            workers -- any P whose leader block fits, the inline quadratic gradient, the momentum step;
+//   register-staged (pull_update_kernel, described next): the fallback for everything else.
+//
+// Register-staged pull form.  A thread owns one 16-byte column (4 consecutive parameters) for ALL P workers.  It
 // reads the global leader's 4 values once, then walks the workers group by group: the group's local
 // leader is read once into registers, after which each member row is read, updated and written.
 // A leader row is taken from the registers it was staged in instead of being read again, so every
