@@ -34,6 +34,8 @@ __device__ __forceinline__ unsigned long long warp_min(unsigned long long k) {
 }
 
 __global__ void __launch_bounds__(kElectThreads) elect_kernel(ElectArgs p) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   if (p.partials != nullptr) {
     for (int i = warp; i < p.P; i += nwarps) {
@@ -105,8 +107,7 @@ cudaError_t launch_leader_copies(const float* x, float* copies, const int32_t* l
 }
 
 cudaError_t launch_elect(const ElectArgs& a, cudaStream_t s) {
-  elect_kernel<<<1, kElectThreads, 0, s>>>(a);
-  return cudaGetLastError();
+  return launch_pdl(elect_kernel, dim3(1), dim3(kElectThreads), 0, s, a);
 }
 
 }  // namespace lsgd

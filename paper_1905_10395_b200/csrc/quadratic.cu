@@ -64,6 +64,8 @@ __device__ __forceinline__ double term(double x, double a, double b) {
 __global__ void __launch_bounds__(kThreads)
 quadratic_loss_kernel(const float* __restrict__ x, const float* __restrict__ a, const float* __restrict__ b, int32_t P,
                       int64_t d, int64_t ld, double* __restrict__ partials, int32_t n_partials) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int i0 = blockIdx.y * kLossRows;
   const int rows = min(kLossRows, P - i0);
   const int64_t c0 = (int64_t)blockIdx.x * kChunkCols;
@@ -130,8 +132,7 @@ int32_t quadratic_loss_blocks(int64_t d) { return (int32_t)((d + kChunkCols - 1)
 cudaError_t launch_quadratic_loss_partials(const float* x, const float* a, const float* b, int32_t P, int64_t d,
                                            int64_t ld, double* partials, int32_t n_partials, cudaStream_t s) {
   dim3 grid((unsigned)n_partials, (unsigned)((P + kLossRows - 1) / kLossRows));
-  quadratic_loss_kernel<<<grid, kThreads, 0, s>>>(x, a, b, P, d, ld, partials, n_partials);
-  return cudaGetLastError();
+  return launch_pdl(quadratic_loss_kernel, grid, dim3(kThreads), 0, s, x, a, b, P, d, ld, partials, n_partials);
 }
 
 }  // namespace lsgd

@@ -429,6 +429,8 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatil
 template <int MODE, bool SHADOW>
 __global__ void __launch_bounds__(kTmaThreads, 1)
 pull_update_staged_kernel(UpdateArgs p, int64_t n_cols4, int W) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ __align__(128) uint8_t s_raw[];
   __shared__ uint64_t full_bar[kTmaStages], empty_bar[kTmaStages];
   __shared__ int s_abort, s_bad, s_gl;
@@ -584,6 +586,8 @@ struct ChunkShape {
 template <int MODE, bool PULL, bool QUAD, bool NOISE, bool SHADOW, bool MOM>
 __global__ void __launch_bounds__(kTmaThreads, 1)
 update_chunked_kernel(UpdateArgs p, int64_t n_cols4, int W, int R, int S) {
+  pdl_wait();                  // launched as a programmatic dependent: nothing is read before the earlier kernels end
+  pdl_launch_dependents();
   extern __shared__ __align__(128) uint8_t s_raw[];
   __shared__ uint64_t full_bar[kChunkMaxStages], empty_bar[kChunkMaxStages], lfull_bar[2], lempty_bar[2];
   __shared__ int s_abort, s_bad, s_gslot;
@@ -847,8 +851,8 @@ cudaError_t launch_chunked(const UpdateArgs& a, const ChunkShape& cs, int64_t n4
   }
   const int64_t tiles = (n4 * 4 + cs.W - 1) / cs.W;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-  update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW, MOM><<<grid, kTmaThreads, cs.smem, s>>>(a, n4, cs.W, cs.R, cs.S);
-  return cudaGetLastError();
+  return launch_pdl(update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW, MOM>, dim3(grid), dim3(kTmaThreads), cs.smem, s, a, n4,
+                    cs.W, cs.R, cs.S);
 }
 
 template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
@@ -874,7 +878,7 @@ cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
     const size_t smem = (size_t)kTmaStages * staged_rows(a) * W * 4 + (size_t)a.P * 4;
     const int64_t tiles = (n4 * 4 + W - 1) / (W > 0 ? W : 1);
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    pull_update_staged_kernel<MODE, SHADOW><<<grid, kTmaThreads, smem, s>>>(a, n4, W);
+    return launch_pdl(pull_update_staged_kernel<MODE, SHADOW>, dim3(grid), dim3(kTmaThreads), smem, s, a, n4, W);
   } else if (!LSGD_K1_NO_STAGED && (a.pull || (QUAD && !SHADOW)) && chunk_shape(a, QUAD, NOISE).W > 0) {
     const ChunkShape cs = chunk_shape(a, QUAD, NOISE);
     if (a.pull) return launch_chunked<MODE, true, QUAD, NOISE, SHADOW>(a, cs, n4, sms, s);
