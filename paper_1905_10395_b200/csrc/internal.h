@@ -115,9 +115,11 @@ cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials,
                                          cudaStream_t s);
 
 // Dense PSD completion objective.
-int32_t psd_loss_blocks(int32_t n);
+int32_t psd_split(int32_t r);                     // CTAs per row block (partial gradients to combine), 1 = none
+int32_t psd_loss_blocks(int32_t n, int32_t r);
+// gpart: DEVICE double[psd_split(r) * P * ld] scratch when psd_split(r) > 1, else unused
 cudaError_t launch_psd_grad(const float* x, float* g, const float* M, int32_t n, int32_t r, int32_t P, int64_t ld,
-                            double* partials, int32_t n_partials, bool write_g, cudaStream_t s);
+                            double* partials, int32_t n_partials, bool write_g, double* gpart, cudaStream_t s);
 
 // Programmatic dependent launch.  A kernel started with launch_pdl() may become resident, and run its
 // prologue (barrier and tensor-memory set-up, descriptor prefetch), while the kernel before it in the stream
@@ -187,4 +189,5 @@ struct lsgd_ctx {
   void* mlp_state;           // opaque MLP pipeline state
   unsigned long long* d_acc64;  // MATCOMP: fixed-point gradient accumulator [P*ld], kept all-zero between steps
   bool mc_step_pending;         // MATCOMP fused step: the gradient sums wait in d_acc64 for lsgd_step
+  double* d_psd_part;           // PSD, small ranks: partial gradients of the CTAs that share a row block
 };

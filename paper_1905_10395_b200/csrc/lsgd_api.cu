@@ -123,6 +123,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->slab = nullptr;
   h->mlp_state = nullptr;
   h->d_acc64 = nullptr;
+  h->d_psd_part = nullptr;
   std::memset(&h->quad, 0, sizeof(h->quad));
   std::memset(&h->mc, 0, sizeof(h->mc));
   std::memset(&h->mlp, 0, sizeof(h->mlp));
@@ -139,7 +140,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
     h->mlp = *static_cast<const lsgd_mlp_desc*>(cfg->objective_desc);
   } else if (cfg->objective == LSGD_OBJ_PSD_COMPLETION) {
     h->psd = *static_cast<const lsgd_psd_desc*>(cfg->objective_desc);
-    h->n_partials = psd_loss_blocks(h->psd.n);
+    h->n_partials = psd_loss_blocks(h->psd.n, h->psd.r);
   }
   h->cfg.objective_desc = nullptr;
 
@@ -196,12 +197,16 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
     ok = cudaMalloc(reinterpret_cast<void**>(&h->d_acc64), bytes) == cudaSuccess &&
          cudaMemsetAsync(h->d_acc64, 0, bytes, h->stream) == cudaSuccess;
   }
+  if (ok && cfg->objective == LSGD_OBJ_PSD_COMPLETION && psd_split(h->psd.r) > 1)
+    ok = cudaMalloc(reinterpret_cast<void**>(&h->d_psd_part),
+                    sizeof(double) * (size_t)psd_split(h->psd.r) * (size_t)P * (size_t)cfg->ld) == cudaSuccess;
   // the gradient kernel of this objective writes columns < d only: clear the padding of g once
   if (ok && cfg->objective == LSGD_OBJ_PSD_COMPLETION && cfg->ld > cfg->d)
     ok = cudaMemsetAsync(cfg->g, 0, sizeof(float) * (size_t)P * (size_t)cfg->ld, h->stream) == cudaSuccess;
   if (!ok) {
     if (h->mlp_state) mlp_destroy(h);
     cudaFree(h->d_acc64);
+    cudaFree(h->d_psd_part);
     cudaFree(h->slab);
     delete h;
     return LSGD_ERR_CUDA;
@@ -238,7 +243,7 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
     }
     case LSGD_OBJ_PSD_COMPLETION:
       LSGD_CUDA(launch_psd_grad(c.x, c.g, h->psd.M, h->psd.n, h->psd.r, c.P, c.ld, h->d_partials, h->n_partials, true,
-                                h->stream));
+                                h->d_psd_part, h->stream));
       h->loss_partials_valid = true;
       break;
     case LSGD_OBJ_MLP: {
@@ -304,7 +309,7 @@ lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
       case LSGD_OBJ_PSD_COMPLETION:
         if (!h->loss_partials_valid)   // otherwise lsgd_grad has just summed F at this x
           LSGD_CUDA(launch_psd_grad(c.x, c.g, h->psd.M, h->psd.n, h->psd.r, c.P, c.ld, h->d_partials, h->n_partials,
-                                    false, h->stream));
+                                    false, h->d_psd_part, h->stream));
         h->loss_partials_valid = true;
         e.partials = h->d_partials;
         e.n_partials = h->n_partials;
@@ -459,6 +464,7 @@ lsgd_status lsgd_destroy(lsgd_handle h) {
   cudaStreamSynchronize(h->stream);
   if (h->mlp_state) mlp_destroy(h);
   cudaFree(h->d_acc64);
+  cudaFree(h->d_psd_part);
   cudaError_t e = cudaFree(h->slab);
   delete h;
   return e == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;

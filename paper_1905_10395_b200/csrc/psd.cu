@@ -24,10 +24,14 @@ constexpr int MT = T / TH;       // micro-tile edge (4)
 // KM = output columns of G per thread = ceil(r / 16) rounded up to 1, 2, 4 or 8: a compile-time bound, so a
 // small rank neither issues the fp64 operations of absent columns (predicated off, they still occupy the pipe:
 // at r = 10 they were seven eighths of its work) nor holds their accumulators in registers.
-template <int KM>
-__global__ void __launch_bounds__(TH * TH)
+// Z = CTAs that share one row block (gridDim.z): CTA z takes the column blocks z, z + Z, ...  At small rank the
+// time is the dependent chain over the column blocks, which only a shorter chain shortens; the Z partial
+// gradients go to gpart[z][P][ld] in fp64 and psd_combine_kernel adds them in z order.  Z = 1 writes g itself.
+template <int KM, int Z>
+__global__ void __launch_bounds__(TH * TH, Z > 1 ? 2 : 1)
 psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float* __restrict__ M, int32_t n, int32_t r,
-                int64_t ld, double* __restrict__ partials, int32_t n_partials, int write_g) {
+                int64_t ld, double* __restrict__ partials, int32_t n_partials, int write_g, double* __restrict__ gpart,
+                int32_t P) {
   extern __shared__ double s_psd[];
   const int pitch = r | 1;                      // odd pitch: conflict-free column walks
   double* XI = s_psd;                           // [T][pitch]
@@ -65,8 +69,9 @@ psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float*
       xj_next[q] = (idx < T * r && J0 + row < n) ? xi[(int64_t)(J0 + row) * r + k] : 0.f;
     }
   };
-  fetch(0);
-  for (int J0 = 0; J0 < n; J0 += T) {
+  const int Jstep = T * Z;
+  fetch((int)blockIdx.z * T);
+  for (int J0 = (int)blockIdx.z * T; J0 < n; J0 += Jstep) {
     float m_cur[MT][MT];
 #pragma unroll
     for (int a = 0; a < MT; ++a)
@@ -79,7 +84,7 @@ psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float*
       if (idx < T * r) XJ[row * pitch + k] = (double)xj_next[q];
     }
     __syncthreads();
-    if (J0 + T < n) fetch(J0 + T);
+    if (J0 + Jstep < n) fetch(J0 + Jstep);
     // R micro-tile: rows ty + 16 a, columns tx + 16 b
     double s[MT][MT];
 #pragma unroll
@@ -129,11 +134,14 @@ psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float*
     for (int a = 0; a < MT; ++a) {
       const int ri = I0 + ty + TH * a;
       if (ri < n) {
-        float* gi = g + (int64_t)i * ld + (int64_t)ri * r;
+        const int64_t row = (int64_t)i * ld + (int64_t)ri * r;
 #pragma unroll
         for (int m = 0; m < KM; ++m) {
           const int k = tx + TH * m;
-          if (k < r) gi[k] = (float)acc[a][m];
+          if (k < r) {
+            if (Z == 1) g[row + k] = (float)acc[a][m];
+            else gpart[((int64_t)blockIdx.z * P) * ld + row + k] = acc[a][m];
+          }
         }
       }
     }
@@ -147,34 +155,67 @@ psd_grad_kernel(const float* __restrict__ x, float* __restrict__ g, const float*
   if (tid == 0) {
     double t = 0.0;
     for (int w = 0; w < TH * TH / 32; ++w) t += s_w[w];
-    partials[(int64_t)i * n_partials + blockIdx.x] = t;
+    partials[(int64_t)i * n_partials + blockIdx.x * Z + blockIdx.z] = t;
+  }
+}
+
+// g = the Z partial gradients added in z order in fp64, rounded once
+__global__ void __launch_bounds__(256)
+psd_combine_kernel(const double* __restrict__ gpart, float* __restrict__ g, int64_t total, int32_t Z, int64_t cols, int64_t ld) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+    if (e % ld >= cols) continue;                 // padding columns of g are not this objective's
+    double t = 0.0;
+    for (int z = 0; z < Z; ++z) t += gpart[(int64_t)z * total + e];
+    g[e] = (float)t;
   }
 }
 
 }  // namespace
 
-int32_t psd_loss_blocks(int32_t n) { return (n + T - 1) / T; }
+#ifndef LSGD_PSD_SPLIT
+#define LSGD_PSD_SPLIT 2
+#endif
+// CTAs per row block: small ranks are latency-bound and split the column blocks (see psd_grad_kernel)
+int32_t psd_split(int32_t r) { return r <= 32 ? LSGD_PSD_SPLIT : 1; }
 
-cudaError_t launch_psd_grad(const float* x, float* g, const float* M, int32_t n, int32_t r, int32_t P, int64_t ld,
-                            double* partials, int32_t n_partials, bool write_g, cudaStream_t s) {
+int32_t psd_loss_blocks(int32_t n, int32_t r) { return ((n + T - 1) / T) * psd_split(r); }
+
+template <int KM, int Z>
+cudaError_t launch_psd_t(const float* x, float* g, const float* M, int32_t n, int32_t r, int32_t P, int64_t ld, double* partials,
+                         int32_t n_partials, int wg, double* gpart, cudaStream_t s) {
   const int pitch = r | 1;
   const size_t smem = sizeof(double) * (size_t)(2 * T * pitch + T * (T + 1));
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(psd_grad_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(psd_grad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(psd_grad_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(psd_grad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(psd_grad_kernel<KM, Z>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
+    if (e == cudaSuccess && Z > 1)   // two CTAs per SM: ask for the largest shared-memory carve-out
+      e = cudaFuncSetAttribute(psd_grad_kernel<KM, Z>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid((unsigned)n_partials, (unsigned)P), block(TH, TH);
-  const int wg = write_g ? 1 : 0;
-  if (r <= 16) psd_grad_kernel<1><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg);
-  else if (r <= 32) psd_grad_kernel<2><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg);
-  else if (r <= 64) psd_grad_kernel<4><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg);
-  else psd_grad_kernel<8><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg);
+  dim3 grid((unsigned)(n_partials / Z), (unsigned)P, (unsigned)Z), block(TH, TH);
+  psd_grad_kernel<KM, Z><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg, gpart, P);
+  if (Z > 1 && wg) {
+    const int64_t total = (int64_t)P * ld;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    psd_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(gpart, g, total, Z, (int64_t)n * r, ld);
+  }
   return cudaGetLastError();
+}
+
+// gpart: DEVICE double[psd_split(r) * P * ld] when psd_split(r) > 1 (unused otherwise)
+cudaError_t launch_psd_grad(const float* x, float* g, const float* M, int32_t n, int32_t r, int32_t P, int64_t ld,
+                            double* partials, int32_t n_partials, bool write_g, double* gpart, cudaStream_t s) {
+  if (n_partials != psd_loss_blocks(n, r)) return cudaErrorInvalidValue;
+  const int wg = write_g ? 1 : 0;
+  constexpr int ZS = LSGD_PSD_SPLIT;
+  if (psd_split(r) > 1 && !gpart) return cudaErrorInvalidValue;
+  if (r <= 16) return launch_psd_t<1, ZS>(x, g, M, n, r, P, ld, partials, n_partials, wg, gpart, s);
+  if (r <= 32) return launch_psd_t<2, ZS>(x, g, M, n, r, P, ld, partials, n_partials, wg, gpart, s);
+  if (r <= 64) return launch_psd_t<4, 1>(x, g, M, n, r, P, ld, partials, n_partials, wg, gpart, s);
+  return launch_psd_t<8, 1>(x, g, M, n, r, P, ld, partials, n_partials, wg, gpart, s);
 }
 
 }  // namespace lsgd
