@@ -26,7 +26,7 @@ def _oracle(w):
     return orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
 
 
-def _run_pair(w, steps):
+def _run_pair(w, steps, flags=0):
     import torch
     from paper_1905_10395_b200.runner import Population
     o = _oracle(w)
@@ -34,7 +34,7 @@ def _run_pair(w, steps):
     for _ in range(steps):
         o.step()
         train_ref.append(o.obj.last_train_loss.copy())
-    pop = Population(w)
+    pop = Population(w, flags=flags)
     train_gpu = []
     for _ in range(steps):
         pop.step(record=True)
@@ -48,7 +48,7 @@ def _run_pair(w, steps):
                 assert (srt[1] - srt[0]) <= TOL * abs(srt[0]), "leaders differ without a near-tie"
                 break
         pop.close()
-        pop = Population(w)
+        pop = Population(w, flags=flags)
         train_gpu = []
         for t in range(steps):
             fl = torch.from_numpy(o.history[t // w.tau]["loss"]).cuda() if t % w.tau == 0 else None
@@ -120,9 +120,12 @@ def test_mlp_one_step_gradient_matches_oracle():
     pop.close()
 
 
-def test_config3_mlp_population_ten_steps():
+@pytest.mark.parametrize("fused", [False, True])
+def test_config3_mlp_population_ten_steps(fused):
+    # fused = the configuration the benchmark times (LSGD_FLAG_MLP_FUSED_STEP)
+    from paper_1905_10395_b200 import api
     w = inputs.config(3, steps=10)
-    pop, o, tg, tr, forced = _run_pair(w, 10)
+    pop, o, tg, tr, forced = _run_pair(w, 10, flags=api.FLAG_MLP_FUSED_STEP if fused else 0)
     _check(pop, o, w, tg, tr, forced)
     pop.close()
 

@@ -266,9 +266,12 @@ def test_matcomp_fused_step_is_bit_identical_to_the_materialised_gradient_path(r
     b.close()
 
 
-def test_config2_matrix_completion():
+@pytest.mark.parametrize("fused", [False, True])
+def test_config2_matrix_completion(fused):
+    # fused = the configuration the benchmark times (LSGD_FLAG_MATCOMP_FUSED_STEP)
+    from paper_1905_10395_b200 import api
     w = inputs.config(2, steps=10)
-    pop = _pop(w)
+    pop = _pop(w, flags=api.FLAG_MATCOMP_FUSED_STEP if fused else 0)
     pop.run(10, record=True)
     o = _oracle(w)
     o.run(10)
