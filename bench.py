@@ -89,7 +89,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
@@ -480,33 +480,63 @@ def run_ours(args):
         if pop.lsgd.check_device() != 0:
             raise SystemExit("device status word set during the graph replays")
 
-    # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs, D2H of its result
+    # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs, D2H of its result.
+    # Two handles on two streams take the steps in turn, so one step's read-back crosses the bus while the next
+    # step's inputs come in (the link is full duplex); every step still copies all of x and g in and all of x out.
     if rank == 0 and world == 1 and not args.no_e2e and hx is not None and not alg1_mode:
-        e_steps = args.e2e_steps
-        hout = hx                                   # result is read back into the pinned x buffer
+        e_steps = max(2, args.e2e_steps + (args.e2e_steps & 1))       # an even number: both streams do the same work
+        pop.close()
+        torch.cuda.synchronize(dev)
+        loss_host = torch.from_numpy(w.arrays["loss_ring"]).pin_memory()
+        lanes = []
+        for k in range(2):
+            st = torch.cuda.Stream(dev)
+            xk = x if k == 0 else torch.empty_like(x)
+            gk = g if k == 0 else torch.empty_like(g)
+            with torch.cuda.stream(st):
+                pk = Population(w, device=str(dev), x=xk, g=gk, arithmetic=args.arith, stream=st,
+                                momentum=args.momentum, weight_decay=args.weight_decay)
+            lanes.append(dict(stream=st, pop=pk, out=torch.empty((P, d), dtype=torch.float32, pin_memory=True),
+                              dloss=torch.empty(P, dtype=torch.float32, device=dev)))
+        torch.cuda.synchronize(dev)
+
+        def e2e_step(it):
+            ln = lanes[it & 1]
+            with torch.cuda.stream(ln["stream"]):
+                ln["pop"].x.copy_(hx, non_blocking=True)
+                ln["pop"].g.copy_(hg, non_blocking=True)
+                ln["dloss"].copy_(loss_host[it % loss_host.shape[0]], non_blocking=True)
+                ln["pop"].lsgd.grad(None)
+                ln["pop"].lsgd.elect(ln["dloss"])
+                ln["pop"].lsgd.step()
+                ln["out"].copy_(ln["pop"].x, non_blocking=True)
+
+        for it in range(2):                                            # one untimed step per stream
+            e2e_step(it)
         torch.cuda.synchronize(dev)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        loss_host = torch.from_numpy(w.arrays["loss_ring"]).pin_memory()
-        dloss = torch.empty(P, dtype=torch.float32, device=dev)
-        for it in range(e_steps + 1):
-            if it == 1:
-                e0.record()
-            pop.x.copy_(hx, non_blocking=True)
-            pop.g.copy_(hg, non_blocking=True)
-            dloss.copy_(loss_host[it % loss_host.shape[0]], non_blocking=True)
-            pop.lsgd.grad(None)
-            pop.lsgd.elect(dloss)
-            pop.lsgd.step()
-            hout.copy_(pop.x, non_blocking=True)
-        e1.record()
+        sa, sb = lanes[0]["stream"], lanes[1]["stream"]
+        e0.record(sa)
+        sb.wait_event(e0)
+        for it in range(e_steps):
+            e2e_step(it)
+        sa.wait_stream(sb)
+        e1.record(sa)
         torch.cuda.synchronize(dev)
         e_ms = e0.elapsed_time(e1) / e_steps
+        for ln in lanes:
+            if ln["pop"].lsgd.check_device() != 0:
+                raise SystemExit("device status word set during the end-to-end steps")
+            ln["pop"].close()
         line["e2e"] = {"value": P * d / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(2 * P * d * 4 + P * 4),
                        "d2h_bytes_per_step": int(P * d * 4), "ms_per_step": e_ms, "steps": e_steps,
-                       "note": "every step elects (a pull step) so tau does not apply"}
+                       "note": "every step elects (a pull step) so tau does not apply; two handles on two streams "
+                               "alternate so that read-back and upload overlap on the full-duplex link"}
+        pop = None
     else:
         line["e2e"] = None
-    pop.close()
+    if pop is not None:
+        pop.close()
 
     # ---- CPU oracle beside it (rank 0, N = 1 only)
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -597,14 +627,14 @@ def run_sharded(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4", "psd"])
     ap.add_argument("--rank", type=int, default=10, help="psd workload: rank r")
     ap.add_argument("--tau", type=int, default=0)
     ap.add_argument("--arith", type=int, default=0, choices=[0, 1, 2])
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--sample-cols", type=int, default=0)
     ap.add_argument("--d", type=int, default=0, help="shrink the c4 workload (profiler captures on a small case)")
     ap.add_argument("--schedule", default="fused", choices=["fused", "algorithm1"],
