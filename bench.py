@@ -268,7 +268,7 @@ def run_reference(args):
         return
     spec = workload_spec(args)
     steps, warmup = args.steps, args.warmup
-    sample = args.sample_cols or (1 << 22)
+    sample = args.sample_cols or (1 << 20)      # about a quarter of a second of oracle work per C4 step
     value, dt, what, _ = oracle_sample_run(spec, steps, warmup, sample)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
