@@ -190,7 +190,7 @@ def workload_spec(args):
 
 # DRAM bytes per worker-parameter of the update kernels, from the ncu counters of a d = 2^22 capture of
 # the same kernels (profiles/pull_update_kernel_c4.md); traffic is proportional to d.
-MEASURED_TRAFFIC_PER_WORKER_PARAM = {"pull": 11.27, "plain": 11.30}
+MEASURED_TRAFFIC_PER_WORKER_PARAM = {"pull": 11.24, "plain": 11.30}
 
 
 def bytes_per_worker_param(spec):
