@@ -198,3 +198,30 @@ def test_election_on_the_running_mean_of_training_losses():
     want = np.mean([tg[t] for t in range(max(0, t_last - 2), t_last + 1)], axis=0)
     assert np.allclose(pop.history[k]["loss"], want, rtol=1e-5, atol=0)
     pop.close()
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_cuda_graph_replay_of_the_mlp_step_equals_the_call_by_call_run(fused):
+    """Whole periods of the MLP step (tensor-core products, programmatic dependent launches, the fused step)
+    captured into a CUDA graph and replayed give the same parameters, bit for bit, as issuing the calls."""
+    import torch
+    from paper_1905_10395_b200 import api
+    from paper_1905_10395_b200.runner import Population
+    w = inputs.make_mlp(4, 2, dims=(64, 128, 128, 10), pool=512, heldout=128, batch=128, steps=4, tau=2, config_id=63)
+    flags = api.FLAG_MLP_FUSED_STEP if fused else 0
+    stream = torch.cuda.Stream()
+    a = Population(w, flags=flags, stream=stream)
+    with torch.cuda.stream(stream):
+        a.run(4)                                     # un-captured: one pass over the batch ring
+        a.capture(4)
+        a.replay()
+        a.replay()
+    stream.synchronize()
+    assert a.lsgd.t() == 12
+    b = Population(w, flags=flags)
+    b.run(12)
+    assert np.array_equal(a.x_host().view(np.uint32), b.x_host().view(np.uint32))
+    assert a.lsgd.leaders()[1] == b.lsgd.leaders()[1]
+    assert a.lsgd.check_device() == 0
+    a.close()
+    b.close()

@@ -377,7 +377,7 @@ def test_matcomp_gradient_is_reproducible_bit_for_bit():
     assert rel_err(runs[0], o.x) <= TOL
 
 
-@pytest.mark.parametrize("kind", ["quadratic", "matcomp"])
+@pytest.mark.parametrize("kind", ["quadratic", "matcomp", "matcomp_fused"])
 def test_cuda_graph_replay_matches_the_oracle(kind):
     """Whole communication periods captured into a CUDA graph and replayed (lsgd_advance_step keeps the
     library's step counter in line) give the same trajectory as issuing the calls one by one."""
@@ -387,8 +387,10 @@ def test_cuda_graph_replay_matches_the_oracle(kind):
     else:
         w = inputs.make_matcomp(4, 2, n_rows=300, n_cols=200, rank=7, n_obs=5000, n_heldout=512, batch=700, steps=4,
                                 tau=2, config_id=58)
+    from paper_1905_10395_b200 import api
     stream = torch.cuda.Stream()
-    pop = _pop(w, fused_quadratic=(kind == "quadratic"), stream=stream)
+    pop = _pop(w, fused_quadratic=(kind == "quadratic"), stream=stream,
+               flags=api.FLAG_MATCOMP_FUSED_STEP if kind == "matcomp_fused" else 0)
     with torch.cuda.stream(stream):
         pop.run(4)                                   # un-captured warm-up: one pass over the batch ring
         pop.capture(4)
