@@ -46,7 +46,8 @@ typedef enum {
   LSGD_ERR_INVALID_ARG = 1,  /* NULL where not allowed, P < 1, tau < 1, non-finite eta, ld < d ...  */
   LSGD_ERR_BAD_GROUPS = 2,   /* G < 1, G > P, group id out of range, or an empty group               */
   LSGD_ERR_ALIGNMENT = 3,    /* a DEVICE pointer is not 16-byte aligned, or ld is not a multiple of 32 */
-  LSGD_ERR_STATE = 4,        /* call order: pull step before any election, step without a gradient   */
+  LSGD_ERR_STATE = 4,        /* call order: pull step before any election, step without a gradient;
+                                or grad / elect / step called while another device is current        */
   LSGD_ERR_CUDA = 5,         /* a CUDA runtime call or launch failed (no usable device included)     */
   LSGD_ERR_UNSUPPORTED = 6,  /* combination not implemented (documented at the argument)             */
   LSGD_ERR_DEVICE_FLAG = 7,  /* a kernel recorded a bounded-wait / bounds failure in its status word */
@@ -80,7 +81,9 @@ typedef struct {
 /* Matrix completion with factors: row i of x is [X (n_rows x rank) | Y (n_cols x rank)], row-major.
  * Minibatch loss (1/(2B)) sum (<X_r, Y_c> - v)^2 over B observed entries per worker per step, given
  * to lsgd_grad as positions into the observed list; election loss = mean squared residual over the
- * fixed held-out positions.  (Low-rank completion is the paper's motivating example, Section 2.1.) */
+ * fixed held-out positions.  (Low-rank completion is the paper's motivating example, Section 2.1.)
+ * batch <= 32768 (LSGD_ERR_UNSUPPORTED beyond): duplicates are summed exactly in a 2^-44 fixed-point
+ * accumulator whose range also needs every contribution |e * y / B| < 2^4 (see LSGD_DEVFLAG_OVERFLOW). */
 typedef struct {
   int32_t n_rows, n_cols, rank;
   int32_t n_obs;
@@ -109,7 +112,7 @@ typedef struct {
 #define LSGD_MLP_MAX_LAYERS 3
 typedef struct {
   int32_t dims[LSGD_MLP_MAX_LAYERS + 1]; /* n_in, hidden, hidden, n_classes                          */
-  int32_t batch;             /* training samples per worker per step (multiple of 128)              */
+  int32_t batch;             /* training samples per worker per step (multiple of 8, at most 1024)   */
   int32_t pool;              /* number of rows of pool_x                                             */
   const float* pool_x;       /* DEVICE float[pool][dims[0]] training samples                         */
   const int32_t* pool_y;     /* DEVICE int32[pool] labels                                            */
@@ -188,8 +191,11 @@ typedef struct {
  *                                if tau | t:   local leaders re-elected, x_i <- x_i - eta lambda (x_i - x~^j), copies refreshed;
  *                                if tau_G | t: global leader re-elected, x_i <- x_i - eta lambda_G (x_i - x~), copy refreshed.
  * All pulls are scaled by eta (Section 3.1.1; pass coefficient / eta for the unscaled form the listing
- * prints).  One loss vector (given, or the objective's own loss at the current x) serves both
- * elections of a communication.  LSGD_FLAG_MLP_FUSED_STEP is ignored in this mode.                  */
+ * prints).  When both periods are due and loss == NULL, the order of the listing is kept: the objective's
+ * loss is evaluated, the local leaders are elected and the local pull applied, then the loss is evaluated
+ * AGAIN on the pulled parameters and the global leader elected from that second vector (lsgd_get_loss then
+ * returns the second vector).  A loss vector given by the caller serves both elections of a communication.
+ * LSGD_FLAG_MLP_FUSED_STEP is ignored in this mode.                                                   */
 #define LSGD_FLAG_ALGORITHM1 2u
 
 /* Validates the configuration on the host, copies the group map, builds the group tables and
@@ -243,11 +249,38 @@ LSGD_API lsgd_status lsgd_get_step(lsgd_handle h, int64_t* t);
  * otherwise).  The paper's deep-network runs elect on a running mean of such training losses
  * (Section 4.1); here it is reported for monitoring and parity checks.                             */
 LSGD_API lsgd_status lsgd_get_train_loss(lsgd_handle h, float* loss /* HOST float[P] */);
+/* The hidden activations the last lsgd_grad stored for its backward pass (MLP objective only), as bf16 bit
+ * patterns: h1 HOST uint16[P][batch][dims[1]], h2 HOST uint16[P][batch][dims[2]] (either may be NULL).  They
+ * hold every ReLU decision of that step, so a parity check can verify them against its own pre-activations
+ * and then follow the same decisions where a pre-activation is within rounding of zero.  Synchronises.   */
+LSGD_API lsgd_status lsgd_mlp_get_activations(lsgd_handle h, uint16_t* h1, uint16_t* h2);
 /* Times each worker has been global / local leader so far (the leader statistics of Section 4.2). */
 LSGD_API lsgd_status lsgd_get_leader_counts(lsgd_handle h, int32_t* global_counts /* HOST int32[P] */,
                                    int32_t* local_counts /* HOST int32[P] */);
-/* Reads and clears the device status word; LSGD_ERR_DEVICE_FLAG if any kernel has set it.        */
+/* Reads and clears the device status word; LSGD_ERR_DEVICE_FLAG if any kernel has set it.  Bits:
+ *   LSGD_DEVFLAG_BAD_LEADER   a leader index outside [0, P) reached an update kernel (the pull was skipped);
+ *   LSGD_DEVFLAG_WAIT_TIMEOUT a bounded wait on a copy / tensor-core barrier ran out (about one second): the
+ *                             kernel left its loops and returned, its output is incomplete;
+ *   LSGD_DEVFLAG_BAD_INDEX    a batch position, sample index or observed row / column out of range: that
+ *                             entry was skipped before anything was dereferenced;
+ *   LSGD_DEVFLAG_OVERFLOW     MATCOMP: a gradient contribution e * y / B was not finite or reached 2^4 in
+ *                             magnitude, the range of the fixed-point accumulator (2^-44 resolution, at most
+ *                             2^15 contributions per entry: batch <= 32768, LSGD_ERR_UNSUPPORTED beyond);
+ *                             the contribution was not added -- a diverging worker is reported instead of
+ *                             being turned into finite garbage.                                          */
+#define LSGD_DEVFLAG_BAD_LEADER 1u
+#define LSGD_DEVFLAG_WAIT_TIMEOUT 2u
+#define LSGD_DEVFLAG_BAD_INDEX 4u
+#define LSGD_DEVFLAG_OVERFLOW 8u
 LSGD_API lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out /* HOST, may be NULL */);
+/* Self-test of the bounded device waits (test support; the paper has no counterpart).  Every wait of the
+ * copy pipelines in the update kernels is limited by a clock budget after which the kernel records
+ * LSGD_DEVFLAG_WAIT_TIMEOUT and returns instead of hanging.  This call runs that same wait routine in a
+ * one-warp kernel on a barrier that nothing completes (no copy is in flight), with a budget of budget_cycles
+ * clock cycles (1 .. 10^8, LSGD_ERR_INVALID_ARG otherwise), synchronises the stream and stores 1 in
+ * *gave_up (HOST) if the wait ran out.  The status word keeps the bit until lsgd_check_device reads it;
+ * the context stays usable.                                                                          */
+LSGD_API lsgd_status lsgd_selftest_wait_timeout(lsgd_handle h, int64_t budget_cycles, int32_t* gave_up);
 /* The "center variable" the paper reports at test time for LSGD (Section 4.1): the average of the
  * parameters of all workers, center[k] = (1/P) sum_i x[i][k], summed in worker order in fp64 and rounded
  * once.  center: DEVICE float[ld] (columns d..ld-1 are written as the mean of the padding).  Enqueued
@@ -327,6 +360,9 @@ typedef struct {
   int64_t ld_mask, stride_mask;
 } lsgd_bgemm_desc;
 LSGD_API lsgd_status lsgd_bgemm_bf16(const lsgd_bgemm_desc* desc, void* stream);
+/* Synchronises the current device, then reads and clears the status word of lsgd_bgemm_bf16 on it (the
+ * product's bounded waits record LSGD_DEVFLAG_WAIT_TIMEOUT there): LSGD_ERR_DEVICE_FLAG if it was set.  */
+LSGD_API lsgd_status lsgd_bgemm_check_device(uint32_t* flag_out /* HOST, may be NULL */);
 
 #ifdef __cplusplus
 }

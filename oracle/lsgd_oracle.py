@@ -17,8 +17,8 @@ Readings of the paper taken here (each is also exercised by a pin in tests/test_
     supplement "Definitions and Notation", and the written-out matrix-completion update
     X+ = (1 - eta lambda) X + eta lambda Z - eta grad F(X); Eq. (1) prints them unscaled).
   * gamma = gamma_G = 0 and tau_G = tau: leaders are re-elected and both pulls applied on steps
-    t = 0, tau, 2 tau, ... ("the leader is updated only at the beginning of each period");
-    all other steps are plain (S)GD steps.
+    t = 0, tau, 2 tau, ... (leaders change only at period boundaries: supplement, "Definitions and
+    Notation"); all other steps are plain (S)GD steps.
   * on a pull step the gradient, both leaders and both pulls are all taken at x_t (Eq. (1): every
     right-hand term carries subscript t), i.e. a simultaneous (Jacobi) update of all workers.
   * argmin ties go to the lowest worker index; the order on losses is
@@ -458,8 +458,11 @@ class Algorithm1Oracle:
                    if tau_G | t:  x~   <- argmin over all workers;                         x_i <- x_i - eta lambda_G (x_i - x~)
 
     Readings: every pull is scaled by eta like the gradient (Section 3.1.1; the listing prints them
-    unscaled -- pass coefficient / eta to obtain that form).  One loss vector per communication,
-    evaluated after the gradient step, serves both elections of that communication."""
+    unscaled -- pass coefficient / eta to obtain that form).  A communication follows the listing's order:
+    the local argmin is taken on losses evaluated after the gradient step; when the global period fires as
+    well, the global argmin is taken on losses evaluated AFTER the local pull has moved the workers (the
+    listing's second "if" comes after the first one's pull).  A loss vector supplied from outside
+    (``forced_loss``, or an objective whose losses do not depend on x) serves both elections."""
 
     def __init__(self, x0, objective, group_of, G, eta, lambda_l, lambda_g, gamma_l, gamma_g, tau, tau_g):
         assert tau >= 1 and tau_g >= 1
@@ -498,19 +501,26 @@ class Algorithm1Oracle:
         self.t += 1
         local, glob = self.t % self.tau == 0, self.t % self.tau_g == 0
         if local or glob:
-            loss = np.asarray(self.obj.loss(self.x, self.n_elections) if forced_loss is None else forced_loss, dtype=F32)
+            n = self.n_elections                      # one communication = one election event
             self.n_elections += 1
-            ll, gl = elect(loss, self.group_of, self.G)
+
+            def losses():
+                return np.asarray(self.obj.loss(self.x, n) if forced_loss is None else forced_loss, dtype=F32)
+
+            loss = losses()
+            loss_global = loss
             if local:
-                self.ll = ll
-                self.z_l = [self.x[int(l)].copy() for l in ll]
+                self.ll, _ = elect(loss, self.group_of, self.G)
+                self.z_l = [self.x[int(l)].copy() for l in self.ll]
                 self._pull(self.eta * self.lambda_l, lambda i: self.z_l[int(self.group_of[i])])
             if glob:
-                self.gl = gl
-                self.z_g = self.x[int(gl)].copy()
+                if local:
+                    loss_global = losses()            # the local pull has moved the workers
+                _, self.gl = elect(loss_global, self.group_of, self.G)
+                self.z_g = self.x[int(self.gl)].copy()
                 self._pull(self.eta * self.lambda_g, lambda i: self.z_g)
-            self.history.append({"t": self.t, "loss": loss.copy(), "ll": self.ll.copy(), "gl": self.gl,
-                                 "local": local, "global": glob})
+            self.history.append({"t": self.t, "loss": loss.copy(), "loss_global": loss_global.copy(),
+                                 "ll": self.ll.copy(), "gl": self.gl, "local": local, "global": glob})
 
     def run(self, steps: int) -> np.ndarray:
         for _ in range(steps):

@@ -18,6 +18,8 @@ ARITH_FP64, ARITH_FP64_FMA, ARITH_FP32 = range(3)
 FLAG_MLP_FUSED_STEP = 1
 FLAG_ALGORITHM1 = 2
 FLAG_MATCOMP_FUSED_STEP = 4
+# bits of the device status word (lsgd_check_device)
+DEVFLAG_BAD_LEADER, DEVFLAG_WAIT_TIMEOUT, DEVFLAG_BAD_INDEX, DEVFLAG_OVERFLOW = 1, 2, 4, 8
 
 
 class LsgdError(RuntimeError):
@@ -97,6 +99,12 @@ def lib() -> C.CDLL:
         L.lsgd_get_leader_counts.argtypes = [H, C.c_void_p, C.c_void_p]
         L.lsgd_check_device.argtypes = [H, C.POINTER(C.c_uint32)]
         L.lsgd_set_eta.argtypes = [H, C.c_float]
+        L.lsgd_mlp_get_activations.argtypes = [H, C.c_void_p, C.c_void_p]
+        L.lsgd_mlp_get_activations.restype = C.c_int
+        L.lsgd_selftest_wait_timeout.argtypes = [H, C.c_int64, C.POINTER(C.c_int32)]
+        L.lsgd_selftest_wait_timeout.restype = C.c_int
+        L.lsgd_bgemm_check_device.argtypes = [C.POINTER(C.c_uint32)]
+        L.lsgd_bgemm_check_device.restype = C.c_int
         L.lsgd_quadratic_loss_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64,
                                                   C.c_void_p, C.c_void_p]
         L.lsgd_quadratic_loss_noalloc.restype = C.c_int
@@ -165,6 +173,15 @@ def lsgd_quadratic_loss_noalloc(x, a, b, P: int, d: int, ld: int, loss, stream: 
 
 def lsgd_bgemm_bf16(desc: BgemmDesc, stream: int = 0) -> None:
     _check(lib().lsgd_bgemm_bf16(C.byref(desc), stream or None), "lsgd_bgemm_bf16")
+
+
+def lsgd_bgemm_check_device() -> int:
+    """Status word of lsgd_bgemm_bf16 on the current device (read and cleared); 0 = no kernel reported anything."""
+    f = C.c_uint32()
+    s = lib().lsgd_bgemm_check_device(C.byref(f))
+    if s not in (OK, ERR_DEVICE_FLAG):
+        raise LsgdError(s, "lsgd_bgemm_check_device")
+    return f.value
 
 
 def mlp_param_offsets(dims: Sequence[int]):
@@ -246,6 +263,15 @@ class Lsgd:
         _check(lib().lsgd_get_train_loss(self.h, out.ctypes.data), "lsgd_get_train_loss")
         return out
 
+    def mlp_activations(self, batch: int, d1: int, d2: int):
+        """Hidden activations stored by the last grad() of the MLP objective, as float32 [P, batch, d1] / [.., d2]
+        (the library holds them as bf16; widening is exact)."""
+        h1 = np.empty((self.P, batch, d1), dtype=np.uint16)
+        h2 = np.empty((self.P, batch, d2), dtype=np.uint16)
+        _check(lib().lsgd_mlp_get_activations(self.h, h1.ctypes.data, h2.ctypes.data), "lsgd_mlp_get_activations")
+        widen = lambda a: (a.astype(np.uint32) << 16).view(np.float32)
+        return widen(h1), widen(h2)
+
     def center(self, out):
         """out (device float[ld]) <- average of all workers' parameters (the paper's center variable)."""
         _check(lib().lsgd_center(self.h, _ptr(out)), "lsgd_center")
@@ -273,6 +299,12 @@ class Lsgd:
         if s not in (OK, ERR_DEVICE_FLAG):
             raise LsgdError(s, "lsgd_check_device")
         return f.value
+
+    def selftest_wait_timeout(self, budget_cycles: int) -> int:
+        """Runs the update pipeline's bounded wait on a barrier nothing completes; 1 if the wait ran out."""
+        out = C.c_int32(-1)
+        _check(lib().lsgd_selftest_wait_timeout(self.h, int(budget_cycles), C.byref(out)), "lsgd_selftest_wait_timeout")
+        return out.value
 
     def set_eta(self, eta: float):
         _check(lib().lsgd_set_eta(self.h, eta), "lsgd_set_eta")

@@ -477,19 +477,15 @@ bool make_tile_map_bf16(CUtensorMap* map, const void* base, int64_t N, int64_t M
 }
 
 cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmShape& p, cudaStream_t s) {
-  static bool attr_set = false;
-  static int sms = 0;
-  if (!attr_set) {
+  static OncePerDevice attr;
+  if (!attr.here()) {
     cudaError_t e = cudaFuncSetAttribute(bgemm_bf16_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(bgemm_bf16_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
-    attr_set = true;
+    attr.here() = true;
   }
+  const int sms = sm_count();
   // Tensor maps of the epilogue: map_c is C (fp32 or bf16) -- for the fused SGD step the parameter block
   // itself, loaded and stored; map_aux is the ReLU mask (input) or the bf16 copy of the parameters (output).
   CUtensorMap map_c, map_aux;

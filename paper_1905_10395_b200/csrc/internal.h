@@ -12,10 +12,34 @@ namespace lsgd {
 
 // Status-word bits set by kernels (reported as LSGD_ERR_DEVICE_FLAG).
 enum : uint32_t {
-  FLAG_BAD_LEADER = 1u << 0,   // a leader index outside [0, P) reached the update kernel
-  FLAG_WAIT_TIMEOUT = 1u << 1, // a bounded mbarrier / tensor-pipe wait ran out
-  FLAG_BAD_INDEX = 1u << 2,    // a batch position / sample index out of range (entry skipped)
+  FLAG_BAD_LEADER = LSGD_DEVFLAG_BAD_LEADER,     // a leader index outside [0, P) reached the update kernel
+  FLAG_WAIT_TIMEOUT = LSGD_DEVFLAG_WAIT_TIMEOUT, // a bounded mbarrier / tensor-pipe wait ran out
+  FLAG_BAD_INDEX = LSGD_DEVFLAG_BAD_INDEX,       // a batch position / sample index out of range (entry skipped)
+  FLAG_OVERFLOW = LSGD_DEVFLAG_OVERFLOW,         // a contribution outside the fixed-point accumulator's range (skipped)
 };
+
+// One-time launch state is per DEVICE, not per process: a kernel's dynamic-shared-memory attribute applies to
+// the device that was current when it was set, and devices need not have the same number of SMs.
+constexpr int kMaxDevices = 64;
+inline int device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+  return dev;
+}
+struct OncePerDevice {
+  bool done[kMaxDevices] = {};
+  bool& here() { return done[device_slot()]; }
+};
+inline int sm_count() {
+  static int sms[kMaxDevices] = {};
+  const int dev = device_slot();
+  if (sms[dev] == 0) {
+    int n = 0;
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    sms[dev] = n > 0 ? n : 148;
+  }
+  return sms[dev];
+}
 
 struct GroupTables {
   // Workers sorted by group: members of group j are rows_by_group[group_start[j] .. group_start[j+1]).
@@ -63,6 +87,9 @@ cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s);
 // Section 4.1 optimiser (a.v != nullptr): Nesterov momentum + weight decay around the same step.
 cudaError_t launch_momentum_update(const UpdateArgs& a, cudaStream_t s);
 cudaError_t launch_momentum_update_chunked(const UpdateArgs& a, cudaStream_t s);   // cudaErrorNotSupported: shape does not fit
+// One warp runs the update pipeline's bounded barrier wait on a barrier nothing completes: *gave_up (DEVICE) <- 1
+// and FLAG_WAIT_TIMEOUT in *status after about budget_cycles clock cycles.
+cudaError_t launch_wait_timeout_selftest(uint32_t* status, long long budget_cycles, int* gave_up, cudaStream_t s);
 cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, int64_t ld, cudaStream_t s);
 
 struct ElectArgs {
@@ -180,6 +207,7 @@ struct lsgd_ctx {
   float* d_loss;
   unsigned long long* d_group_keys;
   double* d_partials;
+  int32_t* d_selftest;          // one word written by lsgd_selftest_wait_timeout
   int32_t n_partials;
   int64_t t;
   int64_t n_elections;

@@ -51,6 +51,8 @@ lsgd_status validate(const lsgd_config* c) {
     if (c->flags & (LSGD_FLAG_MLP_FUSED_STEP | LSGD_FLAG_ALGORITHM1)) return LSGD_ERR_UNSUPPORTED;
   }
   if (c->P > kMaxWorkers) return LSGD_ERR_UNSUPPORTED;
+  // the register-staged pull kernel keeps P + 2 G + 1 table words in shared memory below the 48 KiB default
+  if ((int64_t)c->P + 2 * (int64_t)c->G + 2 > 12288) return LSGD_ERR_UNSUPPORTED;
   if (c->ld % 32 != 0) return LSGD_ERR_ALIGNMENT;
   if (!c->x) return LSGD_ERR_INVALID_ARG;
   if (!aligned16(c->x) || !aligned16(c->g)) return LSGD_ERR_ALIGNMENT;
@@ -72,6 +74,7 @@ lsgd_status validate(const lsgd_config* c) {
       if (!m->obs_r || !m->obs_c || !m->obs_v || !m->heldout_pos) return LSGD_ERR_INVALID_ARG;
       if ((int64_t)(m->n_rows + (int64_t)m->n_cols) * m->rank != c->d) return LSGD_ERR_INVALID_ARG;
       if (m->rank > 32) return LSGD_ERR_UNSUPPORTED;
+      if (m->batch > (1 << 15)) return LSGD_ERR_UNSUPPORTED;   // range of the fixed-point gradient accumulator
       break;
     }
     case LSGD_OBJ_PSD_COMPLETION: {
@@ -95,6 +98,12 @@ lsgd_status validate(const lsgd_config* c) {
 }
 
 lsgd_status algorithm1_pulls(lsgd_ctx* h, bool local, bool glob);
+
+// The handle's buffers, stream and kernel attributes belong to the device that was current at creation.
+inline bool on_own_device(const lsgd_ctx* h) {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
+}
 
 GroupTables tables(const lsgd_ctx* h) { return GroupTables{h->d_rows_by_group, h->d_group_start, h->d_group_of}; }
 
@@ -168,6 +177,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   const size_t o_cg = take(sizeof(int32_t) * P), o_cl = take(sizeof(int32_t) * P), o_status = take(sizeof(uint32_t));
   const size_t o_loss = take(sizeof(float) * P), o_keys = take(sizeof(unsigned long long) * G);
   const size_t o_part = take(sizeof(double) * (size_t)P * (size_t)(h->n_partials > 0 ? h->n_partials : 1));
+  const size_t o_self = take(sizeof(int32_t));
   if (cudaMalloc(&h->slab, off) != cudaSuccess) {
     delete h;
     return LSGD_ERR_CUDA;
@@ -184,6 +194,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->d_loss = reinterpret_cast<float*>(base + o_loss);
   h->d_group_keys = reinterpret_cast<unsigned long long*>(base + o_keys);
   h->d_partials = reinterpret_cast<double*>(base + o_part);
+  h->d_selftest = reinterpret_cast<int32_t*>(base + o_self);
 
   bool ok = cudaMemsetAsync(h->slab, 0, off, h->stream) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(h->d_rows_by_group, rows.data(), sizeof(int32_t) * P, cudaMemcpyHostToDevice, h->stream) == cudaSuccess;
@@ -217,6 +228,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
 
 lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
   if (!h) return LSGD_ERR_INVALID_ARG;
+  if (!on_own_device(h)) return LSGD_ERR_STATE;
   const lsgd_config& c = h->cfg;
   switch (c.objective) {
     case LSGD_OBJ_EXTERNAL:
@@ -262,8 +274,57 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
   return LSGD_OK;
 }
 
+// Evaluates the objective's own election loss at the current x and points the election at it.
+static lsgd_status own_election_loss(lsgd_ctx* h, ElectArgs& e) {
+  const lsgd_config& c = h->cfg;
+  e.loss_in = nullptr;
+  switch (c.objective) {
+    case LSGD_OBJ_QUADRATIC:
+      LSGD_CUDA(launch_quadratic_loss_partials(c.x, h->quad.a, h->quad.b, c.P, c.d, c.ld, h->d_partials,
+                                               h->n_partials, h->stream));
+      e.partials = h->d_partials;
+      e.n_partials = h->n_partials;
+      e.partial_scale = 0.5;
+      return LSGD_OK;
+    case LSGD_OBJ_MATCOMP: {
+      MatcompArgs a{h->mc, c.x, c.g, c.ld, c.P, h->d_status};
+      LSGD_CUDA(launch_matcomp_loss_partials(a, h->d_partials, h->n_partials, h->stream));
+      e.partials = h->d_partials;
+      e.n_partials = h->n_partials;
+      e.partial_scale = 1.0 / (double)h->mc.n_heldout;
+      return LSGD_OK;
+    }
+    case LSGD_OBJ_PSD_COMPLETION:
+      if (!h->loss_partials_valid)   // otherwise lsgd_grad has just summed F at this x
+        LSGD_CUDA(launch_psd_grad(c.x, c.g, h->psd.M, h->psd.n, h->psd.r, c.P, c.ld, h->d_partials, h->n_partials,
+                                  false, h->d_psd_part, h->stream));
+      h->loss_partials_valid = true;
+      e.partials = h->d_partials;
+      e.n_partials = h->n_partials;
+      e.partial_scale = 0.25;
+      return LSGD_OK;
+    case LSGD_OBJ_MLP: {
+      lsgd_status st;
+      if (h->mlp.loss_window > 0) {
+        st = mlp_window_loss(h, h->d_loss);            // running mean of the training losses
+      } else {
+        if (h->fused_applied) return LSGD_ERR_STATE;   // x is between two steps: no loss at x_t any more
+        st = mlp_heldout_loss(h, h->d_loss);
+      }
+      if (st != LSGD_OK) return st;
+      e.loss_in = h->d_loss;
+      e.partials = nullptr;
+      e.n_partials = 0;
+      return LSGD_OK;
+    }
+    default:
+      return LSGD_ERR_INVALID_ARG;  // EXTERNAL has no loss of its own
+  }
+}
+
 lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
   if (!h) return LSGD_ERR_INVALID_ARG;
+  if (!on_own_device(h)) return LSGD_ERR_STATE;
   const lsgd_config& c = h->cfg;
   ElectArgs e{};
   e.loss_in = loss;
@@ -290,46 +351,23 @@ lsgd_status lsgd_elect(lsgd_handle h, const float* loss) {
     if (!e.update_local && !e.update_global) return LSGD_ERR_STATE;   // not a communication step
   }
   if (!loss) {
-    switch (c.objective) {
-      case LSGD_OBJ_QUADRATIC:
-        LSGD_CUDA(launch_quadratic_loss_partials(c.x, h->quad.a, h->quad.b, c.P, c.d, c.ld, h->d_partials,
-                                                 h->n_partials, h->stream));
-        e.partials = h->d_partials;
-        e.n_partials = h->n_partials;
-        e.partial_scale = 0.5;
-        break;
-      case LSGD_OBJ_MATCOMP: {
-        MatcompArgs a{h->mc, c.x, c.g, c.ld, c.P, h->d_status};
-        LSGD_CUDA(launch_matcomp_loss_partials(a, h->d_partials, h->n_partials, h->stream));
-        e.partials = h->d_partials;
-        e.n_partials = h->n_partials;
-        e.partial_scale = 1.0 / (double)h->mc.n_heldout;
-        break;
-      }
-      case LSGD_OBJ_PSD_COMPLETION:
-        if (!h->loss_partials_valid)   // otherwise lsgd_grad has just summed F at this x
-          LSGD_CUDA(launch_psd_grad(c.x, c.g, h->psd.M, h->psd.n, h->psd.r, c.P, c.ld, h->d_partials, h->n_partials,
-                                    false, h->d_psd_part, h->stream));
-        h->loss_partials_valid = true;
-        e.partials = h->d_partials;
-        e.n_partials = h->n_partials;
-        e.partial_scale = 0.25;
-        break;
-      case LSGD_OBJ_MLP: {
-        lsgd_status st;
-        if (h->mlp.loss_window > 0) {
-          st = mlp_window_loss(h, h->d_loss);            // running mean of the training losses
-        } else {
-          if (h->fused_applied) return LSGD_ERR_STATE;   // x is between two steps: no loss at x_t any more
-          st = mlp_heldout_loss(h, h->d_loss);
-        }
-        if (st != LSGD_OK) return st;
-        e.loss_in = h->d_loss;
-        break;
-      }
-      default:
-        return LSGD_ERR_INVALID_ARG;  // EXTERNAL has no loss of its own
-    }
+    lsgd_status st = own_election_loss(h, e);
+    if (st != LSGD_OK) return st;
+  }
+  if (alg1 && !alg1_init && !loss && e.update_local && e.update_global) {
+    // Algorithm 1, both periods due: the listing determines the global best worker after the local pull,
+    // so the objective's loss is evaluated a second time on the pulled parameters.
+    e.update_global = false;
+    LSGD_CUDA(launch_elect(e, h->stream));
+    lsgd_status st = algorithm1_pulls(h, true, false);
+    if (st != LSGD_OK) return st;
+    st = own_election_loss(h, e);
+    if (st != LSGD_OK) return st;
+    e.update_local = false;
+    e.update_global = true;
+    LSGD_CUDA(launch_elect(e, h->stream));
+    h->n_elections++;
+    return algorithm1_pulls(h, false, true);
   }
   LSGD_CUDA(launch_elect(e, h->stream));
   h->n_elections++;
@@ -415,6 +453,7 @@ lsgd_status algorithm1_pulls(lsgd_ctx* h, bool local, bool glob) {
 
 extern "C" lsgd_status lsgd_step(lsgd_handle h) {
   if (!h) return LSGD_ERR_INVALID_ARG;
+  if (!on_own_device(h)) return LSGD_ERR_STATE;
   const lsgd_config& c = h->cfg;
   const bool alg1 = (c.flags & LSGD_FLAG_ALGORITHM1) != 0;
   const bool pull = alg1 ? (c.gamma_l != 0.f || c.gamma_g != 0.f) : (h->t % c.tau) == 0;
@@ -515,6 +554,12 @@ lsgd_status lsgd_get_train_loss(lsgd_handle h, float* loss) {
   return LSGD_OK;
 }
 
+lsgd_status lsgd_mlp_get_activations(lsgd_handle h, uint16_t* h1, uint16_t* h2) {
+  if (!h || (!h1 && !h2)) return LSGD_ERR_INVALID_ARG;
+  if (h->cfg.objective != LSGD_OBJ_MLP) return LSGD_ERR_UNSUPPORTED;
+  return mlp_get_activations(h, h1, h2);
+}
+
 lsgd_status lsgd_get_step(lsgd_handle h, int64_t* t) {
   if (!h || !t) return LSGD_ERR_INVALID_ARG;
   *t = h->t;
@@ -537,6 +582,16 @@ lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out) {
   if (f) LSGD_CUDA(cudaMemset(h->d_status, 0, sizeof(f)));
   if (flag_out) *flag_out = f;
   return f ? LSGD_ERR_DEVICE_FLAG : LSGD_OK;
+}
+
+lsgd_status lsgd_selftest_wait_timeout(lsgd_handle h, int64_t budget_cycles, int32_t* gave_up) {
+  if (!h || !gave_up) return LSGD_ERR_INVALID_ARG;
+  if (budget_cycles < 1 || budget_cycles > 100000000) return LSGD_ERR_INVALID_ARG;   // at most ~50 ms
+  if (!on_own_device(h)) return LSGD_ERR_STATE;
+  LSGD_CUDA(launch_wait_timeout_selftest(h->d_status, (long long)budget_cycles, h->d_selftest, h->stream));
+  LSGD_CUDA(cudaStreamSynchronize(h->stream));
+  LSGD_CUDA(cudaMemcpy(gave_up, h->d_selftest, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return LSGD_OK;
 }
 
 lsgd_status lsgd_center(lsgd_handle h, float* center) {

@@ -11,8 +11,10 @@
 // To keep it independent of the order in which the adds land, every contribution e * y / B is evaluated
 // in fp64, converted to 2^-44 fixed point and added with 64-bit integer atomics (integer addition is
 // associative, so the sum is exact and the same on every run); a second kernel converts the sums to fp32
-// and clears the accumulator for the next step.  |contribution| < 2^4 and at most 2^15 of them meet in one
-// entry, so the 64-bit sum cannot overflow; the resolution is 5.7e-14.
+// and clears the accumulator for the next step.  The resolution is 5.7e-14.  Range: a contribution must be
+// finite and below 2^4 in magnitude, and at most 2^15 of them can meet in one entry (the batch size is capped
+// there at creation), so the 64-bit sum stays below 2^63.  A contribution outside that range -- a diverging
+// worker -- is not added; the kernel raises FLAG_OVERFLOW in the status word instead of saturating silently.
 #include "internal.h"
 
 namespace lsgd {
@@ -24,6 +26,7 @@ constexpr int kLossPerThread = 4;
 
 constexpr double kFixScale = 17592186044416.0;        // 2^44
 constexpr double kFixInv = 1.0 / 17592186044416.0;
+constexpr double kFixLimit = 16.0 * 17592186044416.0;  // 2^48: |contribution| < 2^4 in fixed-point units
 
 // A group of GROUP lanes (8, 16 or 32: the smallest that holds the rank) works on one observed entry, lane k
 // on component k of its two factor rows, so a row is fetched and its sums are updated as one contiguous piece.
@@ -69,8 +72,13 @@ matcomp_grad_kernel(MatcompArgs a, const int32_t* __restrict__ pos, unsigned lon
   const double dot = group_dot<GROUP>(xk, yk, rank, base);          // all 32 lanes take part in the shuffles
   if (mine) {
     const double e = (dot - (double)v) / (double)a.m.batch * kFixScale;
-    atomicAdd(acc + xo + k, (unsigned long long)__double2ll_rn(e * (double)yk));
-    atomicAdd(acc + yo + k, (unsigned long long)__double2ll_rn(e * (double)xk));
+    const double cx = e * (double)yk, cy = e * (double)xk;
+    if (fabs(cx) < kFixLimit && fabs(cy) < kFixLimit) {          // false for NaN and infinities too
+      atomicAdd(acc + xo + k, (unsigned long long)__double2ll_rn(cx));
+      atomicAdd(acc + yo + k, (unsigned long long)__double2ll_rn(cy));
+    } else {
+      atomicOr(a.status, FLAG_OVERFLOW);
+    }
   }
 }
 

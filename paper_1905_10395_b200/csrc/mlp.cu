@@ -590,15 +590,15 @@ lsgd_status mlp_grad(lsgd_ctx* h, const int32_t* batch_idx, bool fuse_sgd) {
   if (launch_bgemm(st->m_dh2, st->m_w2, gd, s) != cudaSuccess) return LSGD_ERR_CUDA;
   // dW3, db3, db2, db1: the sums over the batch (and, fused, the plain step of those parameters)
   const size_t sums_smem = sizeof(float) * ((size_t)B * kDzPitch + (size_t)kBwdSlices * d[3] * kBwdCols);
-  static bool sums_attr = false;
-  if (!sums_attr) {
+  static OncePerDevice sums_attr;
+  if (!sums_attr.here()) {
     if (cudaFuncSetAttribute(batch_sums_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
       return LSGD_ERR_CUDA;
     // two CTAs per SM: ask for the largest shared-memory carve-out (the default fits one CTA only)
     if (cudaFuncSetAttribute(batch_sums_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) !=
         cudaSuccess)
       return LSGD_ERR_CUDA;
-    sums_attr = true;
+    sums_attr.here() = true;
   }
   const int nb2 = (d[2] + kBwdCols - 1) / kBwdCols, nb1 = (d[1] + kBwdCols - 1) / kBwdCols;
   if (launch_pdl(batch_sums_kernel, dim3(2 * nb2 + nb1, P), dim3(kBwdThreadsX, kBwdSlices), sums_smem, s, st->h2, st->dh2, st->dh1,
@@ -664,6 +664,16 @@ lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss) {
   return cudaGetLastError() == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
 }
 
+lsgd_status mlp_get_activations(lsgd_ctx* h, uint16_t* h1, uint16_t* h2) {
+  MlpState* st = state(h);
+  if (!st) return LSGD_ERR_STATE;
+  if (cudaStreamSynchronize(h->stream) != cudaSuccess) return LSGD_ERR_CUDA;
+  const size_t n1 = (size_t)st->P * st->B * st->dims[1], n2 = (size_t)st->P * st->B * st->dims[2];
+  if (h1 && cudaMemcpy(h1, st->h1, n1 * sizeof(uint16_t), cudaMemcpyDeviceToHost) != cudaSuccess) return LSGD_ERR_CUDA;
+  if (h2 && cudaMemcpy(h2, st->h2, n2 * sizeof(uint16_t), cudaMemcpyDeviceToHost) != cudaSuccess) return LSGD_ERR_CUDA;
+  return LSGD_OK;
+}
+
 int mlp_unfused_ranges(lsgd_ctx* h, int64_t (*ranges)[2]) {
   // none: W1, W2 are stepped in the weight-gradient products, the biases and W3 in the batch-sum kernel
   (void)h;
@@ -710,17 +720,39 @@ uint64_t lsgd_mlp_scratch_bytes(const int32_t* dims, int32_t P, int32_t batch, i
   return lsgd::scratch_layout(dims, L.d, P, batch, n_heldout).total;
 }
 
+// Status word of the stand-alone product, one per device, allocated on the first use on that device.
+static uint32_t* bgemm_status_word() {
+  static uint32_t* words[lsgd::kMaxDevices] = {};
+  uint32_t*& w = words[lsgd::device_slot()];
+  if (!w) {
+    if (cudaMalloc(&w, sizeof(uint32_t)) != cudaSuccess) {
+      w = nullptr;
+      return nullptr;
+    }
+    cudaMemset(w, 0, sizeof(uint32_t));
+  }
+  return w;
+}
+
+lsgd_status lsgd_bgemm_check_device(uint32_t* flag_out) {
+  uint32_t* status = bgemm_status_word();
+  if (!status) return LSGD_ERR_CUDA;
+  uint32_t f = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return LSGD_ERR_CUDA;
+  if (cudaMemcpy(&f, status, sizeof(f), cudaMemcpyDeviceToHost) != cudaSuccess) return LSGD_ERR_CUDA;
+  if (f && cudaMemset(status, 0, sizeof(f)) != cudaSuccess) return LSGD_ERR_CUDA;
+  if (flag_out) *flag_out = f;
+  return f ? LSGD_ERR_DEVICE_FLAG : LSGD_OK;
+}
+
 lsgd_status lsgd_bgemm_bf16(const lsgd_bgemm_desc* g, void* stream) {
   using namespace lsgd;
   if (!g || !g->a || !g->b || !g->c) return LSGD_ERR_INVALID_ARG;
   if (g->M < 1 || g->N < 1 || g->K < 1 || g->batch < 1 || g->epilogue < 0 || g->epilogue > 3) return LSGD_ERR_INVALID_ARG;
   if (g->epilogue == GEMM_EPI_BIAS_RELU_BF16 && !g->bias) return LSGD_ERR_INVALID_ARG;
   if (g->epilogue == GEMM_EPI_MASK_BF16 && !g->mask) return LSGD_ERR_INVALID_ARG;
-  static uint32_t* status = nullptr;   // status word of the stand-alone entry point, allocated on first use
-  if (!status) {
-    if (cudaMalloc(&status, sizeof(uint32_t)) != cudaSuccess) return LSGD_ERR_CUDA;
-    cudaMemset(status, 0, sizeof(uint32_t));
-  }
+  uint32_t* status = bgemm_status_word();   // status word of the stand-alone entry point (per device)
+  if (!status) return LSGD_ERR_CUDA;
   CUtensorMap ma, mb;
   const int64_t a_inner = g->a_mn_major ? g->M : g->K, a_outer = g->a_mn_major ? g->K : g->M;
   const int64_t b_inner = g->b_mn_major ? g->N : g->K, b_outer = g->b_mn_major ? g->K : g->N;

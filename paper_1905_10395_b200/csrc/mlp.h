@@ -13,6 +13,8 @@ int mlp_unfused_ranges(lsgd_ctx* h, int64_t (*ranges)[2]);
 lsgd_status mlp_heldout_loss(lsgd_ctx* h, float* loss);
 lsgd_status mlp_window_loss(lsgd_ctx* h, float* loss);  // mean of the recorded minibatch losses (loss_window)
 lsgd_status mlp_train_loss(lsgd_ctx* h, float* loss);   // mean minibatch loss of the last lsgd_grad
+// stored hidden activations of the last mlp_grad as bf16 bit patterns, HOST [P][B][d1] and [P][B][d2]
+lsgd_status mlp_get_activations(lsgd_ctx* h, uint16_t* h1, uint16_t* h2);
 lsgd_status mlp_refresh_shadow(lsgd_ctx* h);             // bf16 copy of the weights <- x
 uint16_t* mlp_weight_shadow(lsgd_ctx* h);
 void mlp_destroy(lsgd_ctx* h);

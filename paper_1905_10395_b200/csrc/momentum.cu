@@ -151,13 +151,7 @@ momentum_update_kernel(UpdateArgs p, int64_t n4) {
 
 template <int MODE, bool PULL, bool SHADOW>
 cudaError_t launch_k(const UpdateArgs& a, cudaStream_t s) {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
-  }
+  const int sms = sm_count();
   const int64_t n4 = (a.d + 3) / 4;
   int64_t blocks = (n4 + kThreads - 1) / kThreads;
   const int64_t cap = (int64_t)sms * 8;

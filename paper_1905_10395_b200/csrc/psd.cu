@@ -186,13 +186,13 @@ cudaError_t launch_psd_t(const float* x, float* g, const float* M, int32_t n, in
                          int32_t n_partials, int wg, double* gpart, cudaStream_t s) {
   const int pitch = r | 1;
   const size_t smem = sizeof(double) * (size_t)(2 * T * pitch + T * (T + 1));
-  static bool attr_set = false;
-  if (!attr_set) {
+  static OncePerDevice attr;
+  if (!attr.here()) {
     cudaError_t e = cudaFuncSetAttribute(psd_grad_kernel<KM, Z>, cudaFuncAttributeMaxDynamicSharedMemorySize, 180 * 1024);
     if (e == cudaSuccess && Z > 1)   // two CTAs per SM: ask for the largest shared-memory carve-out
       e = cudaFuncSetAttribute(psd_grad_kernel<KM, Z>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr.here() = true;
   }
   dim3 grid((unsigned)(n_partials / Z), (unsigned)P, (unsigned)Z), block(TH, TH);
   psd_grad_kernel<KM, Z><<<grid, block, smem, s>>>(x, g, M, n, r, ld, partials, n_partials, wg, gpart, P);

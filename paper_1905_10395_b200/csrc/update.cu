@@ -5,7 +5,7 @@
 // values does so before anyone rewrites them, and every right-hand side is x at time t although x is updated
 // in place.  Three realisations, chosen in launch_t() / launch_momentum_update_chunked():
 //   staged   (pull_update_staged_kernel): all rows of a 3 KiB-wide tile brought into shared memory by bulk
-//            copies, for populations small enough that they fit twice (P <= 26);
+//            copies, for populations small enough that they fit twice (P <= 25 with a gradient row per worker);
 //   chunked  (update_chunked_kernel): a leader block, then the rows streamed through a ring of chunks of 8
 //            workers -- any P whose leader block fits, the inline quadratic gradient, the momentum step;
 //   register-staged (pull_update_kernel, described next): the fallback for everything else.
@@ -17,8 +17,7 @@
 // byte of x and g is read exactly once and every byte of x written exactly once (12 B per
 // worker-parameter, leaders cost nothing extra).  Because the same thread reads a leader's column
 // before it (or anyone) writes it, all right-hand sides are x at time t although x is updated in
-// place -- the simultaneous update the paper describes ("all workers are updated at the same
-// time", Section 2.2).
+// place -- the simultaneous update of all workers at a communication (Section 2.2).
 //
 // A leader's own pull term is (x - x) = 0 exactly, and fmaf(-c, 0, acc) == acc, so the leader's
 // step is bit-identical to the plain step without a branch (supplement, "Definitions and Notation":
@@ -412,17 +411,39 @@ __device__ __forceinline__ bool bar_try(uint64_t* bar, uint32_t parity) {
                : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+// Bounded wait: false once `budget` clock cycles have passed (the status word then carries FLAG_WAIT_TIMEOUT and
+// the CTA-wide abort flag is raised) or when another role of the CTA has already given up.
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t* status,
+                                         long long budget = kTmaWaitCycles) {
   if (bar_try(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (bar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kTmaWaitCycles) {
+    if (clock64() - t0 > budget) {
       *abort_flag = 1;
       atomicOr(status, FLAG_WAIT_TIMEOUT);
       return false;
     }
+  }
+}
+
+// Self-test of the bounded wait: one warp waits, with a short budget, on a barrier that nothing will ever
+// complete (no copy is in flight, nobody arrives), so the wait must run out, set the status bit and return.
+__global__ void __launch_bounds__(32)
+wait_timeout_selftest_kernel(uint32_t* status, long long budget, int* gave_up) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bar)) : "memory");
+  }
+  __syncthreads();
+  const bool ok = bar_wait(&bar, 0, &abort_flag, status, budget);
+  __syncwarp();
+  if (threadIdx.x == 0) {
+    *gave_up = ok ? 0 : 1;
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_addr(&bar)) : "memory");
   }
 }
 
@@ -545,8 +566,9 @@ pull_update_staged_kernel(UpdateArgs p, int64_t n_cols4, int W) {
 }
 
 // Tile width (floats) for the staged kernel, 0 if the shape does not suit it: all P rows of a tile of at
-// least 512 columns (2 KiB per row) must fit twice over in shared memory, i.e. P <= 26; larger populations
-// use the register-staged kernel above.
+// least 512 columns (2 KiB per row) must fit twice over in shared memory: 2 stages x 2 P rows x 2 KiB plus the
+// P-entry leader table within 208 KiB, i.e. P <= 25 when every worker brings a gradient row; larger
+// populations use the chunked or the register-staged kernel.
 inline int staged_rows(const UpdateArgs& a) { return a.P + (a.use_g ? a.P : 0) + (a.snap ? a.G + 1 : 0); }
 inline int staged_tile_width(const UpdateArgs& a) {
   if (!a.pull || (a.use_g && a.g == nullptr)) return 0;
@@ -842,12 +864,12 @@ inline ChunkShape chunk_shape(const UpdateArgs& a, bool quad, bool noise, bool m
 
 template <int MODE, bool PULL, bool QUAD, bool NOISE, bool SHADOW, bool MOM = false>
 cudaError_t launch_chunked(const UpdateArgs& a, const ChunkShape& cs, int64_t n4, int sms, cudaStream_t s) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static OncePerDevice attr;
+  if (!attr.here()) {
     cudaError_t e = cudaFuncSetAttribute(update_chunked_kernel<MODE, PULL, QUAD, NOISE, SHADOW, MOM>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kChunkSmemBudget);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr.here() = true;
   }
   const int64_t tiles = (n4 * 4 + cs.W - 1) / cs.W;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
@@ -857,23 +879,17 @@ cudaError_t launch_chunked(const UpdateArgs& a, const ChunkShape& cs, int64_t n4
 
 template <int MODE, bool QUAD, bool NOISE, bool SHADOW>
 cudaError_t launch_t(const UpdateArgs& a, cudaStream_t s) {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
-  }
+  const int sms = sm_count();
   const int64_t n4 = (a.d + 3) / 4;
   const int64_t cap = (int64_t)sms * (a.pull ? LSGD_K1_PULL_CTAS_PER_SM : LSGD_K1_PLAIN_CTAS_PER_SM);
   const int W = (QUAD || LSGD_K1_NO_STAGED) ? 0 : staged_tile_width(a);
   if (W > 0) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static OncePerDevice attr;
+    if (!attr.here()) {
       cudaError_t e = cudaFuncSetAttribute(pull_update_staged_kernel<MODE, SHADOW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            kTmaSmemBudget + 1024);
       if (e != cudaSuccess) return e;
-      attr_done = true;
+      attr.here() = true;
     }
     const size_t smem = (size_t)kTmaStages * staged_rows(a) * W * 4 + (size_t)a.P * 4;
     const int64_t tiles = (n4 * 4 + W - 1) / (W > 0 ? W : 1);
@@ -947,10 +963,7 @@ cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, i
 namespace {
 template <int MODE>
 cudaError_t launch_momentum_chunked_m(const UpdateArgs& a, const ChunkShape& cs, cudaStream_t s) {
-  int dev = 0, sms = 0;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (sms <= 0) sms = 148;
+  const int sms = sm_count();
   const int64_t n4 = (a.d + 3) / 4;
   const bool shadow = a.x_bf16 != nullptr;
   if (a.pull) return shadow ? launch_chunked<MODE, true, false, false, true, true>(a, cs, n4, sms, s)
@@ -971,6 +984,11 @@ cudaError_t launch_momentum_update_chunked(const UpdateArgs& a, cudaStream_t s) 
     case 1: return launch_momentum_chunked_m<1>(a, cs, s);
     default: return launch_momentum_chunked_m<2>(a, cs, s);
   }
+}
+
+cudaError_t launch_wait_timeout_selftest(uint32_t* status, long long budget_cycles, int* gave_up, cudaStream_t s) {
+  wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status, budget_cycles, gave_up);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_update(const UpdateArgs& a, cudaStream_t s) {

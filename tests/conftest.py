@@ -8,8 +8,13 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def pytest_addoption(parser):
+    parser.addoption("--runslow", action="store_true", default=False, help="also run the tests marked slow")
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    config.addinivalue_line("markers", "slow: exhaustive CPU checks that take minutes (run with --runslow)")
 
 
 def pytest_collection_modifyitems(config, items):
@@ -18,9 +23,10 @@ def pytest_collection_modifyitems(config, items):
         has_gpu = torch.cuda.is_available()
     except Exception:
         has_gpu = False
-    if has_gpu:
-        return
-    skip = pytest.mark.skip(reason="no CUDA device")
+    skip_slow = pytest.mark.skip(reason="slow: pass --runslow")
+    skip_gpu = pytest.mark.skip(reason="no CUDA device")
     for item in items:
-        if "gpu" in item.keywords:
-            item.add_marker(skip)
+        if "slow" in item.keywords and not config.getoption("--runslow"):
+            item.add_marker(skip_slow)
+        if "gpu" in item.keywords and not has_gpu:
+            item.add_marker(skip_gpu)

@@ -33,15 +33,15 @@ def test_struct_layout_matches_header(api, tmp_path):
     # the header compiles as plain C, and the binding's structs have the sizes the C compiler gives
     import subprocess
     src = tmp_path / "sz.c"
-    src.write_text('#include <stdio.h>\n#include "lsgd.h"\nint main(void){printf("%zu %zu %zu %zu\\n",'
+    src.write_text('#include <stdio.h>\n#include "lsgd.h"\nint main(void){printf("%zu %zu %zu %zu %zu %zu\\n",'
                    'sizeof(lsgd_config),sizeof(lsgd_quadratic_desc),sizeof(lsgd_matcomp_desc),'
-                   'sizeof(lsgd_mlp_desc));return 0;}\n')
+                   'sizeof(lsgd_mlp_desc),sizeof(lsgd_psd_desc),sizeof(lsgd_bgemm_desc));return 0;}\n')
     exe = tmp_path / "sz"
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o",
                     str(exe)], check=True)
     sizes = [int(v) for v in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()]
     assert sizes == [C.sizeof(api.Config), C.sizeof(api.QuadraticDesc), C.sizeof(api.MatcompDesc),
-                     C.sizeof(api.MlpDesc)]
+                     C.sizeof(api.MlpDesc), C.sizeof(api.PsdDesc), C.sizeof(api.BgemmDesc)]
 
 
 def _cfg(api, **over):
@@ -64,6 +64,26 @@ def test_create_rejects_bad_arguments_on_the_host(api, over, status):
     s = api.lib().lsgd_create(C.byref(cfg), C.byref(h))
     assert s == status, api.status_string(s)
     assert h.value is None
+
+
+def test_create_rejects_shapes_beyond_the_documented_capacities(api):
+    # population too large for the group tables of the register-staged pull kernel (P + 2 G + 2 > 12288)
+    P = 4096
+    cfg, keep = _cfg(api, P=P, G=P, group_of=np.arange(P))
+    h = C.c_void_p()
+    assert api.lib().lsgd_create(C.byref(cfg), C.byref(h)) == api.ERR_UNSUPPORTED
+    # matrix-completion batch beyond the range of the fixed-point accumulator
+    desc = api.MatcompDesc(10, 10, 5, 50, 4096, 4096, 4096, (1 << 15) + 1, 8, 4096)
+    cfg, keep = _cfg(api, d=100, objective=api.OBJ_MATCOMP, desc=desc)
+    assert api.lib().lsgd_create(C.byref(cfg), C.byref(h)) == api.ERR_UNSUPPORTED
+
+
+def test_device_flag_bits_match_the_header(api):
+    with open(os.path.join(ROOT, "include", "lsgd.h")) as fh:
+        header = fh.read()
+    bits = {m.group(1): int(m.group(2)) for m in re.finditer(r"#define LSGD_DEVFLAG_(\w+) (\d+)u", header)}
+    assert bits == {"BAD_LEADER": api.DEVFLAG_BAD_LEADER, "WAIT_TIMEOUT": api.DEVFLAG_WAIT_TIMEOUT,
+                    "BAD_INDEX": api.DEVFLAG_BAD_INDEX, "OVERFLOW": api.DEVFLAG_OVERFLOW}
 
 
 def test_struct_size_is_checked(api):

@@ -62,10 +62,36 @@ def test_external_ragged_unequal_groups_bit_exact():
 def test_quadratic_multi_leader_bit_exact(fused):
     w = inputs.config(1, d=(1 << 15) + 24, tau=2, steps=12)
     pop, o = _run(w, 12, fused_quadratic=fused)
+    assert any(h.get("local") and h.get("global") for h in o.history)
     for hg, ho in zip(pop.history, o.history):
-        assert np.allclose(hg["loss"], ho["loss"], rtol=3e-7, atol=0)
+        # after a communication with both periods due the library holds the second loss vector (taken after
+        # the local pull), which is the one the global election used
+        assert np.allclose(hg["loss"], ho.get("loss_global", ho["loss"]), rtol=3e-7, atol=0)
     assert np.array_equal(pop.x_host().view(np.uint32), o.x.view(np.uint32))
     pop.close()
+
+
+def test_global_leader_is_elected_after_the_local_pull():
+    """The hand-worked two-group case of tests/test_oracle_algorithm1.py (Algorithm 1, Section 2.2): the local
+    pull moves worker 1 onto the minimiser, so the global election that follows it must pick worker 1, not the
+    worker that was best before the pull."""
+    d, ld = 1, 32
+    a, b = np.zeros(ld, F32), np.zeros(ld, F32)
+    a[0] = 1.0
+    x0 = np.zeros((4, ld), F32)
+    x0[:, 0] = [2.0, -6.0, 1.8, 2.2]
+    w = inputs.Workload(name="alg1-order", objective="quadratic", P=4, G=2, d=d, ld=ld,
+                        group_of=np.asarray([0, 0, 1, 1], np.int32), eta=0.5, lambda_l=1.5, lambda_g=0.5, tau=1, steps=1,
+                        x0=x0, arrays={"a": a, "b": b, "noise": None}, meta={"sigma": 0.0})
+    alg = dict(gamma_l=0.0, gamma_g=0.0, tau_g=1)
+    for fused in (False, True):
+        pop, o = _run(w, 1, alg=alg, fused_quadratic=fused)
+        assert pop.history[-1]["gl"] == 1 and list(pop.history[-1]["ll"]) == [0, 2]
+        x = pop.x_host()
+        assert np.array_equal(x.view(np.uint32), o.x.view(np.uint32))
+        assert np.allclose(x[:, 0], [0.75, 0.0, 0.675, 0.7125], rtol=1e-6, atol=0)
+        assert np.allclose(pop.history[-1]["loss"], [0.5, 0.0, 0.405, 0.45125], rtol=1e-6)
+        pop.close()
 
 
 def test_zero_searching_scope_and_larger_shape():

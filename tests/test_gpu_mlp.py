@@ -12,6 +12,8 @@ pytestmark = pytest.mark.gpu
 
 TOL = 2e-2
 LOSS_FLOOR = 1.0     # cross-entropy has a natural O(1) scale (chance level ln 10 = 2.3)
+PARAM_FLOOR = 1e-3   # floor of the elementwise relative parameter error
+FREE_RUN_OUTLIERS = 2e-2   # free-running trajectories: fraction of entries allowed beyond the elementwise bound
 
 
 def loss_close(got, ref):
@@ -58,9 +60,33 @@ def _run_pair(w, steps, flags=0):
     return pop, o, train_gpu, train_ref, forced
 
 
+def elementwise_errors(x, ref, x_before):
+    """The elementwise figures of the parity statement for this objective:
+    parameters   |x - ref| / max(|ref|, 1e-3) for every entry of every worker (the metric of the fp32
+                 configurations, here with the 2e-2 bound of the bf16 products): its maximum, and the fraction of
+                 entries beyond 2e-2;
+    change       max |dx - dref| / max(|dref|, largest |dref| of the same worker), dx = x - x_before."""
+    e = np.abs(x - ref) / np.maximum(np.abs(ref), PARAM_FLOOR)
+    dx, dref = x - x_before, ref - x_before
+    floor = np.abs(dref).max(axis=1, keepdims=True)
+    e_delta = float((np.abs(dx - dref) / np.maximum(np.abs(dref), floor)).max())
+    return float(e.max()), float((e > TOL).mean()), e_delta
+
+
 def _check(pop, o, w, train_gpu, train_ref, forced):
+    """A FREE-RUNNING trajectory.  On this workload it amplifies differences of accumulation order by about 3x
+    per step while the losses overshoot (eta = 0.05 on inputs of norm ~60): two CPU evaluations of the oracle's
+    own definition, one accumulating in float64 and one in float32, already differ by more than 2e-2 on some
+    entries after two steps (tests/test_oracle_mlp_sensitivity.py).  So here the elementwise error is bounded in
+    the bulk (at most FREE_RUN_OUTLIERS of the entries beyond 2e-2) and norm-wise; the elementwise 2e-2 bound
+    on EVERY entry is asserted step by step from the oracle's state in
+    test_config3_every_step_from_the_oracle_state."""
     x = pop.x_host().astype(np.float64)
     ref = o.x.astype(np.float64)
+    e_param, frac, e_delta = elementwise_errors(x, ref, w.x0.astype(np.float64))
+    print(f"free-running: elementwise parameter error max {e_param:.3e}, beyond 2e-2: {frac:.3e} of the entries, "
+          f"change error {e_delta:.3e}")
+    assert frac <= FREE_RUN_OUTLIERS, (e_param, frac)
     scale = np.abs(ref).max()
     assert np.abs(x - ref).max() <= TOL * scale
     # the discriminating number: error of the parameter change, norm-wise per worker
@@ -130,30 +156,134 @@ def test_config3_mlp_population_ten_steps(fused):
     pop.close()
 
 
-def test_config3_single_steps_from_the_oracle_state():
-    """Per-step parity without the amplification of a free-running trajectory: before every step the
-    GPU parameters are set to the oracle's, so each step's losses and parameter change are compared
-    for the same x_t.  Losses here must agree to 2e-2 relative with no floor."""
-    import torch
-    from paper_1905_10395_b200.runner import Population
-    w = inputs.config(3, P=8, G=2, steps=8)
+ACC_EPS = 2.0 ** -18      # bound on the error of a float32 sum of ~1000 products, relative to sum |h||W| + |b|
+RND_EPS = 2.0 ** -8       # one bf16 unit in the last place, relative (round-to-nearest is within half of it)
+
+
+class OneWorkerMlp(orc.Mlp):
+    """The oracle's MLP objective for ONE worker (x is a single row).  With ``given`` = (h1, h2) the backward pass
+    runs on those stored hidden activations instead of the oracle's own -- everything else (the products, the
+    roundings of the deltas, the mask h > 0, the sums) is the base class's arithmetic -- and ``check_given``
+    verifies first that each given activation is a valid bf16 rounding of relu(z) for the oracle's own float64
+    pre-activation z of that layer."""
+
+    def __init__(self, base: orc.Mlp, worker: int, t: int, given=None):
+        idx = base.batch_idx[t % len(base.batch_idx)][worker]
+        super().__init__(base.segs, base.data_x, base.data_y, [[idx]], base.held_x, base.held_y)
+        self.given = given
+
+    def _forward(self, xi, inp):
+        if self.given is None:
+            return super()._forward(xi, inp)
+        Ws, bs = self._weights(xi)
+        hs = [self.rd(inp).astype(np.float64)] + [np.asarray(h, dtype=np.float64) for h in self.given]
+        return Ws, hs, hs[-1] @ Ws[-1].T + bs[-1]
+
+    def check_given(self, xi):
+        """Layer by layer, from the GIVEN input of that layer: |h - relu(z)| <= one bf16 ulp of |z| plus the
+        accumulation bound (which also covers a ReLU decision taken within rounding of zero)."""
+        Ws, bs = self._weights(xi)
+        inp = self.rd(self.data_x[self.batch_idx[0][0]]).astype(np.float64)
+        worst = 0.0
+        for l, h in enumerate(self.given):
+            z = inp @ Ws[l].T + bs[l]
+            slack = RND_EPS * np.abs(z) + ACC_EPS * (np.abs(inp) @ np.abs(Ws[l]).T + np.abs(bs[l]))
+            worst = max(worst, float((np.abs(h - np.maximum(z, 0.0)) / np.maximum(slack, 1e-300)).max()))
+            inp = np.asarray(h, dtype=np.float64)
+        return worst
+
+
+def _row_after_step(x_t, i, g_i, o, w, pull):
+    """Worker i's parameters after the step of Eq. (1) from state x_t with gradient g_i and the oracle's leaders."""
+    if not pull:
+        sub = x_t[i:i + 1].copy()
+        orc.update(sub, g_i[None, :], [0], (), -1, w.eta, w.lambda_l, w.lambda_g, False)
+        return sub[0]
+    ll_i = int(o.ll[int(w.group_of[i])])
+    sub = np.stack([x_t[i], x_t[ll_i], x_t[int(o.gl)]])
+    g = np.zeros_like(sub)
+    g[0] = g_i
+    orc.update(sub, g, [0, 0, 0], [1], 2, w.eta, w.lambda_l, w.lambda_g, True)
+    return sub[0]
+
+
+def _a17_rows(x, ref):
+    return (np.abs(x.astype(np.float64) - ref) / np.maximum(np.abs(ref.astype(np.float64)), PARAM_FLOOR)).max(axis=1)
+
+
+def test_one_worker_objective_is_the_oracle_objective():
+    # the helper above is the oracle's arithmetic: bit-identical gradients without given activations, and with
+    # the oracle's own activations given back to it
+    w = inputs.make_mlp(3, 1, dims=(40, 72, 136, 7), pool=256, heldout=40, batch=24, n_classes=7, steps=2, tau=1,
+                        config_id=84)
     o = _oracle(w)
-    pop = Population(w)
-    for t in range(8):
+    g = o.obj.grad(w.x0, 1)
+    for i in range(w.P):
+        one = OneWorkerMlp(o.obj, i, 1)
+        gi = one.grad(w.x0[i:i + 1], 0)[0]
+        assert np.array_equal(gi.view(np.uint32), g[i].view(np.uint32))
+        _, hs, _ = one._forward(w.x0[i], one.data_x[one.batch_idx[0][0]])
+        again = OneWorkerMlp(o.obj, i, 1, given=(hs[1], hs[2]))
+        assert again.check_given(w.x0[i]) <= 1.0
+        assert np.array_equal(again.grad(w.x0[i:i + 1], 0)[0].view(np.uint32), g[i].view(np.uint32))
+        bad = hs[1].copy()
+        bad[3, 5] = bad[3, 5] * 1.05 + 0.01                      # not a rounding of relu(z): must be noticed
+        assert OneWorkerMlp(o.obj, i, 1, given=(bad, hs[2])).check_given(w.x0[i]) > 1.0
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_config3_every_step_from_the_oracle_state(fused):
+    """Element-by-element parity of the whole configuration (32 workers, 4 groups, 10 steps) without the
+    amplification of a free-running trajectory: before every step the GPU parameters are set to the oracle's x_t,
+    so each step is compared for the same state.  Every entry of every worker's parameters must agree within
+    2e-2 relative (|x - ref| / max(|ref|, 1e-3)), the training and held-out losses within 2e-2 relative with no
+    floor, and the leaders exactly.
+
+    One thing is not unique.  A hidden activation is a decision taken in floating point: which bf16 neighbour a
+    sum is rounded to and, for a pre-activation within rounding of zero, whether the unit is on at all -- and the
+    ReLU mask gates that sample's whole back-propagated delta.  The kernel takes these decisions on float32
+    sums, the oracle on float64 sums.  So (1) for every worker and step the activations the kernel stored are
+    checked, entry by entry, to be valid roundings of relu(z) for the oracle's own float64 z of that layer; and
+    (2) a worker whose parameters miss the bound against the oracle's own decisions is compared instead, entry by
+    entry within the same 2e-2, with the oracle's backward pass run on those (verified) stored activations."""
+    import torch
+    from paper_1905_10395_b200 import api
+    from paper_1905_10395_b200.runner import Population
+    w = inputs.config(3, steps=10)
+    dims, B = w.meta["dims"], w.meta["batch"]
+    o = _oracle(w)
+    pop = Population(w, flags=api.FLAG_MLP_FUSED_STEP if fused else 0)
+    worst, worst_act, followed = 0.0, 0.0, 0
+    for t in range(10):
         x_t = o.x.copy()
         pop.x.copy_(torch.from_numpy(x_t))
         pop.lsgd.sync_parameters()
         o.step()
         pop.step(record=True)
+        pull = t % w.tau == 0
         assert np.allclose(pop.lsgd.train_loss(), o.obj.last_train_loss, rtol=TOL, atol=0), t
-        if t % w.tau == 0:
+        if pull:
             hg, ho = pop.history[-1], o.history[-1]
             assert np.allclose(hg["loss"], ho["loss"], rtol=TOL, atol=0), t
             assert hg["gl"] == ho["gl"] and np.array_equal(hg["ll"], ho["ll"]), t
-        dx = pop.x_host().astype(np.float64) - x_t
-        dref = o.x.astype(np.float64) - x_t
+        xg = pop.x_host()
+        h1, h2 = pop.lsgd.mlp_activations(B, dims[1], dims[2])
+        e_rows = _a17_rows(xg, o.x)
         for i in range(w.P):
-            assert np.linalg.norm(dx[i] - dref[i]) <= TOL * np.linalg.norm(dref[i]), (t, i)
+            one = OneWorkerMlp(o.obj, i, t, given=(h1[i], h2[i]))
+            act = one.check_given(x_t[i])
+            worst_act = max(worst_act, act)
+            assert act <= 1.0, (t, i, act)
+            if e_rows[i] > TOL:
+                g_i = one.grad(x_t[i:i + 1], 0)[0]
+                e = float(_a17_rows(xg[i:i + 1], _row_after_step(x_t, i, g_i, o, w, pull)[None, :])[0])
+                assert e <= TOL, (t, i, float(e_rows[i]), e)
+                e_rows[i] = e
+                followed += 1
+        worst = max(worst, float(e_rows.max()))
+    print(f"step by step: worst elementwise parameter error {worst:.3e}; stored activations within {worst_act:.3f} of "
+          f"their rounding bound; {followed} worker-steps of {10 * w.P} compared on the kernel's stored decisions")
+    assert pop.lsgd.check_device() == 0
     pop.close()
 
 

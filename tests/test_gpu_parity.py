@@ -187,17 +187,25 @@ def test_config1_reduced_multi_leader_quadratic(fused, arith):
     pop.close()
 
 
-def test_config1_full_size_ten_steps():
+def test_config1_full_size_at_step_10_and_step_100():
+    """The whole configuration: 64 workers in 8 groups, d = 2^20, tau = 4, the noise ring reused cyclically,
+    compared on every entry after 10 steps and again at the end of the 100-step run."""
     w = inputs.config(1)
     pop = _pop(w, fused_quadratic=True)
-    pop.run(10, record=True)
     o = _oracle(w)
-    o.run(10)
-    _leaders_equal(pop, o)
-    for hg, ho in zip(pop.history, o.history):
-        assert np.allclose(hg["loss"], ho["loss"], rtol=3e-7, atol=0)
-    x = pop.x_host()
-    assert rel_err(x, o.x) <= TOL
+    done = 0
+    for upto in (10, 100):
+        pop.run(upto - done, record=True)
+        o.run(upto - done)
+        done = upto
+        _leaders_equal(pop, o)
+        for hg, ho in zip(pop.history, o.history):
+            assert np.allclose(hg["loss"], ho["loss"], rtol=3e-7, atol=0), (upto, hg["t"])
+        x = pop.x_host()
+        e = rel_err(x, o.x)
+        assert e <= TOL, (upto, e)
+    assert len(o.history) == 25
+    assert pop.lsgd.check_device() == 0
     pop.close()
 
 

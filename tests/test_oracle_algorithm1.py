@@ -101,3 +101,60 @@ def test_small_pulls_use_the_stale_copies_not_the_moving_leader():
     o.run(3)
     assert np.array_equal(o.z_l[0], z0)                   # not refreshed between communications
     assert not np.array_equal(o.x[int(o.ll[0])], z0)      # while the leader itself has moved on
+
+
+def _two_group_case():
+    """One coordinate, f(x) = x^2 / 2, eta = 1/2, groups {0, 1} and {2, 3}, both periods 1, no small pulls.
+    Worked by hand (every value below is exact in binary or differs by one rounding):
+      x_0                = [ 2,  -6,  1.8,   2.2 ]   losses [2, 18, 1.62, 2.42]: local leaders 0 and 2, global 2
+      gradient step x/2  = [ 1,  -3,  0.9,   1.1 ]   losses [0.5, 4.5, 0.405, 0.605]: local leaders 0 and 2
+      local pull, eta lambda = 3/4:
+                           [ 1,   0,  0.9,   0.95]   losses [0.5, 0, 0.405, 0.45125]: worker 1 is now the best
+      global pull towards worker 1 (x = 0), eta lambda_G = 1/4:
+                           [0.75, 0,  0.675, 0.7125]
+    Electing the global leader from the losses taken before the local pull would pick worker 2 instead."""
+    a, b = np.ones(1, F32), np.zeros(1, F32)
+    x0 = np.asarray([[2.0], [-6.0], [1.8], [2.2]], dtype=F32)
+    obj = orc.Quadratic(a, b, 0.0, None)
+    return orc.Algorithm1Oracle(x0, obj, [0, 0, 1, 1], 2, eta=0.5, lambda_l=1.5, lambda_g=0.5, gamma_l=0.0, gamma_g=0.0,
+                                tau=1, tau_g=1)
+
+
+def test_global_leader_is_elected_after_the_local_pull():
+    """Algorithm 1 (Section 2.2): the second conditional of a communication follows the first one's pull, so
+    the global best worker is determined on the parameters the local pull has produced."""
+    o = _two_group_case()
+    assert list(o.ll) == [0, 2] and o.gl == 2
+    o.step()
+    h = o.history[-1]
+    assert h["local"] and h["global"]
+    assert list(o.ll) == [0, 2]
+    assert o.gl == 1                                             # not 2: the local pull moved worker 1 to the minimiser
+    assert np.allclose(h["loss"], [0.5, 4.5, 0.405, 0.605], rtol=1e-6)
+    assert np.allclose(h["loss_global"], [0.5, 0.0, 0.405, 0.45125], rtol=1e-6)
+    assert np.allclose(o.x[:, 0], [0.75, 0.0, 0.675, 0.7125], rtol=1e-6, atol=0)
+    assert np.array_equal(o.z_g, o.x[1]) and np.array_equal(o.z_l[0], o.x[0] / F32(0.75))
+
+
+def test_a_supplied_loss_vector_serves_both_elections():
+    o = _two_group_case()
+    o.step(forced_loss=np.asarray([3.0, 4.0, 1.0, 2.0], dtype=F32))
+    assert list(o.ll) == [0, 2] and o.gl == 2
+    h = o.history[-1]
+    assert np.array_equal(h["loss"], h["loss_global"])
+
+
+def test_one_loss_vector_for_both_elections_would_fail_the_hand_worked_case(monkeypatch):
+    """Plants the shortcut (global argmin from the losses taken before the local pull) in the oracle and
+    checks that the hand-worked case above catches it."""
+    real = orc.Quadratic.loss
+    cache = {}
+
+    def loss_once_per_communication(self, x, n):
+        if n not in cache:
+            cache[n] = real(self, x, n)
+        return cache[n]
+
+    monkeypatch.setattr(orc.Quadratic, "loss", loss_once_per_communication)
+    with pytest.raises(AssertionError):
+        test_global_leader_is_elected_after_the_local_pull()

@@ -209,6 +209,46 @@ def test_election_matches_brute_force_exhaustively():
                 assert gl == _brute_argmin(loss, list(range(P)))
 
 
+def _set_partitions(P):
+    """Every grouping of P workers up to renaming the groups (restricted-growth strings)."""
+    def rec(prefix, n_used):
+        if len(prefix) == P:
+            yield tuple(prefix)
+            return
+        for j in range(n_used + 1):
+            yield from rec(prefix + [j], max(n_used, j + 1))
+    yield from rec([], 0)
+
+
+def _exhaustive_election(P):
+    vals = [-1.0, -0.0, 0.0, 1.0, math.inf, math.nan]
+    parts = [(m, max(m) + 1, [[i for i in range(P) if m[i] == j] for j in range(max(m) + 1)])
+             for m in _set_partitions(P)]
+    for combo in itertools.product(vals, repeat=P):
+        loss = np.asarray(combo, dtype=F32)
+        best = {}
+        for m, G, members in parts:
+            ll, gl = orc.elect(loss, m, G)
+            for j in range(G):
+                key = tuple(members[j])
+                if key not in best:
+                    best[key] = _brute_argmin(loss, members[j])
+                assert ll[j] == best[key], (combo, m)
+            key = tuple(range(P))
+            if key not in best:
+                best[key] = _brute_argmin(loss, list(range(P)))
+            assert gl == best[key], (combo, m)
+
+
+def test_election_matches_brute_force_five_workers_all_groupings():
+    _exhaustive_election(5)                                # 6^5 loss vectors x 52 groupings
+
+
+@pytest.mark.slow
+def test_election_matches_brute_force_six_workers_all_groupings():
+    _exhaustive_election(6)                                # 6^6 loss vectors x 203 groupings; run with --runslow
+
+
 def test_election_tie_examples():
     ll, gl = orc.elect(np.asarray([0.5, 0.5, 0.25, 0.25], F32), [0, 0, 1, 1], 2)
     assert list(ll) == [0, 2] and gl == 2

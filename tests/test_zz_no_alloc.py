@@ -8,6 +8,7 @@ still in the shared array -- and an over-capacity problem is refused.  Collected
 import numpy as np
 import pytest
 
+from oracle import lsgd_oracle as orc
 from paper_1905_10395_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -34,8 +35,8 @@ def test_noalloc_loss_matches_regular_entry_point_twice_in_a_row():
                                         torch.cuda.current_stream().cuda_stream)
         got = out.cpu().numpy()
         assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), (call, got, want)
-        # and against the defining formula, within the tolerance the parity tests use for losses
-        ref = 0.5 * (w.arrays["a"].astype(np.float64) * (w.x0.astype(np.float64) - w.arrays["b"]) ** 2).sum(axis=1)
+        # and against the oracle's election loss, within the tolerance the parity tests use for losses
+        ref = orc.Quadratic(w.arrays["a"], w.arrays["b"], w.meta["sigma"], None).loss(w.x0, 0)
         assert np.allclose(got, ref, rtol=3e-7, atol=0)
         pop.close()
 
