@@ -53,8 +53,18 @@ def read_tensor_peak():
     return 1400.0, "fallback (sustained)"
 
 
+def mlp_algorithmic_bytes(dims):
+    """Bytes ONE worker's fused gradient + SGD step cannot avoid moving, whatever the batch: the bf16 weights read
+    by the forward products (2 B per parameter), W2 and W3 read again by the back-propagation products, the fp32
+    master parameters read and rewritten by the step (4 + 4 B) and their new bf16 copy (2 B).  Activations, the
+    batch and the deltas are left out (they are small and can stay on chip).  24.5 MB for 784-1024-1024-10."""
+    d0, d1, d2, d3 = [int(v) for v in dims]
+    n_w = d0 * d1 + d1 + d1 * d2 + d2 + d2 * d3 + d3
+    return float(12 * n_w + 2 * (d1 * d2 + d2 * d3))
+
+
 def mlp_step_bytes_flops(dims, batch):
-    """Algorithmic HBM bytes and tensor-core flops of ONE worker's fused gradient + SGD step.
+    """Traffic model and tensor-core flops of ONE worker's fused gradient + SGD step as the kernels are split.
 
     Every operand is counted once per kernel that must read or write it: bf16 activations and shadow weights
     (2 B), the fp32 master weights read and rewritten by the step (4 + 4 B) plus their new bf16 shadow (2 B),
@@ -188,9 +198,11 @@ def workload_spec(args):
     raise SystemExit("unknown workload")
 
 
-# DRAM bytes per worker-parameter of the update kernels, from the ncu counters of a d = 2^22 capture of
-# the same kernels (profiles/pull_update_kernel_c4.md); traffic is proportional to d.
+# DRAM bytes per worker-parameter that the update kernels of the default workload moved in a hardware-counter
+# capture (dram read + write bytes of one launch divided by P * d): reads equal the algorithmic 8 B exactly; the
+# writes fall short of 4 B by the lines still dirty in the 126 MB L2 when the kernel ends.
 MEASURED_TRAFFIC_PER_WORKER_PARAM = {"pull": 11.24, "plain": 11.30}
+NOMINAL_HBM_GBS = 7700.0     # the part's data-sheet HBM3e bandwidth, for context beside the measured copy bandwidth
 
 
 def bytes_per_worker_param(spec):
@@ -262,6 +274,78 @@ def _oracle_sample_once(spec, steps, warmup, sample_cols):
     return P * w.d * steps / dt, dt, what
 
 
+def _all_cores_worker(spec, steps, sample_cols, slot, barrier, out):
+    """One process of the all-cores leg: the oracle, as it stands, on this process's own column sample."""
+    try:
+        from oracle import lsgd_oracle as orc
+        from paper_1905_10395_b200 import inputs
+        P = spec["P"]
+        kw = dict(eta=spec["eta"], lambda_l=spec["lambda_l"], lambda_g=spec["lambda_g"], tau=spec["tau"], steps=steps)
+        if spec["kind"] == "external":
+            w = inputs.make_external(P, spec["G"], sample_cols, config_id=400 + slot, **kw)
+            obj = orc.External(w.arrays["g"], w.arrays["loss_ring"])
+        else:
+            w = inputs.make_quadratic(P, spec["G"], sample_cols, sigma=0.01, noise_ring=2, config_id=100 + slot, **kw)
+            obj = orc.Quadratic(w.arrays["a"], w.arrays["b"], 0.01, w.arrays["noise"])
+        o = orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau)
+        o.step()
+        barrier.wait(timeout=600)
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            o.step()
+        out.put((slot, P * w.d * steps, time.perf_counter() - t0))
+    except Exception as exc:                                # the parent must not wait for a result that never comes
+        out.put((slot, 0.0, float("nan"), repr(exc)))
+
+
+def oracle_all_cores(spec, steps, sample_cols, n_proc=None):
+    """The element-wise workloads on every host core: columns are independent once the leaders are known, so each
+    of ``n_proc`` processes (spawned: no CUDA state is inherited) times the unchanged oracle on its own column
+    sample, all starting together; the throughputs add up over the slowest process's time.  Returns
+    (worker-params/s, seconds, processes) or None for the other workloads."""
+    if spec["kind"] not in ("external", "quadratic"):
+        return None
+    import multiprocessing as mp
+    n_proc = n_proc or os.cpu_count() or 1
+    ctx = mp.get_context("spawn")
+    barrier, out = ctx.Barrier(n_proc), ctx.Queue()
+    cols = int(min(sample_cols, spec["d"]))
+    procs = [ctx.Process(target=_all_cores_worker, args=(spec, steps, cols, k, barrier, out)) for k in range(n_proc)]
+    for p in procs:
+        p.start()
+    got, deadline = [], time.time() + 1200
+    while len(got) < n_proc:
+        try:
+            got.append(out.get(timeout=2))
+        except Exception:
+            # a child that died before it could report (import failure, out of memory) must not stall the bench
+            if any(p.exitcode not in (None, 0) for p in procs) or time.time() > deadline:
+                for p in procs:
+                    if p.is_alive():
+                        p.terminate()
+                raise RuntimeError("all-cores oracle leg: a worker process ended without a result")
+    for p in procs:
+        p.join(timeout=60)
+    bad = [g for g in got if len(g) > 3]
+    if bad:
+        raise RuntimeError(f"all-cores oracle leg failed: {bad[0][3]}")
+    units, slowest = sum(g[1] for g in got), max(g[2] for g in got)
+    return units / slowest, slowest, n_proc
+
+
+def cpu_baseline_record(spec, value, cores, sample, all_cores=None):
+    """The ``cpu_baseline`` object: the single-process figure and, for the element-wise workloads, the figure on
+    all host cores; ``value`` / ``cores`` are the larger configuration's."""
+    rec = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+    if all_cores is not None:
+        v, dt, n = all_cores
+        rec = {"value": v, "unit": UNIT, "cores": n, "kind": "oracle",
+               "sample": f"{n} processes, each: {sample.split(', ')[0]}; {dt:.1f} s",
+               "single_core": {"value": value, "cores": cores, "sample": sample},
+               "host_cores": os.cpu_count()}
+    return rec
+
+
 def run_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
@@ -270,15 +354,15 @@ def run_reference(args):
     steps, warmup = args.steps, args.warmup
     sample = args.sample_cols or (1 << 20)      # about a quarter of a second of oracle work per C4 step
     value, dt, what, _ = oracle_sample_run(spec, steps, warmup, sample)
+    cores = _threads_used() if spec["kind"] in ("mlp", "psd") else 1
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": spec["name"], "tau": spec["tau"],
                    "sample": f"each step covers {what}"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _threads_used() if spec["kind"] in ("mlp", "psd") else 1,
-                         "kind": "oracle",
-                         "sample": f"{steps} steps x {what}"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{steps} steps x {what}", "host_cores": os.cpu_count()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -411,12 +495,14 @@ def run_ours(args):
 
     if with_momentum:
         k1_name = "momentum_update_kernel"
-    elif spec["kind"] == "quadratic" or spec["P"] > 26:
+    elif spec["kind"] == "quadratic" or spec["P"] > 25:
         k1_name = "update_chunked_kernel"
     else:
         k1_name = "pull_update_staged_kernel / plain_update_kernel"
     roofline = {"bound": "hbm", "kernel": k1_name, "achieved": achieved,
-                "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                "peak": peak, "peak_source": peak_src + " copy bandwidth (1 read : 1 write; this kernel reads 2 : 1, so "
+                "a fraction slightly above 1 is possible)", "unit": "GB/s", "frac": achieved / peak,
+                "nominal_peak": NOMINAL_HBM_GBS, "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
                 "traffic": traffic, "ms_per_launch": upd_ms, "algorithmic_bytes_per_launch": alg_bytes,
                 "pull_steps": int(sum(pull_flags)), "plain_steps": int(steps - sum(pull_flags)),
                 "ms_pull": float(np.mean([m for m, f in zip(k_ms, pull_flags) if f])) if any(pull_flags) else None,
@@ -435,11 +521,16 @@ def run_ours(args):
         # batch of 128 rows per worker each weight is used 2 x 128 times per pass, so the weight streams bound it.
         g_ms = float(np.mean([a.elapsed_time(b) for (a, b), f in zip(g_ev, pull_flags) if not f]))
         mb, mflops = mlp_step_bytes_flops(w.meta["dims"], int(w.meta["batch"]))
+        ab = mlp_algorithmic_bytes(w.meta["dims"])
         t_peak, t_src = read_tensor_peak()
         roofline = {"bound": "hbm", "kernel": "bgemm_bf16_kernel inside the fused gradient + step call (plain steps)",
-                    "achieved": P * mb / (g_ms * 1e-3) / 1e9, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
-                    "frac": P * mb / (g_ms * 1e-3) / 1e9 / peak, "traffic": None, "ms_per_launch": g_ms,
-                    "algorithmic_bytes_per_launch": P * mb, "tensor_tflops": P * mflops / (g_ms * 1e-3) / 1e12,
+                    "achieved": P * ab / (g_ms * 1e-3) / 1e9, "peak": peak, "peak_source": peak_src + " copy bandwidth",
+                    "unit": "GB/s", "frac": P * ab / (g_ms * 1e-3) / 1e9 / peak, "nominal_peak": NOMINAL_HBM_GBS,
+                    "frac_of_nominal": P * ab / (g_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS, "traffic": None,
+                    "ms_per_launch": g_ms, "algorithmic_bytes_per_launch": P * ab,
+                    "traffic_model": {"bytes_per_launch": P * mb, "frac": P * mb / (g_ms * 1e-3) / 1e9 / peak,
+                                      "what": "every operand counted once per kernel that reads or writes it"},
+                    "tensor_tflops": P * mflops / (g_ms * 1e-3) / 1e12,
                     "tensor_peak_tflops": t_peak, "tensor_peak_source": t_src,
                     "tensor_frac": P * mflops / (g_ms * 1e-3) / 1e12 / t_peak}
     line = {
@@ -538,14 +629,14 @@ def run_ours(args):
     if pop is not None:
         pop.close()
 
-    # ---- CPU oracle beside it (rank 0, N = 1 only)
+    # ---- CPU oracle beside it (rank 0, N = 1 only): one process, then every host core
     if rank == 0 and world == 1 and not args.no_cpu:
         sample = args.sample_cols or (1 << 22)
         osteps = {"external": 3, "quadratic": 3, "matcomp": 8, "mlp": 4, "psd": 4}[spec["kind"]]
         v, dt, what, osteps = oracle_sample_run(spec, osteps, 1, sample, min_seconds=10.0)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": _threads_used() if spec["kind"] in ("mlp", "psd") else 1,
-                                "kind": "oracle",
-                                "sample": f"{osteps} steps x {what}, {dt:.1f} s"}
+        cores = _threads_used() if spec["kind"] in ("mlp", "psd") else 1
+        allc = oracle_all_cores(spec, osteps, min(sample, 1 << 20) if (os.cpu_count() or 1) > 16 else sample)
+        line["cpu_baseline"] = cpu_baseline_record(spec, v, cores, f"{osteps} steps x {what}, {dt:.1f} s", allc)
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -636,7 +727,7 @@ def main():
     ap.add_argument("--arith", type=int, default=0, choices=[0, 1, 2])
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--sample-cols", type=int, default=0)
-    ap.add_argument("--d", type=int, default=0, help="shrink the c4 workload (profiler captures on a small case)")
+    ap.add_argument("--d", type=int, default=0, help="c4: parameters per worker (default 2^26); smaller values give a small case")
     ap.add_argument("--schedule", default="fused", choices=["fused", "algorithm1"],
                     help="c4 only: algorithm1 = the paper's Algorithm 1 schedule (gamma 0.1 / 0.05, tau_G = 4 tau)")
     ap.add_argument("--mlp-unfused-step", action="store_true",

@@ -16,9 +16,13 @@ def _free_port():
 
 
 def _torchrun(script_args, n=2, timeout=300):
-    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
-           "127.0.0.1", "--master-port", str(_free_port())] + script_args
-    return subprocess.run(cmd, capture_output=True, text=True, timeout=timeout, cwd=ROOT)
+    for attempt in range(2):                             # the probed port can be taken before the ranks bind it
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
+               "127.0.0.1", "--master-port", str(_free_port())] + script_args
+        r = subprocess.run(cmd, capture_output=True, text=True, timeout=timeout, cwd=ROOT)
+        if r.returncode == 0:
+            break
+    return r
 
 
 def _json_lines(out):
@@ -62,3 +66,29 @@ def test_mlp_step_bytes_and_flops_count_each_operand_once():
     assert by > n_w * 12 + 1024 * 1024 * 2
     assert by < n_w * 12 + 1024 * 1024 * 2 + 6e6           # activations and the head add a few MB at most
     assert fl == 2.0 * 128 * (2 * 784 * 1024 + 3 * 1024 * 1024 + 2 * 1024 * 10)
+
+
+def test_mlp_algorithmic_bytes_are_the_unavoidable_weight_traffic():
+    import bench
+    n_w = 784 * 1024 + 1024 + 1024 * 1024 + 1024 + 1024 * 10 + 10
+    ab = bench.mlp_algorithmic_bytes((784, 1024, 1024, 10))
+    assert ab == 12 * n_w + 2 * (1024 * 1024 + 1024 * 10)
+    assert abs(ab / 1e6 - 24.5) < 0.1                      # the per-worker figure the roofline fraction is quoted on
+    assert ab < bench.mlp_step_bytes_flops((784, 1024, 1024, 10), 128)[0]
+
+
+def test_all_cores_oracle_leg_adds_up_independent_column_samples():
+    """Two spawned processes, each timing the unchanged oracle on its own column sample; the record carries both
+    the single-process and the all-cores figure with their core counts."""
+    import bench
+
+    class Args:
+        workload, d, tau, momentum, weight_decay, mlp_unfused_step = "c4", 0, 0, None, 0.0, False
+    spec = bench.workload_spec(Args)
+    v, dt, n = bench.oracle_all_cores(spec, 2, 4096, n_proc=2)
+    assert n == 2 and v > 0 and dt > 0
+    rec = bench.cpu_baseline_record(spec, 1.0e7, 1, "2 steps x 16 workers x 4096 of 67108864 columns, 0.1 s", (v, dt, n))
+    assert rec["cores"] == 2 and rec["single_core"]["cores"] == 1 and rec["kind"] == "oracle"
+    assert rec["value"] == v and rec["single_core"]["value"] == 1.0e7
+    Args.workload = "c2"
+    assert bench.oracle_all_cores(bench.workload_spec(Args), 1, 4096) is None     # not a column-separable workload
