@@ -526,3 +526,60 @@ class Algorithm1Oracle:
         for _ in range(steps):
             self.step()
         return self.x
+
+
+# ----------------------------------------------------------------------------------------------
+# EAGD / EASGD, the elastic-averaging comparison line of the paper's matrix-completion experiment
+# ----------------------------------------------------------------------------------------------
+def eagd_center_update(center: np.ndarray, x: np.ndarray, eta: float, lam: float) -> np.ndarray:
+    """X~+ = (1 - p eta lambda) X~ + p eta lambda (1/p sum_i X^i)  (supplement, "Low-Rank Matrix Completion
+    Experiments"), p = number of workers.  Evaluated in float64 as printed -- k = (p eta) lambda, the mean as
+    the worker-order sum times 1/p, then (1 - k) X~ + k mean -- and rounded once."""
+    eta, lam = float(F32(eta)), float(F32(lam))
+    p = x.shape[0]
+    k = (p * eta) * lam
+    acc = np.zeros(x.shape[1], dtype=F64)
+    for i in range(p):
+        acc = acc + x[i].astype(F64)
+    mean = acc * (1.0 / p)
+    return ((1.0 - k) * center.astype(F64) + k * mean).astype(F32)
+
+
+class EagdOracle:
+    """Elastic averaging (S)GD as the paper states it beside LGD: every worker takes the same step as in LGD,
+    X+ = (1 - eta lambda) X + eta lambda Z - eta grad F(X), but towards Z = X~, a center variable that is itself
+    updated by ``eagd_center_update``.  Communication every tau steps (the paper's experiment uses tau = 1);
+    plain (S)GD steps in between, as for LSGD.
+
+    Readings (the paper does not say): all right-hand sides of a communication step are taken at time t -- the
+    workers move towards the old center while the center moves towards the old workers' mean; the center starts
+    at the mean of the workers' starting points (with that start and 100 iterations the supplement's toy problem
+    gives the printed EAGD value)."""
+
+    def __init__(self, x0, objective, eta, lam, tau=1):
+        self.x = np.array(x0, dtype=F32, copy=True)
+        self.obj = objective
+        self.eta, self.lam, self.tau = eta, lam, int(tau)
+        self.t = 0
+        self.center = center_variable(self.x)
+
+    def step(self) -> None:
+        g = self.obj.grad(self.x, self.t)
+        P = self.x.shape[0]
+        if self.t % self.tau == 0:
+            new_center = eagd_center_update(self.center, self.x, self.eta, self.lam)
+            # the workers' step is the pull form of Eq. (1) with the center as the only guide point: run it on the
+            # population extended by the center as a row that is everybody's leader (its own step is x - eta 0)
+            ext = np.concatenate([self.x, self.center[None, :]], axis=0)
+            gext = np.concatenate([g, np.zeros_like(self.center)[None, :]], axis=0)
+            update(ext, gext, [0] * (P + 1), [P], P, self.eta, 0.0, self.lam, True)
+            self.x = ext[:P]
+            self.center = new_center
+        else:
+            update(self.x, g, [0] * P, (), -1, self.eta, 0.0, 0.0, False)
+        self.t += 1
+
+    def run(self, steps: int) -> np.ndarray:
+        for _ in range(steps):
+            self.step()
+        return self.x

@@ -137,6 +137,9 @@ struct MatcompArgs {
 cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, bool finish, cudaStream_t s);
 cudaError_t launch_matcomp_finish_step(unsigned long long* acc, float* x, int32_t P, int64_t ld, double eta, int arith,
                                        cudaStream_t s);
+// the same step, visiting only the entries of the batch `pos` that produced the sums (pos must still be valid)
+cudaError_t launch_matcomp_step_from_batch(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, float* x,
+                                           double eta, int arith, cudaStream_t s);
 int32_t matcomp_loss_blocks(int32_t n_heldout);
 cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials, int32_t n_partials,
                                          cudaStream_t s);
@@ -217,5 +220,6 @@ struct lsgd_ctx {
   void* mlp_state;           // opaque MLP pipeline state
   unsigned long long* d_acc64;  // MATCOMP: fixed-point gradient accumulator [P*ld], kept all-zero between steps
   bool mc_step_pending;         // MATCOMP fused step: the gradient sums wait in d_acc64 for lsgd_step
+  const int32_t* mc_pending_pos;  // ... and this is the batch that produced them (caller's DEVICE pointer)
   double* d_psd_part;           // PSD, small ranks: partial gradients of the CTAs that share a row block
 };

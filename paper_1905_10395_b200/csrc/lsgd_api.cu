@@ -11,6 +11,9 @@ using namespace lsgd;
 
 namespace {
 
+#ifndef LSGD_MATCOMP_SCAN_STEP
+#define LSGD_MATCOMP_SCAN_STEP 0   // 1: the fused matrix-completion step scans the whole accumulator instead of the batch
+#endif
 constexpr int32_t kMaxWorkers = 4096;  // group tables live in shared memory of the update kernel
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -128,6 +131,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->grad_ready = false;
   h->fused_applied = false;
   h->mc_step_pending = false;
+  h->mc_pending_pos = nullptr;
   h->armed_noise = nullptr;
   h->slab = nullptr;
   h->mlp_state = nullptr;
@@ -251,6 +255,7 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
                         (h->t % c.tau) != 0;
       LSGD_CUDA(launch_matcomp_grad(a, static_cast<const int32_t*>(batch), h->d_acc64, !fuse, h->stream));
       h->mc_step_pending = fuse;
+      h->mc_pending_pos = static_cast<const int32_t*>(batch);
       break;
     }
     case LSGD_OBJ_PSD_COMPLETION:
@@ -481,7 +486,13 @@ extern "C" lsgd_status lsgd_step(lsgd_handle h) {
     }
   } else if (h->mc_step_pending) {
     // plain step straight from the fixed-point gradient sums (only the entries the batch touched move)
+#if LSGD_MATCOMP_SCAN_STEP
     LSGD_CUDA(launch_matcomp_finish_step(h->d_acc64, c.x, c.P, c.ld, (double)c.eta, (int)c.arithmetic, h->stream));
+#else
+    MatcompArgs ma{h->mc, c.x, c.g, c.ld, c.P, h->d_status};
+    LSGD_CUDA(launch_matcomp_step_from_batch(ma, h->mc_pending_pos, h->d_acc64, c.x, (double)c.eta, (int)c.arithmetic,
+                                             h->stream));
+#endif
   } else if (a.v) {
     LSGD_CUDA(launch_momentum_update(a, h->stream));
   } else {
