@@ -146,7 +146,7 @@ typedef struct {
   void* stream;              /* cudaStream_t; NULL = the legacy default stream                       */
   int32_t arithmetic;        /* lsgd_arithmetic                                                      */
   uint32_t flags;            /* bit set of LSGD_FLAG_*; 0 = defaults                                 */
-  /* --- only read with LSGD_FLAG_ALGORITHM1 (see below) --- */
+  /* --- only read with LSGD_FLAG_ALGORITHM1 (see below); leader_copies also with LSGD_FLAG_EAGD --- */
   float gamma_l;             /* searching scope gamma: every step pulls with strength eta gamma / tau  */
   float gamma_g;             /* gamma_G: every step pulls with strength eta gamma_G / tau_G           */
   int32_t tau_g;             /* global communication period tau_G >= 1                               */
@@ -197,6 +197,18 @@ typedef struct {
  * returns the second vector).  A loss vector given by the caller serves both elections of a communication.
  * LSGD_FLAG_MLP_FUSED_STEP is ignored in this mode.                                                   */
 #define LSGD_FLAG_ALGORITHM1 2u
+
+/* Elastic averaging (EAGD / EASGD), the method the paper compares LGD with (supplement, "Low-Rank Matrix
+ * Completion Experiments"): instead of a leader, every worker is pulled towards a center variable X~,
+ *   x_i <- x_i - eta g_i - eta lambda (x_i - X~),   X~ <- (1 - P eta lambda) X~ + P eta lambda (1/P) sum_i x_i,
+ * both from the values at time t, on the steps t = 0, tau, 2 tau, ...; plain steps in between.  lambda is
+ * lambda_l; lambda_g must be 0 (LSGD_ERR_INVALID_ARG).  leader_copies (DEVICE float[(G+1)*ld], as above) is
+ * required: row G holds X~ (readable by the caller once the stream has drained), row 0 is scratch for the new
+ * center; the library clears the buffer at creation and starts X~ at the workers' mean on the first step (the
+ * paper does not say where it starts).  No election takes place: lsgd_elect is not needed, and the groups
+ * play no role.  Not combined with LSGD_FLAG_ALGORITHM1, the fused-step flags or a momentum buffer
+ * (LSGD_ERR_UNSUPPORTED).  A comparison line: it reuses the pull kernels and is not tuned.               */
+#define LSGD_FLAG_EAGD 8u
 
 /* Validates the configuration on the host, copies the group map, builds the group tables and
  * allocates O(P + G) words of device state plus reduction scratch for the objective's election

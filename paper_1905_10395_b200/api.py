@@ -18,6 +18,7 @@ ARITH_FP64, ARITH_FP64_FMA, ARITH_FP32 = range(3)
 FLAG_MLP_FUSED_STEP = 1
 FLAG_ALGORITHM1 = 2
 FLAG_MATCOMP_FUSED_STEP = 4
+FLAG_EAGD = 8
 # bits of the device status word (lsgd_check_device)
 DEVFLAG_BAD_LEADER, DEVFLAG_WAIT_TIMEOUT, DEVFLAG_BAD_INDEX, DEVFLAG_OVERFLOW = 1, 2, 4, 8
 

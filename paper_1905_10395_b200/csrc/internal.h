@@ -92,6 +92,10 @@ cudaError_t launch_momentum_update_chunked(const UpdateArgs& a, cudaStream_t s);
 cudaError_t launch_wait_timeout_selftest(uint32_t* status, long long budget_cycles, int* gave_up, cudaStream_t s);
 cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, int64_t ld, cudaStream_t s);
 
+// out[k] <- (1 - kk) center[k] + kk * mean_i x[i][k] over all ld columns (EAGD center rule, kk = P eta lambda)
+cudaError_t launch_eagd_center(const float* x, const float* center, float* out, int32_t P, int64_t ld, double kk,
+                               cudaStream_t s);
+
 struct ElectArgs {
   const float* loss_in;     // DEVICE float[P] or nullptr when partials are given
   const double* partials;   // DEVICE double[P][n_partials] (row sums in fixed order) or nullptr
@@ -215,6 +219,7 @@ struct lsgd_ctx {
   int64_t t;
   int64_t n_elections;
   bool grad_ready;
+  bool eagd_center_ready;    // EAGD: the center row has been initialised to the workers' mean
   bool fused_applied;        // MLP: the pending gradient has already stepped W1, W2 (plain step)
   const float* armed_noise;  // QUADRATIC with g == NULL: noise pointer for the next step
   void* mlp_state;           // opaque MLP pipeline state

@@ -47,6 +47,13 @@ lsgd_status validate(const lsgd_config* c) {
     if (!c->leader_copies) return LSGD_ERR_INVALID_ARG;
     if (!aligned16(c->leader_copies)) return LSGD_ERR_ALIGNMENT;
   }
+  if (c->flags & LSGD_FLAG_EAGD) {
+    if (!c->leader_copies) return LSGD_ERR_INVALID_ARG;
+    if (!aligned16(c->leader_copies)) return LSGD_ERR_ALIGNMENT;
+    if (c->lambda_g != 0.f) return LSGD_ERR_INVALID_ARG;
+    if ((c->flags & (LSGD_FLAG_ALGORITHM1 | LSGD_FLAG_MLP_FUSED_STEP | LSGD_FLAG_MATCOMP_FUSED_STEP)) || c->v)
+      return LSGD_ERR_UNSUPPORTED;
+  }
   if (c->v) {
     if (!std::isfinite(c->momentum) || !std::isfinite(c->weight_decay)) return LSGD_ERR_INVALID_ARG;
     if (!c->g) return LSGD_ERR_INVALID_ARG;
@@ -129,6 +136,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->t = 0;
   h->n_elections = 0;
   h->grad_ready = false;
+  h->eagd_center_ready = false;
   h->fused_applied = false;
   h->mc_step_pending = false;
   h->mc_pending_pos = nullptr;
@@ -215,6 +223,9 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   if (ok && cfg->objective == LSGD_OBJ_PSD_COMPLETION && psd_split(h->psd.r) > 1)
     ok = cudaMalloc(reinterpret_cast<void**>(&h->d_psd_part),
                     sizeof(double) * (size_t)psd_split(h->psd.r) * (size_t)P * (size_t)cfg->ld) == cudaSuccess;
+  // EAGD: rows 0 .. G-1 of leader_copies are read (with a zero coefficient) before the library writes them all
+  if (ok && (cfg->flags & LSGD_FLAG_EAGD))
+    ok = cudaMemsetAsync(cfg->leader_copies, 0, sizeof(float) * (size_t)(G + 1) * (size_t)cfg->ld, h->stream) == cudaSuccess;
   // the gradient kernel of this objective writes columns < d only: clear the padding of g once
   if (ok && cfg->objective == LSGD_OBJ_PSD_COMPLETION && cfg->ld > cfg->d)
     ok = cudaMemsetAsync(cfg->g, 0, sizeof(float) * (size_t)P * (size_t)cfg->ld, h->stream) == cudaSuccess;
@@ -461,11 +472,26 @@ extern "C" lsgd_status lsgd_step(lsgd_handle h) {
   if (!on_own_device(h)) return LSGD_ERR_STATE;
   const lsgd_config& c = h->cfg;
   const bool alg1 = (c.flags & LSGD_FLAG_ALGORITHM1) != 0;
+  const bool eagd = (c.flags & LSGD_FLAG_EAGD) != 0;
   const bool pull = alg1 ? (c.gamma_l != 0.f || c.gamma_g != 0.f) : (h->t % c.tau) == 0;
-  if ((pull || alg1) && h->n_elections == 0) return LSGD_ERR_STATE;
+  if ((pull || alg1) && !eagd && h->n_elections == 0) return LSGD_ERR_STATE;
   if (c.objective != LSGD_OBJ_EXTERNAL && !h->grad_ready) return LSGD_ERR_STATE;
   UpdateArgs a = base_update_args(h);
   a.pull = pull;
+  float* const center = eagd ? c.leader_copies + (size_t)c.G * (size_t)c.ld : nullptr;
+  if (eagd && pull) {
+    // elastic averaging: the guide point of every worker is the center variable (row G of leader_copies).  The
+    // new center is formed from x_t and the old center into row 0 first, the workers then step towards the OLD
+    // center, and the new one replaces it afterwards: every right-hand side is taken at time t.
+    if (!h->eagd_center_ready) {
+      LSGD_CUDA(launch_center(c.x, center, c.P, c.d, c.ld, h->stream));
+      h->eagd_center_ready = true;
+    }
+    const double kk = ((double)c.P * (double)c.eta) * (double)c.lambda_l;
+    LSGD_CUDA(launch_eagd_center(c.x, center, c.leader_copies, c.P, c.ld, kk, h->stream));
+    a.snap = c.leader_copies;
+    set_pull_coefficients(a, 0.0, (double)c.eta * (double)c.lambda_l);
+  }
   if (alg1 && pull) {
     // small pulls towards the (stale) copies of the leaders' parameters
     a.snap = c.leader_copies;
@@ -498,6 +524,8 @@ extern "C" lsgd_status lsgd_step(lsgd_handle h) {
   } else {
     LSGD_CUDA(launch_update(a, h->stream));
   }
+  if (eagd && pull)
+    LSGD_CUDA(cudaMemcpyAsync(center, c.leader_copies, sizeof(float) * (size_t)c.ld, cudaMemcpyDeviceToDevice, h->stream));
   h->t++;
   h->loss_partials_valid = false;
   h->fused_applied = false;

@@ -939,6 +939,33 @@ center_kernel(const float* __restrict__ x, float* __restrict__ center, int32_t P
   }
 }
 
+// EAGD center rule (supplement, "Low-Rank Matrix Completion Experiments"):
+//   out[k] = (1 - kk) center[k] + kk * ((sum_i x[i][k]) * (1 / P)),  kk = P eta lambda,
+// one IEEE fp64 operation per printed operation (no contraction), worker-order sum, one rounding to fp32.
+__global__ void __launch_bounds__(256)
+eagd_center_kernel(const float* __restrict__ x, const float* __restrict__ center, float* __restrict__ out, int32_t P,
+                   int64_t n4, int64_t ld, double kk) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const double inv = 1.0 / (double)P, keep = __dsub_rn(1.0, kk);
+  for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < n4; c += stride) {
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    for (int i = 0; i < P; ++i) {
+      const float4 v = ld4(x + (int64_t)i * ld + c * 4);
+      s0 += (double)v.x;
+      s1 += (double)v.y;
+      s2 += (double)v.z;
+      s3 += (double)v.w;
+    }
+    const float4 z = ld4(center + c * 4);
+    float4 o;
+    o.x = (float)__dadd_rn(__dmul_rn(keep, (double)z.x), __dmul_rn(kk, __dmul_rn(s0, inv)));
+    o.y = (float)__dadd_rn(__dmul_rn(keep, (double)z.y), __dmul_rn(kk, __dmul_rn(s1, inv)));
+    o.z = (float)__dadd_rn(__dmul_rn(keep, (double)z.z), __dmul_rn(kk, __dmul_rn(s2, inv)));
+    o.w = (float)__dadd_rn(__dmul_rn(keep, (double)z.w), __dmul_rn(kk, __dmul_rn(s3, inv)));
+    *reinterpret_cast<float4*>(out + c * 4) = o;
+  }
+}
+
 template <int MODE>
 cudaError_t launch_m(const UpdateArgs& a, cudaStream_t s) {
   const bool quad = (a.g == nullptr);
@@ -957,6 +984,15 @@ cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, i
   int64_t blocks = (n4 + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   center_kernel<<<(unsigned)blocks, 256, 0, s>>>(x, center, P, n4, ld);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_eagd_center(const float* x, const float* center, float* out, int32_t P, int64_t ld, double kk,
+                               cudaStream_t s) {
+  const int64_t n4 = ld / 4;
+  int64_t blocks = (n4 + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  eagd_center_kernel<<<(unsigned)blocks, 256, 0, s>>>(x, center, out, P, n4, ld, kk);
   return cudaGetLastError();
 }
 

@@ -17,7 +17,7 @@ class Population:
                  device: str = "cuda:0", x: Optional[torch.Tensor] = None, g: Optional[torch.Tensor] = None,
                  upload_noise: bool = True, flags: int = 0, algorithm1: Optional[dict] = None,
                  stream: Optional["torch.cuda.Stream"] = None, momentum: Optional[float] = None,
-                 weight_decay: float = 0.0):
+                 weight_decay: float = 0.0, eagd: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.w = w
@@ -91,6 +91,12 @@ class Population:
             flags |= api.FLAG_ALGORITHM1
             extra = dict(gamma_l=algorithm1["gamma_l"], gamma_g=algorithm1["gamma_g"], tau_g=algorithm1["tau_g"],
                          leader_copies=self.leader_copies)
+        self.eagd = bool(eagd)
+        if self.eagd:
+            # elastic averaging instead of leaders: row G of the copies buffer is the center variable
+            self.leader_copies = torch.zeros((w.G + 1, w.ld), dtype=torch.float32, device=dev)
+            flags |= api.FLAG_EAGD
+            extra = dict(leader_copies=self.leader_copies)
         self.v = None
         if momentum is not None:
             # Section 4.1 optimiser: Nesterov momentum + weight decay; the buffers start at zero
@@ -135,6 +141,11 @@ class Population:
         if self.alg1 is not None:
             return self._step_algorithm1(forced_loss, record)
         w = self.w
+        if self.eagd:
+            self.lsgd.grad(self.batches[self.t % len(self.batches)] if self.batches else None)
+            self.lsgd.step()
+            self.t += 1
+            return
         batch = self.batches[self.t % len(self.batches)] if self.batches else None
         self.lsgd.grad(batch)
         if self.t % w.tau == 0:
@@ -191,6 +202,11 @@ class Population:
             self.lsgd.advance_step(self._graph_steps)
         self.t += self._graph_steps
         self.n_elections += self._graph_steps // self.w.tau
+
+    def center_host(self) -> np.ndarray:
+        """EAGD: the center variable."""
+        torch.cuda.synchronize(self.dev)
+        return self.leader_copies[self.w.G].cpu().numpy()
 
     def x_host(self) -> np.ndarray:
         torch.cuda.synchronize(self.dev)
