@@ -255,6 +255,24 @@ LSGD_API lsgd_status lsgd_get_leaders(lsgd_handle h, int32_t* local_leaders /* H
  * Counts as an election for the step protocol; the leader statistics are not changed.
  * LSGD_ERR_BAD_GROUPS if an index is out of range or not in its group.                              */
 LSGD_API lsgd_status lsgd_set_leaders(lsgd_handle h, const int32_t* local_leaders, int32_t global_leader);
+/* A population whose groups live on several devices (Section 2.2 maps a group to a node; see
+ * paper_1905_10395_b200/sharded.py): the global election across devices, in two device-side halves around ONE
+ * exchange of 8 bytes per device.  A handle then holds its device's own workers first (n_own rows, in global
+ * order) followed by a guest row that receives the global leader's parameters when another device owns it.
+ *
+ * lsgd_shard_best_key  after lsgd_elect: packs the best of the first n_own workers' election losses with that
+ *   worker's GLOBAL index (global_index: DEVICE int32[n_own]) into *key_out (DEVICE int64[1], enqueued on the
+ *   stream): (orderable loss << 32) | global index, an unsigned key whose minimum over all devices is the
+ *   global leader under the rule of lsgd_elect (ties to the lowest global index).
+ * lsgd_shard_pick_global  given every device's key (keys: DEVICE int64[world], e.g. from an all-gather), takes
+ *   the minimum, points this handle's global leader at its own best worker (if my_rank won) or at guest_row, and
+ *   returns result (HOST int32[3]) = {winning rank, the winner's global worker index, this device's best own
+ *   worker (its row is what the winning device sends)}.  Synchronises the stream once.
+ * The caller then broadcasts the winner's row into the other devices' guest rows and calls lsgd_step; the update
+ * kernels read local memory only.  LSGD_ERR_STATE before any election.                                  */
+LSGD_API lsgd_status lsgd_shard_best_key(lsgd_handle h, int32_t n_own, const int32_t* global_index, int64_t* key_out);
+LSGD_API lsgd_status lsgd_shard_pick_global(lsgd_handle h, const int64_t* keys, int32_t world, int32_t my_rank,
+                                            int32_t guest_row, int32_t* result);
 LSGD_API lsgd_status lsgd_get_loss(lsgd_handle h, float* loss /* HOST float[P]: losses of the last election */);
 LSGD_API lsgd_status lsgd_get_step(lsgd_handle h, int64_t* t);
 /* Mean minibatch loss of every worker from the last lsgd_grad (MLP objective only; LSGD_ERR_UNSUPPORTED

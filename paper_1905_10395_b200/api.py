@@ -100,6 +100,10 @@ def lib() -> C.CDLL:
         L.lsgd_get_leader_counts.argtypes = [H, C.c_void_p, C.c_void_p]
         L.lsgd_check_device.argtypes = [H, C.POINTER(C.c_uint32)]
         L.lsgd_set_eta.argtypes = [H, C.c_float]
+        L.lsgd_shard_best_key.argtypes = [H, C.c_int32, C.c_void_p, C.c_void_p]
+        L.lsgd_shard_best_key.restype = C.c_int
+        L.lsgd_shard_pick_global.argtypes = [H, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+        L.lsgd_shard_pick_global.restype = C.c_int
         L.lsgd_mlp_get_activations.argtypes = [H, C.c_void_p, C.c_void_p]
         L.lsgd_mlp_get_activations.restype = C.c_int
         L.lsgd_selftest_wait_timeout.argtypes = [H, C.c_int64, C.POINTER(C.c_int32)]
@@ -253,6 +257,17 @@ class Lsgd:
         ll = None if local_leaders is None else np.ascontiguousarray(local_leaders, dtype=np.int32)
         _check(lib().lsgd_set_leaders(self.h, None if ll is None else ll.ctypes.data, int(global_leader)),
                "lsgd_set_leaders")
+
+    def shard_best_key(self, n_own: int, global_index, key_out):
+        """key_out (device int64[1]) <- this device's best own worker as a cross-device election key."""
+        _check(lib().lsgd_shard_best_key(self.h, int(n_own), _ptr(global_index), _ptr(key_out)), "lsgd_shard_best_key")
+
+    def shard_pick_global(self, keys, world: int, my_rank: int, guest_row: int):
+        """(winning rank, winner's global worker index, this device's best own worker) from all devices' keys."""
+        out = np.empty(3, dtype=np.int32)
+        _check(lib().lsgd_shard_pick_global(self.h, _ptr(keys), int(world), int(my_rank), int(guest_row), out.ctypes.data),
+               "lsgd_shard_pick_global")
+        return int(out[0]), int(out[1]), int(out[2])
 
     def loss(self):
         out = np.empty(self.P, dtype=np.float32)

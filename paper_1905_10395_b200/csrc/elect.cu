@@ -92,7 +92,83 @@ leader_copies_kernel(const float* __restrict__ x, float* __restrict__ copies, co
   for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < n4; c += stride) d4[c] = s4[c];
 }
 
+// Cross-device election, first half: the best of this device's OWN workers (the first n_own rows of the handle)
+// as a key whose low word is the worker's GLOBAL index, so that keys of different devices compare by the rule of
+// the single-device election (loss order, then lowest global index).  One warp.
+__global__ void __launch_bounds__(32)
+shard_best_key_kernel(const float* __restrict__ loss, const int32_t* __restrict__ global_index, int32_t n_own,
+                      unsigned long long* __restrict__ key_out, int32_t* __restrict__ best_local) {
+  const int lane = threadIdx.x;
+  unsigned long long best = ~0ull;
+  int arg = 0;
+  for (int i = lane; i < n_own; i += 32) {
+    const unsigned long long k = ((unsigned long long)orderable(loss[i]) << 32) | (uint32_t)global_index[i];
+    if (k < best) {
+      best = k;
+      arg = i;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+    const int oarg = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+    if (other < best) {
+      best = other;
+      arg = oarg;
+    }
+  }
+  if (lane == 0) {
+    *key_out = best;
+    *best_local = arg;
+  }
+}
+
+// Second half: the minimum of the gathered keys names the device that owns the global leader.  This device's
+// global-leader index becomes its own best worker if it won, else the guest row that receives the winner's
+// parameters.  result = {winning rank, winner's global worker index, this device's best local worker}.
+__global__ void __launch_bounds__(32)
+shard_pick_global_kernel(const unsigned long long* __restrict__ keys, int32_t world, int32_t my_rank, int32_t guest_row,
+                         const int32_t* __restrict__ best_local, int32_t* __restrict__ gl, int32_t* __restrict__ result) {
+  const int lane = threadIdx.x;
+  unsigned long long best = ~0ull;
+  int arg = 0;
+  for (int r = lane; r < world; r += 32) {
+    const unsigned long long k = keys[r];
+    if (k < best || (k == best && r < arg)) {
+      best = k;
+      arg = r;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+    const int oarg = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+    if (other < best || (other == best && oarg < arg)) {
+      best = other;
+      arg = oarg;
+    }
+  }
+  if (lane == 0) {
+    *gl = (arg == my_rank) ? *best_local : guest_row;
+    result[0] = arg;
+    result[1] = (int32_t)(uint32_t)best;
+    result[2] = *best_local;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_shard_best_key(const float* loss, const int32_t* global_index, int32_t n_own, unsigned long long* key_out,
+                                  int32_t* best_local, cudaStream_t s) {
+  shard_best_key_kernel<<<1, 32, 0, s>>>(loss, global_index, n_own, key_out, best_local);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_shard_pick_global(const unsigned long long* keys, int32_t world, int32_t my_rank, int32_t guest_row,
+                                     const int32_t* best_local, int32_t* gl, int32_t* result, cudaStream_t s) {
+  shard_pick_global_kernel<<<1, 32, 0, s>>>(keys, world, my_rank, guest_row, best_local, gl, result);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_leader_copies(const float* x, float* copies, const int32_t* ll, const int32_t* gl, int32_t G, int32_t r0,
                                  int32_t r1, int64_t d, int64_t ld, cudaStream_t s) {

@@ -113,6 +113,11 @@ struct ElectArgs {
   bool update_global;       // write gl (and count)
 };
 cudaError_t launch_elect(const ElectArgs& a, cudaStream_t s);
+// cross-device election (groups spread over devices), see elect.cu
+cudaError_t launch_shard_best_key(const float* loss, const int32_t* global_index, int32_t n_own, unsigned long long* key_out,
+                                  int32_t* best_local, cudaStream_t s);
+cudaError_t launch_shard_pick_global(const unsigned long long* keys, int32_t world, int32_t my_rank, int32_t guest_row,
+                                     const int32_t* best_local, int32_t* gl, int32_t* result, cudaStream_t s);
 // copies[r] <- x[ll[r]] for r in [r0, min(r1, G)), and copies[G] <- x[gl] if r1 > G
 cudaError_t launch_leader_copies(const float* x, float* copies, const int32_t* ll, const int32_t* gl, int32_t G,
                                  int32_t r0, int32_t r1, int64_t d, int64_t ld, cudaStream_t s);
@@ -141,9 +146,6 @@ struct MatcompArgs {
 cudaError_t launch_matcomp_grad(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, bool finish, cudaStream_t s);
 cudaError_t launch_matcomp_finish_step(unsigned long long* acc, float* x, int32_t P, int64_t ld, double eta, int arith,
                                        cudaStream_t s);
-// the same step, visiting only the entries of the batch `pos` that produced the sums (pos must still be valid)
-cudaError_t launch_matcomp_step_from_batch(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, float* x,
-                                           double eta, int arith, cudaStream_t s);
 int32_t matcomp_loss_blocks(int32_t n_heldout);
 cudaError_t launch_matcomp_loss_partials(const MatcompArgs& a, double* partials, int32_t n_partials,
                                          cudaStream_t s);
@@ -215,6 +217,7 @@ struct lsgd_ctx {
   unsigned long long* d_group_keys;
   double* d_partials;
   int32_t* d_selftest;          // one word written by lsgd_selftest_wait_timeout
+  int32_t* d_shard;             // cross-device election: [0] this device's best own worker, [1..3] the result triple
   int32_t n_partials;
   int64_t t;
   int64_t n_elections;
@@ -225,6 +228,5 @@ struct lsgd_ctx {
   void* mlp_state;           // opaque MLP pipeline state
   unsigned long long* d_acc64;  // MATCOMP: fixed-point gradient accumulator [P*ld], kept all-zero between steps
   bool mc_step_pending;         // MATCOMP fused step: the gradient sums wait in d_acc64 for lsgd_step
-  const int32_t* mc_pending_pos;  // ... and this is the batch that produced them (caller's DEVICE pointer)
   double* d_psd_part;           // PSD, small ranks: partial gradients of the CTAs that share a row block
 };

@@ -11,9 +11,6 @@ using namespace lsgd;
 
 namespace {
 
-#ifndef LSGD_MATCOMP_SCAN_STEP
-#define LSGD_MATCOMP_SCAN_STEP 0   // 1: the fused matrix-completion step scans the whole accumulator instead of the batch
-#endif
 constexpr int32_t kMaxWorkers = 4096;  // group tables live in shared memory of the update kernel
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -139,7 +136,6 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->eagd_center_ready = false;
   h->fused_applied = false;
   h->mc_step_pending = false;
-  h->mc_pending_pos = nullptr;
   h->armed_noise = nullptr;
   h->slab = nullptr;
   h->mlp_state = nullptr;
@@ -190,6 +186,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   const size_t o_loss = take(sizeof(float) * P), o_keys = take(sizeof(unsigned long long) * G);
   const size_t o_part = take(sizeof(double) * (size_t)P * (size_t)(h->n_partials > 0 ? h->n_partials : 1));
   const size_t o_self = take(sizeof(int32_t));
+  const size_t o_shard = take(sizeof(int32_t) * 4);
   if (cudaMalloc(&h->slab, off) != cudaSuccess) {
     delete h;
     return LSGD_ERR_CUDA;
@@ -207,6 +204,7 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->d_group_keys = reinterpret_cast<unsigned long long*>(base + o_keys);
   h->d_partials = reinterpret_cast<double*>(base + o_part);
   h->d_selftest = reinterpret_cast<int32_t*>(base + o_self);
+  h->d_shard = reinterpret_cast<int32_t*>(base + o_shard);
 
   bool ok = cudaMemsetAsync(h->slab, 0, off, h->stream) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(h->d_rows_by_group, rows.data(), sizeof(int32_t) * P, cudaMemcpyHostToDevice, h->stream) == cudaSuccess;
@@ -266,7 +264,6 @@ lsgd_status lsgd_grad(lsgd_handle h, const void* batch) {
                         (h->t % c.tau) != 0;
       LSGD_CUDA(launch_matcomp_grad(a, static_cast<const int32_t*>(batch), h->d_acc64, !fuse, h->stream));
       h->mc_step_pending = fuse;
-      h->mc_pending_pos = static_cast<const int32_t*>(batch);
       break;
     }
     case LSGD_OBJ_PSD_COMPLETION:
@@ -512,13 +509,7 @@ extern "C" lsgd_status lsgd_step(lsgd_handle h) {
     }
   } else if (h->mc_step_pending) {
     // plain step straight from the fixed-point gradient sums (only the entries the batch touched move)
-#if LSGD_MATCOMP_SCAN_STEP
     LSGD_CUDA(launch_matcomp_finish_step(h->d_acc64, c.x, c.P, c.ld, (double)c.eta, (int)c.arithmetic, h->stream));
-#else
-    MatcompArgs ma{h->mc, c.x, c.g, c.ld, c.P, h->d_status};
-    LSGD_CUDA(launch_matcomp_step_from_batch(ma, h->mc_pending_pos, h->d_acc64, c.x, (double)c.eta, (int)c.arithmetic,
-                                             h->stream));
-#endif
   } else if (a.v) {
     LSGD_CUDA(launch_momentum_update(a, h->stream));
   } else {
@@ -571,6 +562,30 @@ lsgd_status lsgd_set_leaders(lsgd_handle h, const int32_t* local_leaders, int32_
   if (global_leader >= 0)
     LSGD_CUDA(cudaMemcpyAsync(h->d_gl, &global_leader, sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
   h->n_elections++;
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_shard_best_key(lsgd_handle h, int32_t n_own, const int32_t* global_index, int64_t* key_out) {
+  if (!h || !global_index || !key_out) return LSGD_ERR_INVALID_ARG;
+  if (n_own < 1 || n_own > h->cfg.P) return LSGD_ERR_INVALID_ARG;
+  if (h->n_elections == 0) return LSGD_ERR_STATE;                  // no loss vector yet
+  if (!on_own_device(h)) return LSGD_ERR_STATE;
+  LSGD_CUDA(launch_shard_best_key(h->d_loss, global_index, n_own, reinterpret_cast<unsigned long long*>(key_out), h->d_shard,
+                                  h->stream));
+  return LSGD_OK;
+}
+
+lsgd_status lsgd_shard_pick_global(lsgd_handle h, const int64_t* keys, int32_t world, int32_t my_rank, int32_t guest_row,
+                                   int32_t* result) {
+  if (!h || !keys || !result) return LSGD_ERR_INVALID_ARG;
+  if (world < 1 || my_rank < 0 || my_rank >= world) return LSGD_ERR_INVALID_ARG;
+  if (guest_row < 0 || guest_row >= h->cfg.P) return LSGD_ERR_BAD_GROUPS;
+  if (h->n_elections == 0) return LSGD_ERR_STATE;
+  if (!on_own_device(h)) return LSGD_ERR_STATE;
+  LSGD_CUDA(launch_shard_pick_global(reinterpret_cast<const unsigned long long*>(keys), world, my_rank, guest_row, h->d_shard,
+                                     h->d_gl, h->d_shard + 1, h->stream));
+  LSGD_CUDA(cudaStreamSynchronize(h->stream));
+  LSGD_CUDA(cudaMemcpy(result, h->d_shard + 1, sizeof(int32_t) * 3, cudaMemcpyDeviceToHost));
   return LSGD_OK;
 }
 

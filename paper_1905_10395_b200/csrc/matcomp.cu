@@ -120,41 +120,6 @@ matcomp_finish_step_kernel(unsigned long long* __restrict__ acc, float* __restri
   }
 }
 
-// The same plain step, visiting only what the batch touched: the kernel walks the batch again with the gradient
-// kernel's layout (a lane group per observed entry, lane k on component k) and takes each touched sum out of the
-// accumulator with an atomic exchange -- the first group to reach a row gets the whole sum and steps the
-// parameter, later groups with the same row (duplicates in the batch) find zero and do nothing.  Entries the
-// gradient kernel skipped (bad index) are skipped here too.  A plain load in front of the exchange keeps the
-// duplicates off the atomic unit.
-template <int GROUP>
-__global__ void __launch_bounds__(kThreads)
-matcomp_step_from_batch_kernel(MatcompArgs a, const int32_t* __restrict__ pos, unsigned long long* __restrict__ acc,
-                               float* __restrict__ x, double eta, int arith) {
-  const int i = blockIdx.y;
-  const int lane = threadIdx.x & 31, k = lane % GROUP;
-  const int p = (blockIdx.x * kThreads + threadIdx.x) / GROUP;
-  const int rank = a.m.rank;
-  if (p >= a.m.batch || k >= rank) return;
-  const int q = pos[(int64_t)i * a.m.batch + p];
-  if (q < 0 || q >= a.m.n_obs) return;
-  const int r = a.m.obs_r[q], c = a.m.obs_c[q];
-  if (r < 0 || r >= a.m.n_rows || c < 0 || c >= a.m.n_cols) return;
-  const int64_t off[2] = {(int64_t)i * a.ld + (int64_t)r * rank + k, (int64_t)i * a.ld + ((int64_t)a.m.n_rows + c) * rank + k};
-#pragma unroll
-  for (int j = 0; j < 2; ++j) {
-    if (acc[off[j]] == 0ull) continue;
-    const long long v = (long long)atomicExch(acc + off[j], 0ull);
-    if (v == 0) continue;
-    const float g = (float)((double)v * kFixInv);
-    const float xv = x[off[j]];
-    float xn;
-    if (arith == 0) xn = (float)__dsub_rn((double)xv, __dmul_rn(eta, (double)g));
-    else if (arith == 1) xn = (float)fma(-eta, (double)g, (double)xv);
-    else xn = fmaf(-(float)eta, g, xv);
-    x[off[j]] = xn;
-  }
-}
-
 // Held-out loss: one thread per entry (the kernel is bound by the L2 gathers of the factor rows, 2 sectors per
 // row whoever fetches them; one entry per thread keeps the most of them in flight), fp64 residuals, partial sums
 // per CTA in a fixed order.
@@ -223,18 +188,6 @@ cudaError_t launch_matcomp_finish_step(unsigned long long* acc, float* x, int32_
   const int64_t total = (int64_t)P * ld;                    // ld is a multiple of 32
   const int64_t blocks = (total / 4 + kThreads - 1) / kThreads;
   matcomp_finish_step_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(acc, x, total, eta, arith);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_matcomp_step_from_batch(const MatcompArgs& a, const int32_t* pos, unsigned long long* acc, float* x,
-                                           double eta, int arith, cudaStream_t s) {
-  const int rank = a.m.rank;
-  const int group = rank <= 8 ? 8 : (rank <= 16 ? 16 : 32);
-  const int per_cta = kThreads / group;
-  dim3 grid((unsigned)((a.m.batch + per_cta - 1) / per_cta), (unsigned)a.P);
-  if (group == 8) matcomp_step_from_batch_kernel<8><<<grid, kThreads, 0, s>>>(a, pos, acc, x, eta, arith);
-  else if (group == 16) matcomp_step_from_batch_kernel<16><<<grid, kThreads, 0, s>>>(a, pos, acc, x, eta, arith);
-  else matcomp_step_from_batch_kernel<32><<<grid, kThreads, 0, s>>>(a, pos, acc, x, eta, arith);
   return cudaGetLastError();
 }
 

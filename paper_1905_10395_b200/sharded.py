@@ -4,12 +4,14 @@ local leader is shared inside the node, the global leader across nodes, less oft
 Each rank owns whole groups.  Everything inside a rank is the single-device path unchanged: the rank's handle
 holds its workers plus one extra row, the *guest row*, in a group of its own.  On a pull step
 
-  1. every rank evaluates its workers' election losses and elects its local leaders (``lsgd_elect``);
-  2. the ranks exchange (best local loss, global index of that worker) -- a few bytes per rank;
+  1. every rank evaluates its workers' election losses, elects its local leaders (``lsgd_elect``) and packs its
+     best own worker into an 8-byte key on the device (``lsgd_shard_best_key``);
+  2. ONE all-gather of those keys; each rank's ``lsgd_shard_pick_global`` takes their minimum on the device,
+     points its global leader at its own winner or at the guest row, and hands the host the winning rank -- the
+     one host synchronisation of the step;
   3. the rank that owns the global leader sends that worker's parameters (d floats) to the others, which receive
      them INTO THEIR OWN MEMORY (the guest row) -- the only bulk transfer, once per period, as in the paper;
-  4. every rank points its global leader at the local winner or at the guest row (``lsgd_set_leaders``) and
-     takes the fused step; the update kernel reads nothing but local memory.
+  4. every rank takes the fused step; the update kernel reads nothing but local memory.
 
 The result equals the single-device run bit for bit: the losses are per worker, the election rule is the same
 total order (-inf < finite < +inf < NaN, -0 == +0, ties to the lowest GLOBAL worker index), and the update of a
@@ -19,7 +21,7 @@ The exchange is written against ``torch.distributed`` (NCCL between GPUs, gloo i
 emulating several ranks inside one process, as ``run_lockstep``.  Objectives: EXTERNAL and QUADRATIC."""
 from __future__ import annotations
 
-from typing import List, Optional, Sequence, Tuple
+from typing import List, Optional, Sequence
 
 import numpy as np
 
@@ -36,25 +38,6 @@ def partition_groups(G: int, world: int) -> List[range]:
         out.append(range(lo, lo + n))
         lo += n
     return out
-
-
-def _order_key(loss: float, index: int) -> Tuple[int, float, int]:
-    """Sort key of the election's total order: NaN after +inf, -0 == +0, then the lower worker index."""
-    v = float(np.float32(loss))
-    if v != v:
-        return (1, 0.0, int(index))
-    return (0, v + 0.0, int(index))
-
-
-def argmin_by_rule(loss: Sequence[float], indices: Sequence[int]) -> int:
-    """Position (into the given sequences) of the election winner among (loss, worker index) pairs."""
-    keys = [_order_key(l, i) for l, i in zip(loss, indices)]
-    return min(range(len(keys)), key=lambda p: keys[p])
-
-
-def pick_global_leader(best_loss: Sequence[float], best_index: Sequence[int]) -> int:
-    """Given every rank's best (loss, GLOBAL worker index), the rank that owns the global leader."""
-    return argmin_by_rule(best_loss, best_index)
 
 
 class Shard:
@@ -120,34 +103,49 @@ class CudaShardEngine:
                                     x=self.x, g=self.g, desc=desc, arithmetic=arithmetic,
                                     stream=torch.cuda.current_stream(self.dev).cuda_stream)
         self.lsgd = api.Lsgd(cfg, keepalive=(keep, desc))
-        self.local_leaders_global: Optional[np.ndarray] = None
         self.global_leader_global: Optional[int] = None
         self._best_local = -1
+        self.global_index = torch.from_numpy(sh.workers.astype(np.int32)).to(self.dev)
+        self._key = torch.zeros(1, dtype=torch.int64, device=self.dev)
 
-    # -- the four pieces of a step
+    # -- the pieces of a step
     def is_pull_step(self) -> bool:
         return self.t % self.w.tau == 0
 
-    def phase_local(self) -> Optional[Tuple[float, int]]:
-        """Gradient; on a pull step also the local election.  Returns this rank's best (loss, global index)."""
-        sh = self.shard
+    def begin_step(self) -> bool:
+        """Gradient; on a pull step also the local election and this rank's key.  True on a pull step."""
         batch = self.batches[self.t % len(self.batches)] if self.batches else None
         self.lsgd.grad(batch)
         if not self.is_pull_step():
-            return None
+            return False
         if self.w.objective == "external":
-            slot = self.n_elections % self.loss_ring.shape[0]
-            self.lsgd.elect(self.loss_ring[slot])
-            loss = self.loss_ring_host[slot, : sh.P_local]
+            self.lsgd.elect(self.loss_ring[self.n_elections % self.loss_ring.shape[0]])
         else:
             self.lsgd.elect(None)
-            loss = self.lsgd.loss()[: sh.P_local]
         self.n_elections += 1
+        self.lsgd.shard_best_key(self.shard.P_local, self.global_index, self._key)
+        return True
+
+    def key(self):
+        """This rank's best own worker as an 8-byte election key (a one-element int64 tensor on the device)."""
+        return self._key
+
+    def new_keys(self, world: int):
+        import torch
+        return torch.empty(world, dtype=torch.int64, device=self.dev)
+
+    def pick_global(self, keys, world: int):
+        """From all ranks' keys: the winning rank and the winner's global worker index; sets this rank's global
+        leader (own winner or guest row) on the device.  The one host synchronisation of a pull step."""
+        winner, gidx, self._best_local = self.lsgd.shard_pick_global(keys, world, self.shard.rank, self.shard.guest)
+        self.global_leader_global = gidx
+        return winner, gidx
+
+    @property
+    def local_leaders_global(self) -> np.ndarray:
+        """Global indices of this rank's local leaders (reads them back: for checks, not part of a step)."""
         ll, _ = self.lsgd.leaders()
-        self.local_leaders_global = sh.workers[ll[: sh.G_local]]
-        p = argmin_by_rule(loss, sh.workers)
-        self._best_local = p
-        return float(loss[p]), int(sh.workers[p])
+        return self.shard.workers[ll[: self.shard.G_local]]
 
     def leader_row(self):
         """This rank's best worker's parameters (what it sends if it owns the global leader)."""
@@ -156,13 +154,6 @@ class CudaShardEngine:
     def guest_row(self):
         """Where a global leader owned by another rank is received."""
         return self.x[self.shard.guest]
-
-    def phase_global(self, winner_rank: int, winner_index: int) -> None:
-        """Point the global leader at the local winner or at the guest row, then take the step."""
-        mine = winner_rank == self.shard.rank
-        self.lsgd.set_leaders(None, self._best_local if mine else self.shard.guest)
-        self.global_leader_global = int(winner_index)
-        self.finish_step()
 
     def finish_step(self) -> None:
         self.lsgd.step()
@@ -179,45 +170,45 @@ class CudaShardEngine:
 
 # -------------------------------------------------------------------------------------- exchange ----
 def distributed_step(engine, group=None) -> None:
-    """One step of one rank under torch.distributed (one process per device).  The engine's rows must live where
-    the process group can send them (CUDA tensors for NCCL, CPU tensors for gloo)."""
-    import torch
+    """One step of one rank under torch.distributed (one process per device).  The engine's rows and keys must
+    live where the process group can send them (CUDA tensors for NCCL, CPU tensors for gloo).  A pull step costs
+    one all-gather of 8 bytes per rank, one host synchronisation and the broadcast of the leader's row."""
     import torch.distributed as dist
-    best = engine.phase_local()
-    if best is None:
+    if not engine.begin_step():
         engine.finish_step()
         return
     world = dist.get_world_size(group)
-    row = engine.leader_row()
-    mine = torch.tensor([best[0]], dtype=torch.float32, device=row.device)
-    idx = torch.tensor([best[1]], dtype=torch.int64, device=row.device)
-    losses = [torch.empty_like(mine) for _ in range(world)]
-    indices = [torch.empty_like(idx) for _ in range(world)]
-    dist.all_gather(losses, mine, group=group)
-    dist.all_gather(indices, idx, group=group)
-    best_loss = [float(t.item()) for t in losses]
-    best_index = [int(t.item()) for t in indices]
-    winner = pick_global_leader(best_loss, best_index)
+    keys = engine.new_keys(world)
+    dist.all_gather(list(keys.view(world, 1).unbind(0)), engine.key(), group=group)
+    winner, _ = engine.pick_global(keys, world)
     # the winner's row goes into every other rank's own memory; the update kernel then reads local memory only
-    buf = row if winner == dist.get_rank(group) else engine.guest_row()
+    buf = engine.leader_row() if winner == dist.get_rank(group) else engine.guest_row()
     dist.broadcast(buf, src=dist.get_global_rank(group, winner) if group is not None else winner, group=group)
-    engine.phase_global(winner, best_index[winner])
+    engine.finish_step()
 
 
 def run_lockstep(engines: Sequence, steps: int) -> None:
     """Several ranks inside one process (any engines whose rows can be copied with ``copy_``): the same
     protocol with the exchange done by hand.  No rank's kernels wait on another's, so this is also valid on a
     single device."""
+    world = len(engines)
     for _ in range(steps):
-        bests = [e.phase_local() for e in engines]
-        if bests[0] is None:
+        pulls = [e.begin_step() for e in engines]
+        if not pulls[0]:
             for e in engines:
                 e.finish_step()
             continue
-        winner = pick_global_leader([b[0] for b in bests], [b[1] for b in bests])
+        winners = []
+        for e in engines:
+            keys = e.new_keys(world)
+            for r, other in enumerate(engines):
+                keys[r:r + 1].copy_(other.key())
+            winners.append(e.pick_global(keys, world)[0])
+        winner = winners[0]
+        assert all(v == winner for v in winners)
         src = engines[winner].leader_row()
         for r, e in enumerate(engines):
             if r != winner:
                 e.guest_row().copy_(src)
         for e in engines:
-            e.phase_global(winner, bests[winner][1])
+            e.finish_step()

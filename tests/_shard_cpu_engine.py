@@ -1,12 +1,40 @@
 """Test infrastructure: a CPU stand-in for one rank of paper_1905_10395_b200.sharded, built from the oracle's
-election and update on the rank's rows plus the guest row (EXTERNAL objective).  It has the same four-piece
-interface as the CUDA engine, so the exchange logic (who owns the global leader, which row travels where) can
-be run on CPU tensors: in one process, or under torch.distributed with the gloo backend."""
+election and update on the rank's rows plus the guest row (EXTERNAL objective).  It has the same interface as the
+CUDA engine, so the exchange logic (who owns the global leader, which row travels where) can be run on CPU
+tensors: in one process, or under torch.distributed with the gloo backend.  The cross-rank election keys are
+packed here independently of the CUDA library (same published format: orderable float bits, then the global
+worker index), and ``argmin_by_rule`` is the plain restatement of the rule that the tests check both against."""
 import numpy as np
 import torch
 
 from oracle import lsgd_oracle as orc
-from paper_1905_10395_b200.sharded import Shard, argmin_by_rule
+from paper_1905_10395_b200.sharded import Shard
+
+
+def _order_key(loss, index):
+    """Sort key of the election's total order: NaN after +inf, -0 == +0, then the lower worker index."""
+    v = float(np.float32(loss))
+    if v != v:
+        return (1, 0.0, int(index))
+    return (0, v + 0.0, int(index))
+
+
+def argmin_by_rule(loss, indices) -> int:
+    """Position (into the given sequences) of the election winner among (loss, worker index) pairs."""
+    keys = [_order_key(l, i) for l, i in zip(loss, indices)]
+    return min(range(len(keys)), key=lambda p: keys[p])
+
+
+def pack_key(loss, global_index) -> int:
+    """(orderable(loss) << 32) | global index as an unsigned 64-bit integer: floats map monotonically to
+    uint32 (negative: all bits flipped; non-negative: sign bit set), -0 counts as +0, NaN sorts last."""
+    v = np.float32(loss)
+    if v != v:
+        o = 0xFFFFFFFF
+    else:
+        u = int((v + np.float32(0.0)).view(np.uint32))
+        o = (~u) & 0xFFFFFFFF if u & 0x80000000 else u | 0x80000000
+    return (o << 32) | int(global_index)
 
 
 class CpuShardEngine:
@@ -24,13 +52,14 @@ class CpuShardEngine:
         self._best_local = -1
         self.global_leader_global = None
         self.local_leaders_global = None
+        self._key = torch.zeros(1, dtype=torch.int64)
 
     def is_pull_step(self):
         return self.t % self.w.tau == 0
 
-    def phase_local(self):
+    def begin_step(self):
         if not self.is_pull_step():
-            return None
+            return False
         sh = self.shard
         loss = self.ring[self.n_elections % self.ring.shape[0]][sh.workers]
         self.n_elections += 1
@@ -39,18 +68,27 @@ class CpuShardEngine:
         self.local_leaders_global = sh.workers[self.ll[: sh.G_local]]
         p = argmin_by_rule(loss, sh.workers)
         self._best_local = p
-        return float(loss[p]), int(sh.workers[p])
+        self._key[0] = int(np.uint64(pack_key(loss[p], sh.workers[p])).astype(np.int64))
+        return True
+
+    def key(self):
+        return self._key
+
+    def new_keys(self, world):
+        return torch.empty(world, dtype=torch.int64)
+
+    def pick_global(self, keys, world):
+        u = keys.numpy().astype(np.int64).view(np.uint64)
+        winner = int(np.argmin(u))                        # first minimum: the lowest rank among equal keys
+        self.gl = self._best_local if winner == self.shard.rank else self.shard.guest
+        self.global_leader_global = int(u[winner] & np.uint64(0xFFFFFFFF))
+        return winner, self.global_leader_global
 
     def leader_row(self):
         return self.x[self._best_local]
 
     def guest_row(self):
         return self.x[self.shard.guest]
-
-    def phase_global(self, winner_rank, winner_index):
-        self.gl = self._best_local if winner_rank == self.shard.rank else self.shard.guest
-        self.global_leader_global = int(winner_index)
-        self.finish_step()
 
     def finish_step(self):
         w, pull = self.w, self.is_pull_step()

@@ -80,3 +80,41 @@ def test_set_leaders_overrides_the_election(P, G, d):
     assert np.array_equal(pop.x_host().view(np.uint32), x.view(np.uint32))
     assert pop.lsgd.check_device() == 0
     pop.close()
+
+
+def test_device_keys_equal_the_independently_packed_keys_and_pick_the_global_leader():
+    """lsgd_shard_best_key / lsgd_shard_pick_global against the CPU packing of the same published key format, on
+    losses with ties, signed zeros, infinities and NaN."""
+    import itertools
+    import torch
+    from paper_1905_10395_b200 import api
+    from tests._shard_cpu_engine import argmin_by_rule, pack_key
+    P = 5                                                   # 4 own workers + a guest row
+    x = torch.zeros(P, 32, device="cuda")
+    cfg, keep = api.make_config(P=P, G=3, group_of=np.asarray([0, 0, 1, 1, 2], np.int32), d=32, ld=32, eta=0.1, lambda_l=0.1,
+                                lambda_g=0.1, tau=1, objective=api.OBJ_EXTERNAL, x=x, g=x)
+    h = api.Lsgd(cfg, keep)
+    gidx = np.asarray([7, 9, 12, 40], dtype=np.int32)
+    gidx_d = torch.from_numpy(gidx).cuda()
+    key = torch.zeros(1, dtype=torch.int64, device="cuda")
+    vals = [-np.inf, -1.0, -0.0, 0.0, 1.0, np.inf, np.nan]
+    with pytest.raises(api.LsgdError) as e:
+        h.shard_best_key(4, gidx_d, key)                    # before any election
+    assert e.value.status == api.ERR_STATE
+    for n, combo in enumerate(itertools.product(vals, repeat=4)):
+        if n % 7:                                           # every 7th combination: 343 device round trips
+            continue
+        loss = np.asarray(list(combo) + [np.nan], dtype=np.float32)
+        h.elect(torch.from_numpy(loss).cuda())
+        h.shard_best_key(4, gidx_d, key)
+        mine = int(key.cpu().numpy().view(np.uint64)[0])
+        p = argmin_by_rule(loss[:4], gidx)
+        assert mine == pack_key(loss[p], gidx[p]), combo
+        other = pack_key(0.0, 8)                            # another device's key: zero loss at global worker 8
+        keys = torch.from_numpy(np.asarray([other, mine], dtype=np.uint64).view(np.int64)).cuda()
+        winner, g_index, best_local = h.shard_pick_global(keys, 2, 1, 4)
+        assert best_local == p
+        want = 0 if other < mine else 1
+        assert winner == want and g_index == (8 if want == 0 else gidx[p]), combo
+        assert h.leaders()[1] == (4 if want == 0 else p)    # guest row, or this device's own winner
+    h.destroy()

@@ -14,7 +14,7 @@ import pytest
 
 from oracle import lsgd_oracle as orc
 from paper_1905_10395_b200 import inputs, sharded
-from tests._shard_cpu_engine import CpuShardEngine
+from tests._shard_cpu_engine import CpuShardEngine, argmin_by_rule, pack_key
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -29,20 +29,29 @@ def test_partition_covers_every_group_once():
 
 
 def test_cross_rank_election_rule_equals_the_election_on_the_whole_population():
-    # every rank reports its best (loss, global index); the winner among those must be the global argmin with
+    # every rank packs its best (loss, global index) into a key; the minimum key must be the global argmin with
     # the same treatment of ties, signed zeros, infinities and NaN
     vals = [-np.inf, -1.0, -0.0, 0.0, 1.0, np.inf, np.nan]
     for combo in itertools.product(vals, repeat=4):
         loss = np.array(combo, dtype=np.float32)
         group_of = np.array([0, 0, 1, 1], dtype=np.int32)
         ll, gl = orc.elect(loss, group_of, 2)
-        bests = []
+        keys = []
         for r, idx in enumerate(([0, 1], [2, 3])):
-            p = sharded.argmin_by_rule(loss[idx], idx)
+            p = argmin_by_rule(loss[idx], idx)
             assert idx[p] == ll[r]                       # the local pick is the local leader
-            bests.append((float(loss[idx[p]]), idx[p]))
-        win = sharded.pick_global_leader([b[0] for b in bests], [b[1] for b in bests])
-        assert bests[win][1] == gl, (combo, bests, gl)
+            keys.append(pack_key(loss[idx[p]], idx[p]))
+        assert (min(keys) & 0xFFFFFFFF) == gl, (combo, keys, gl)
+
+
+def test_packed_keys_order_like_the_election_rule():
+    vals = [-np.inf, -3.5, -1e-30, -0.0, 0.0, 1e-30, 2.0, np.inf, np.nan]
+    for a in vals:
+        for b in vals:
+            for ia, ib in ((1, 2), (2, 1)):
+                want = argmin_by_rule([a, b], [ia, ib])
+                got = 0 if pack_key(a, ia) < pack_key(b, ib) else 1
+                assert got == want, (a, b, ia, ib)
 
 
 @pytest.mark.parametrize("world", [1, 2, 3])
