@@ -213,7 +213,7 @@ typedef struct {
 /* Validates the configuration on the host, copies the group map, builds the group tables and
  * allocates O(P + G) words of device state plus reduction scratch for the objective's election
  * loss (MATCOMP additionally 8 bytes per worker-parameter for its order-independent gradient
- * accumulator; PSD_COMPLETION at ranks up to 32 additionally 16 bytes per worker-parameter for the two
+ * accumulator; PSD_COMPLETION at ranks up to 64 additionally 16 bytes per worker-parameter for the two
  * partial gradients it combines).  Nothing is allocated after this call.  Returns LSGD_ERR_CUDA if no CUDA device is
  * usable.  *out is NULL on failure.                                                              */
 LSGD_API lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out);
