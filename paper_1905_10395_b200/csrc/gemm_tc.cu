@@ -427,6 +427,251 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// CTA-pair form (cta_group::2) for large products with bf16 output: a cluster of two CTAs on neighbouring SMs
+// computes one 256 x 256 tile.  Each CTA loads only ITS half of both operands per k-slice -- 128 rows of A (its
+// half of the tile's rows) and 128 rows of B (its half of the tile's columns), 32 KiB instead of the 48 KiB a
+// 128 x 256 tile needs -- and one thread of the leader CTA (cluster rank 0) issues tcgen05.mma.cta_group::2
+// (M = 256, N = 256, K = 16), which reads both CTAs' shared memory and writes both CTAs' tensor memory (each
+// holds its 128 rows x 256 columns of the accumulator).  A third less operand traffic from L2 per flop, which is
+// what bounds these products.  No load is multicast: every CTA fetches its own operand halves.
+//
+// Synchronisation (all barriers live at the same shared-memory offsets in both CTAs):
+//   full[s]      leader only; one arrival (the leader's expect_tx) plus the bytes of BOTH CTAs' loads, which
+//                the peer directs at the leader's barrier (cp.async.bulk.tensor ... .cta_group::2);
+//   empty[s]     each CTA; the leader's tcgen05.commit arrives on its own and on the peer's barrier;
+//   acc_full[b]  each CTA; likewise by commit after the tile's last product;
+//   acc_empty[b] leader only; 2 x kEpiWarps arrivals, the peer's epilogue warps arrive remotely.
+// The two CTAs meet at a cluster barrier after set-up (barriers initialised, tensor memory allocated in both)
+// and before they free tensor memory and exit.  Every mbarrier wait is bounded as in the kernel above.
+#ifndef LSGD_GEMM_CTA_PAIRS
+#define LSGD_GEMM_CTA_PAIRS 1     // 0: never use the CTA-pair kernel
+#endif
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = 2 * kABytes;                 // 128 x 64 of A and 128 x 64 of B per CTA
+constexpr int kPairEpiBytes = BM * 128 * 2;                  // half of this CTA's 128 x 256 bf16 output rows at a time
+constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + kPairEpiBytes + 1024;
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory location in the CTA with the given rank of this cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
+  uint32_t a;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(smem_addr), "r"(rank));
+  return a;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(void* dst, const CUtensorMap* map, uint32_t leader_bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(leader_bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void mma_bf16_pair(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n}"
+      ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(0u)
+      : "memory");
+}
+// arrival on an mbarrier (cluster address: this CTA's or the peer's) once the MMAs issued so far have completed
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar_cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+bgemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const __grid_constant__ CUtensorMap map_c, GemmShape p) {
+  constexpr int BN = 256;
+  constexpr uint32_t kTmemCols = 2 * BN;                    // two accumulator tiles: all of tensor memory
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* buf_b16 = smem + kPairStages * kPairStageBytes;
+  __shared__ uint64_t full_bar[kPairStages], empty_bar[kPairStages], acc_full[2], acc_empty[2];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();                     // 0: leader (issues the products), 1: peer
+  const int mt = (p.M + 2 * BM - 1) / (2 * BM), nt = (p.N + BN - 1) / BN;
+  const int n_tiles = mt * nt * p.batch;
+  const int nk = (p.K + BK - 1) / BK;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    abort_s = 0;
+    for (int s = 0; s < kPairStages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 2 * kEpiWarps);   // one arrival per epilogue warp of either CTA
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();                                       // both CTAs' barriers and tensor memory are ready
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_s;
+  volatile int* abort_flag = &abort_s;
+  pdl_wait();
+  pdl_launch_dependents();
+
+  if (warp == 0 && lane == 0) {
+    // ---------------------------------------------------------------- TMA producer (each CTA: its own halves)
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = pair; t < n_tiles && ok; t += n_pairs) {
+      const Tile q = tile_of(t, mt, nt, BN);                // q.m0 is in units of BM: scale to the 256-row tile
+      const int m0 = 2 * q.m0 + (int)rank * BM, n0 = q.n0 + (int)rank * BM;
+      const int za = p.a_batched ? q.z : 0, zb = p.b_batched ? q.z : 0;
+      for (int kt = 0; kt < nk; ++kt, ++it) {
+        const int s = it % kPairStages;
+        ok = mbar_wait(&empty_bar[s], ((it / kPairStages) & 1) ^ 1, abort_flag, p.status);
+        if (!ok) break;
+        uint8_t* sa = smem + s * kPairStageBytes;
+        uint8_t* sb = sa + kABytes;
+        if (rank == 0) mbar_expect_tx(&full_bar[s], 2 * kPairStageBytes);     // both CTAs' bytes land on this barrier
+        const uint32_t bar = map_to_rank(smem_u32(&full_bar[s]), 0);
+        const int k0 = kt * BK;
+        tma_load_3d_pair(sa, &map_a, bar, k0, m0, za);
+        tma_load_3d_pair(sa + 8192, &map_a, bar, k0, m0 + 64, za);
+        tma_load_3d_pair(sb, &map_b, bar, k0, n0, zb);
+        tma_load_3d_pair(sb + 8192, &map_b, bar, k0, n0 + 64, zb);
+      }
+    }
+  } else if (warp == 1 && lane == 0 && rank == 0) {
+    // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+    uint32_t it = 0;
+    int local = 0;
+    bool ok = true;
+    for (int t = pair; t < n_tiles && ok; t += n_pairs, ++local) {
+      const int b = local & 1;
+      ok = mbar_wait(&acc_empty[b], ((local >> 1) & 1) ^ 1, abort_flag, p.status);   // both epilogues have drained it
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t tacc = tmem_base + (uint32_t)(b * BN);
+      for (int kt = 0; kt < nk; ++kt, ++it) {
+        const int s = it % kPairStages;
+        ok = mbar_wait(&full_bar[s], (it / kPairStages) & 1, abort_flag, p.status);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t sa = smem_u32(smem + s * kPairStageBytes), sb = sa + kABytes;
+#pragma unroll
+        for (int k = 0; k < BK / 16; ++k)
+          mma_bf16_pair(tacc, smem_desc(sa + k * 32, 16, 1024), smem_desc(sb + k * 32, 16, 1024), idesc, (kt | k) != 0 ? 1u : 0u);
+        // the stage is free in both CTAs once these products have read it
+        mma_commit_pair(map_to_rank(smem_u32(&empty_bar[s]), 0));
+        mma_commit_pair(map_to_rank(smem_u32(&empty_bar[s]), 1));
+      }
+      if (ok) {
+        mma_commit_pair(map_to_rank(smem_u32(&acc_full[b]), 0));
+        mma_commit_pair(map_to_rank(smem_u32(&acc_full[b]), 1));
+      }
+    }
+  } else if (warp >= 2) {
+    // ---------------------------------------------------------------- epilogue (8 warps in each CTA: its 128 rows)
+    const int q4 = warp & 3;
+    const int part = (warp - 2) >> 2;
+    static_assert(kEpiWarps == 8, "the pair kernel's epilogue is written for two warp groups");
+    const int row = q4 * 32 + lane;
+    const bool leader_thread = (threadIdx.x == 64);
+    int local = 0;
+    bool ok = true;
+    for (int t = pair; t < n_tiles && ok; t += n_pairs, ++local) {
+      const Tile q = tile_of(t, mt, nt, BN);
+      const int m0 = 2 * q.m0 + (int)rank * BM;
+      const int b = local & 1;
+      ok = mbar_wait(&acc_full[b], (local >> 1) & 1, abort_flag, p.status);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t tacc = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * BN);
+      // the 256 columns leave in two halves through one 128-column staging buffer (that leaves room for six
+      // operand stages); within a half, each of the two warp groups converts 64 columns into its own box
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+#pragma unroll 1
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = 4 * half + 2 * part + cc;               // 32-column chunk of the tile
+          if (q.n0 + c * 32 >= p.N) break;
+          uint32_t r[32];
+          tmem_ld32(tacc + (uint32_t)(c * 32), r);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          uint8_t* b16_box = buf_b16 + part * 16384;
+          const int b16_u0 = cc * 4;
+          float v[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+          if (p.epilogue == GEMM_EPI_BIAS_RELU_BF16) {
+            const float* bias = p.bias + (int64_t)q.z * p.stride_bias + q.n0 + c * 32;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float bj = (q.n0 + c * 32 + j < p.N) ? bias[j] : 0.f;
+              v[j] = fmaxf(v[j] + bj, 0.f);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(v[8 * u], v[8 * u + 1]), h1 = __floats2bfloat162_rn(v[8 * u + 2], v[8 * u + 3]);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * u + 4], v[8 * u + 5]), h3 = __floats2bfloat162_rn(v[8 * u + 6], v[8 * u + 7]);
+            uint4 w;
+            w.x = *reinterpret_cast<uint32_t*>(&h0);
+            w.y = *reinterpret_cast<uint32_t*>(&h1);
+            w.z = *reinterpret_cast<uint32_t*>(&h2);
+            w.w = *reinterpret_cast<uint32_t*>(&h3);
+            *reinterpret_cast<uint4*>(b16_box + swz(row, b16_u0 + u)) = w;
+          }
+        }
+        if (half == 1) {
+          // this CTA's half of the accumulator has been read: tell the leader's issuer (one arrival per warp)
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[b]), 0));
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        epi_barrier();
+        if (leader_thread) {
+#pragma unroll
+          for (int bx = 0; bx < 2; ++bx) {
+            const int col = q.n0 + half * 128 + bx * 64;
+            if (col < p.N && m0 < p.M) tma_store_3d(buf_b16 + bx * 16384, &map_c, col, m0, q.z);
+          }
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the buffer may be overwritten again
+        }
+        epi_barrier();
+      }
+    }
+    if (leader_thread) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();      // nobody frees tensor memory or leaves while the other CTA may still signal or be read
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -513,6 +758,22 @@ cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, con
   const int64_t mtiles = (p.M + BM - 1) / BM;
   const int64_t tiles256 = (int64_t)((p.N + 255) / 256) * mtiles * p.batch;
   const bool bf16_out = p.epilogue != GEMM_EPI_F32 && p.epilogue != GEMM_EPI_SGD;
+#if LSGD_GEMM_CTA_PAIRS
+  // CTA pairs on 256 x 256 tiles: K-major operands, plain or bias + ReLU bf16 output, at least two rounds of tiles
+  const int64_t pair_tiles = (int64_t)((p.N + 255) / 256) * ((p.M + 255) / 256) * p.batch;
+  const int n_pairs = sms / 2;
+  if ((p.epilogue == GEMM_EPI_BIAS_RELU_BF16 || p.epilogue == GEMM_EPI_BF16) && !p.a_mn && !p.b_mn && p.M >= 256 && p.N >= 256 &&
+      pair_tiles >= 2 * (int64_t)n_pairs) {
+    static OncePerDevice pair_attr;
+    if (!pair_attr.here()) {
+      cudaError_t e = cudaFuncSetAttribute(bgemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+      if (e != cudaSuccess) return e;
+      pair_attr.here() = true;
+    }
+    const unsigned grid = 2u * (unsigned)(pair_tiles < n_pairs ? pair_tiles : n_pairs);
+    return launch_pdl(bgemm_pair_kernel, dim3(grid), dim3(kThreads), kPairSmemBytes, s, map_a, map_b, map_c, p);
+  }
+#endif
   if (bf16_out && p.N >= 256 && tiles256 >= 2 * (int64_t)sms) {
     const unsigned grid = (unsigned)(tiles256 < sms ? tiles256 : sms);
     return launch_pdl(bgemm_bf16_kernel<256>, dim3(grid), dim3(kThreads), kSmemBytes, s, map_a, map_b, map_c, map_aux, p);

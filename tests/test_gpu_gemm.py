@@ -106,3 +106,21 @@ def test_bgemm_wide_tiles_on_large_products(a_mn, b_mn):
     mask = torch.randint(-1, 2, (batch, M, N), generator=gen, device="cuda").to(torch.bfloat16)
     got = _run(api, torch, A, B, M, N, K, batch, a_mn, b_mn, epilogue=2, mask=mask)
     assert torch.equal(got, torch.where(mask.double() > 0, ref, torch.zeros_like(ref)).to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("M,N,K,batch,share_a", [(1024, 1024, 784, 12, False), (512, 768, 1024, 40, True),
+                                                 (1000, 1096, 200, 12, False), (300, 264, 72, 80, False)])
+def test_bgemm_cta_pair_tiles(M, N, K, batch, share_a):
+    """K-major products with bf16 output and at least two rounds of 256 x 256 tiles run on CTA pairs
+    (tcgen05 cta_group::2: each CTA of a pair loads half of both operands).  Exact against fp64 on integer
+    operands, with full and ragged tiles, a shared A operand (the held-out batch) and both epilogues."""
+    import torch
+    from paper_1905_10395_b200 import api
+    gen = torch.Generator(device="cuda").manual_seed(500 + M + N)
+    A, B, ref = _operands(torch, gen, M, N, K, batch, 0, 0, integer=True, share_a=share_a)
+    got = _run(api, torch, A, B, M, N, K, batch, 0, 0, epilogue=3, share_a=share_a)
+    assert torch.equal(got, ref.to(torch.bfloat16))
+    bias = torch.randint(-3, 4, (batch, N), generator=gen, device="cuda").float()
+    got = _run(api, torch, A, B, M, N, K, batch, 0, 0, epilogue=1, bias=bias, share_a=share_a)
+    assert torch.equal(got, torch.relu(ref + bias[:, None, :].double()).to(torch.bfloat16))
+    assert api.lsgd_bgemm_check_device() == 0
