@@ -198,10 +198,11 @@ def workload_spec(args):
     raise SystemExit("unknown workload")
 
 
-# DRAM bytes per worker-parameter that the update kernels of the default workload moved in a hardware-counter
-# capture (dram read + write bytes of one launch divided by P * d): reads equal the algorithmic 8 B exactly; the
-# writes fall short of 4 B by the lines still dirty in the 126 MB L2 when the kernel ends.
-MEASURED_TRAFFIC_PER_WORKER_PARAM = {"pull": 11.24, "plain": 11.30}
+# DRAM bytes per worker-parameter that the update kernels of the default workload moved in a one-pass
+# hardware-counter capture of the full-size launch (dram read + write bytes divided by P * d = 2^30): reads are the
+# algorithmic 8 B exactly (8.59 GB); writes 4.24-4.25 GB of the algorithmic 4.29 GB, the rest being lines still
+# dirty in the 126 MB L2 when the kernel ends.  Quoted for that workload only (d = 2^26).
+MEASURED_TRAFFIC_PER_WORKER_PARAM = {"pull": 11.95, "plain": 11.96}
 NOMINAL_HBM_GBS = 7700.0     # the part's data-sheet HBM3e bandwidth, for context beside the measured copy bandwidth
 
 
@@ -486,7 +487,7 @@ def run_ours(args):
     peak, peak_src = read_peaks()
     achieved = alg_bytes / (upd_ms * 1e-3) / 1e9
     traffic = None
-    if spec["kind"] == "external" and args.arith == 0 and not alg1_mode and not with_momentum:
+    if spec["kind"] == "external" and args.arith == 0 and not alg1_mode and not with_momentum and d == (1 << 26):
         n_pull = sum(pull_flags)
         traffic = P * d * (n_pull * MEASURED_TRAFFIC_PER_WORKER_PARAM["pull"] +
                            (steps - n_pull) * MEASURED_TRAFFIC_PER_WORKER_PARAM["plain"]) / steps
@@ -718,7 +719,9 @@ def run_sharded(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=0,
+                    help="timed steps (default: 100 for c4; 1000-4000 for the small workloads, so that the timed "
+                         "region lasts a few tenths of a second and holds several clock samples)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4", "psd"])
@@ -741,6 +744,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
+    if args.steps <= 0:
+        args.steps = 100 if args.impl == "reference" else \
+            {"c4": 100, "c0": 4000, "c1": 2000, "c2": 4000, "c3": 1000, "psd": 2000}[args.workload]
     if args.impl == "reference":
         run_reference(args)
     elif args.sharded:
