@@ -636,7 +636,8 @@ def run_ours(args):
         osteps = {"external": 3, "quadratic": 3, "matcomp": 8, "mlp": 4, "psd": 4}[spec["kind"]]
         v, dt, what, osteps = oracle_sample_run(spec, osteps, 1, sample, min_seconds=10.0)
         cores = _threads_used() if spec["kind"] in ("mlp", "psd") else 1
-        allc = oracle_all_cores(spec, osteps, min(sample, 1 << 20) if (os.cpu_count() or 1) > 16 else sample)
+        # fewer steps for the all-cores leg: the processes share the memory system and run about three times longer
+        allc = oracle_all_cores(spec, max(2, osteps // 3), min(sample, 1 << 20) if (os.cpu_count() or 1) > 16 else sample)
         line["cpu_baseline"] = cpu_baseline_record(spec, v, cores, f"{osteps} steps x {what}, {dt:.1f} s", allc)
     if rank == 0:
         print(json.dumps(line), flush=True)
