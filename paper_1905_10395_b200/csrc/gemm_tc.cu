@@ -434,7 +434,7 @@ bgemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 // 128 x 256 tile needs -- and one thread of the leader CTA (cluster rank 0) issues tcgen05.mma.cta_group::2
 // (M = 256, N = 256, K = 16), which reads both CTAs' shared memory and writes both CTAs' tensor memory (each
 // holds its 128 rows x 256 columns of the accumulator).  A third less operand traffic from L2 per flop, which is
-// what bounds these products.  No load is multicast: every CTA fetches its own operand halves.
+// what bounds these products.  Every CTA fetches its own operand halves with ordinary tiled loads; no load is shared between CTAs.
 //
 // Synchronisation (all barriers live at the same shared-memory offsets in both CTAs):
 //   full[s]      leader only; one arrival (the leader's expect_tx) plus the bytes of BOTH CTAs' loads, which
