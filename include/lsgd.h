@@ -93,6 +93,10 @@ typedef struct {
   int32_t batch;             /* B, entries per worker per step                                       */
   int32_t n_heldout;
   const int32_t* heldout_pos;/* DEVICE int32[n_heldout] positions into the observed list             */
+  void* scratch;             /* DEVICE, 256-byte aligned, lsgd_matcomp_scratch_bytes(P, ld) bytes: the exact
+                                fixed-point gradient accumulator (8 bytes per worker-parameter), owned by the
+                                caller and cleared by lsgd_create.  NULL: the library allocates it itself     */
+  uint64_t scratch_bytes;
 } lsgd_matcomp_desc;
 
 /* Positive semi-definite low-rank completion, the paper's motivating example (Section 2.1; settings in
@@ -102,6 +106,10 @@ typedef struct {
 typedef struct {
   int32_t n, r;
   const float* M;            /* DEVICE float[n*n], row-major, symmetric; shared by all workers       */
+  void* scratch;             /* DEVICE, 256-byte aligned, lsgd_psd_scratch_bytes(r, P, ld) bytes (0 above rank 32):
+                                the fp64 partial gradients of the two CTAs that share a row block at small
+                                rank, owned by the caller.  NULL: the library allocates them itself          */
+  uint64_t scratch_bytes;
 } lsgd_psd_desc;
 
 /* MLP population: row i of x is [W1 | b1 | W2 | b2 | W3 | b3]; W_l is [n_out][n_in] row-major
@@ -212,9 +220,10 @@ typedef struct {
 
 /* Validates the configuration on the host, copies the group map, builds the group tables and
  * allocates O(P + G) words of device state plus reduction scratch for the objective's election
- * loss (MATCOMP additionally 8 bytes per worker-parameter for its order-independent gradient
- * accumulator; PSD_COMPLETION at ranks up to 64 additionally 16 bytes per worker-parameter for the two
- * partial gradients it combines).  Nothing is allocated after this call.  Returns LSGD_ERR_CUDA if no CUDA device is
+ * loss.  Large scratch is the caller's: the MLP's in lsgd_mlp_desc.scratch, MATCOMP's gradient accumulator
+ * (8 bytes per worker-parameter) and PSD_COMPLETION's partial gradients (16 bytes per worker-parameter at ranks
+ * up to 32) in the scratch field of their descriptors; only when that field is NULL does the library allocate
+ * the buffer itself, here.  Nothing is allocated after this call.  Returns LSGD_ERR_CUDA if no CUDA device is
  * usable.  *out is NULL on failure.                                                              */
 LSGD_API lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out);
 
@@ -363,6 +372,9 @@ LSGD_API lsgd_status lsgd_quadratic_loss_noalloc(const float* x, const float* a,
 LSGD_API lsgd_status lsgd_mlp_param_offsets(const int32_t* dims /* HOST int32[4] */, int64_t* w_off /* [3] */,
                                    int64_t* b_off /* [3] */, int64_t* d_out);
 LSGD_API uint64_t lsgd_mlp_scratch_bytes(const int32_t* dims, int32_t P, int32_t batch, int32_t n_heldout);
+/* Sizes of the caller-owned scratch of the MATCOMP and PSD_COMPLETION descriptors (host only).             */
+LSGD_API uint64_t lsgd_matcomp_scratch_bytes(int32_t P, int64_t ld);
+LSGD_API uint64_t lsgd_psd_scratch_bytes(int32_t r, int32_t P, int64_t ld);
 
 /* Batched bf16 x bf16 -> fp32-accumulate matrix product on the tensor cores: C[z] = A[z] . B[z] for
  * z < batch, C is M x N, contraction length K.  This is the product the MLP objective is built from

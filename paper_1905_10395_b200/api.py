@@ -36,11 +36,13 @@ class QuadraticDesc(C.Structure):
 class MatcompDesc(C.Structure):
     _fields_ = [("n_rows", C.c_int32), ("n_cols", C.c_int32), ("rank", C.c_int32), ("n_obs", C.c_int32),
                 ("obs_r", C.c_void_p), ("obs_c", C.c_void_p), ("obs_v", C.c_void_p), ("batch", C.c_int32),
-                ("n_heldout", C.c_int32), ("heldout_pos", C.c_void_p)]
+                ("n_heldout", C.c_int32), ("heldout_pos", C.c_void_p), ("scratch", C.c_void_p),
+                ("scratch_bytes", C.c_uint64)]
 
 
 class PsdDesc(C.Structure):
-    _fields_ = [("n", C.c_int32), ("r", C.c_int32), ("M", C.c_void_p)]
+    _fields_ = [("n", C.c_int32), ("r", C.c_int32), ("M", C.c_void_p), ("scratch", C.c_void_p),
+                ("scratch_bytes", C.c_uint64)]
 
 
 class MlpDesc(C.Structure):
@@ -120,6 +122,10 @@ def lib() -> C.CDLL:
         L.lsgd_mlp_param_offsets.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int64)]
         L.lsgd_mlp_scratch_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32]
         L.lsgd_mlp_scratch_bytes.restype = C.c_uint64
+        L.lsgd_matcomp_scratch_bytes.argtypes = [C.c_int32, C.c_int64]
+        L.lsgd_matcomp_scratch_bytes.restype = C.c_uint64
+        L.lsgd_psd_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int64]
+        L.lsgd_psd_scratch_bytes.restype = C.c_uint64
         for name in ("lsgd_create", "lsgd_grad", "lsgd_elect", "lsgd_step", "lsgd_destroy", "lsgd_get_leaders",
                      "lsgd_get_loss", "lsgd_get_step", "lsgd_get_leader_counts", "lsgd_check_device",
                      "lsgd_set_eta", "lsgd_mlp_param_offsets"):
@@ -201,6 +207,14 @@ def mlp_param_offsets(dims: Sequence[int]):
 def mlp_scratch_bytes(dims: Sequence[int], P: int, batch: int, n_heldout: int) -> int:
     d4 = (C.c_int32 * 4)(*dims)
     return int(lib().lsgd_mlp_scratch_bytes(d4, P, batch, n_heldout))
+
+
+def matcomp_scratch_bytes(P: int, ld: int) -> int:
+    return int(lib().lsgd_matcomp_scratch_bytes(int(P), int(ld)))
+
+
+def psd_scratch_bytes(r: int, P: int, ld: int) -> int:
+    return int(lib().lsgd_psd_scratch_bytes(int(r), int(P), int(ld)))
 
 
 def make_config(*, P: int, G: int, group_of: np.ndarray, d: int, ld: int, eta: float, lambda_l: float,

@@ -229,4 +229,5 @@ struct lsgd_ctx {
   unsigned long long* d_acc64;  // MATCOMP: fixed-point gradient accumulator [P*ld], kept all-zero between steps
   bool mc_step_pending;         // MATCOMP fused step: the gradient sums wait in d_acc64 for lsgd_step
   double* d_psd_part;           // PSD, small ranks: partial gradients of the CTAs that share a row block
+  bool owns_acc64, owns_psd_part;   // false: the buffer is the caller's (descriptor scratch field)
 };

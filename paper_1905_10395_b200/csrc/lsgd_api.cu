@@ -82,6 +82,10 @@ lsgd_status validate(const lsgd_config* c) {
       if ((int64_t)(m->n_rows + (int64_t)m->n_cols) * m->rank != c->d) return LSGD_ERR_INVALID_ARG;
       if (m->rank > 32) return LSGD_ERR_UNSUPPORTED;
       if (m->batch > (1 << 15)) return LSGD_ERR_UNSUPPORTED;   // range of the fixed-point gradient accumulator
+      if (m->scratch) {
+        if (reinterpret_cast<uintptr_t>(m->scratch) & 255u) return LSGD_ERR_ALIGNMENT;
+        if (m->scratch_bytes < lsgd_matcomp_scratch_bytes(c->P, c->ld)) return LSGD_ERR_INVALID_ARG;
+      }
       break;
     }
     case LSGD_OBJ_PSD_COMPLETION: {
@@ -89,6 +93,10 @@ lsgd_status validate(const lsgd_config* c) {
       if (!m || !c->g || !m->M || m->n < 1 || m->r < 1) return LSGD_ERR_INVALID_ARG;
       if ((int64_t)m->n * m->r != c->d) return LSGD_ERR_INVALID_ARG;
       if (m->r > 128) return LSGD_ERR_UNSUPPORTED;
+      if (m->scratch) {
+        if (reinterpret_cast<uintptr_t>(m->scratch) & 255u) return LSGD_ERR_ALIGNMENT;
+        if (m->scratch_bytes < lsgd_psd_scratch_bytes(m->r, c->P, c->ld)) return LSGD_ERR_INVALID_ARG;
+      }
       break;
     }
     case LSGD_OBJ_MLP: {
@@ -141,6 +149,8 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   h->mlp_state = nullptr;
   h->d_acc64 = nullptr;
   h->d_psd_part = nullptr;
+  h->owns_acc64 = false;
+  h->owns_psd_part = false;
   std::memset(&h->quad, 0, sizeof(h->quad));
   std::memset(&h->mc, 0, sizeof(h->mc));
   std::memset(&h->mlp, 0, sizeof(h->mlp));
@@ -214,13 +224,23 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
   ok = ok && cudaStreamSynchronize(h->stream) == cudaSuccess;
   if (ok && cfg->objective == LSGD_OBJ_MLP) ok = (mlp_create(h) == LSGD_OK);
   if (ok && cfg->objective == LSGD_OBJ_MATCOMP) {
-    const size_t bytes = sizeof(unsigned long long) * (size_t)P * (size_t)cfg->ld;
-    ok = cudaMalloc(reinterpret_cast<void**>(&h->d_acc64), bytes) == cudaSuccess &&
-         cudaMemsetAsync(h->d_acc64, 0, bytes, h->stream) == cudaSuccess;
+    const size_t bytes = (size_t)lsgd_matcomp_scratch_bytes(P, cfg->ld);
+    if (h->mc.scratch) {
+      h->d_acc64 = static_cast<unsigned long long*>(h->mc.scratch);           // the caller's buffer
+    } else {
+      ok = cudaMalloc(reinterpret_cast<void**>(&h->d_acc64), bytes) == cudaSuccess;
+      h->owns_acc64 = ok;
+    }
+    ok = ok && cudaMemsetAsync(h->d_acc64, 0, bytes, h->stream) == cudaSuccess;
   }
-  if (ok && cfg->objective == LSGD_OBJ_PSD_COMPLETION && psd_split(h->psd.r) > 1)
-    ok = cudaMalloc(reinterpret_cast<void**>(&h->d_psd_part),
-                    sizeof(double) * (size_t)psd_split(h->psd.r) * (size_t)P * (size_t)cfg->ld) == cudaSuccess;
+  if (ok && cfg->objective == LSGD_OBJ_PSD_COMPLETION && psd_split(h->psd.r) > 1) {
+    if (h->psd.scratch) {
+      h->d_psd_part = static_cast<double*>(h->psd.scratch);
+    } else {
+      ok = cudaMalloc(reinterpret_cast<void**>(&h->d_psd_part), (size_t)lsgd_psd_scratch_bytes(h->psd.r, P, cfg->ld)) == cudaSuccess;
+      h->owns_psd_part = ok;
+    }
+  }
   // EAGD: rows 0 .. G-1 of leader_copies are read (with a zero coefficient) before the library writes them all
   if (ok && (cfg->flags & LSGD_FLAG_EAGD))
     ok = cudaMemsetAsync(cfg->leader_copies, 0, sizeof(float) * (size_t)(G + 1) * (size_t)cfg->ld, h->stream) == cudaSuccess;
@@ -229,8 +249,8 @@ lsgd_status lsgd_create(const lsgd_config* cfg, lsgd_handle* out) {
     ok = cudaMemsetAsync(cfg->g, 0, sizeof(float) * (size_t)P * (size_t)cfg->ld, h->stream) == cudaSuccess;
   if (!ok) {
     if (h->mlp_state) mlp_destroy(h);
-    cudaFree(h->d_acc64);
-    cudaFree(h->d_psd_part);
+    if (h->owns_acc64) cudaFree(h->d_acc64);
+    if (h->owns_psd_part) cudaFree(h->d_psd_part);
     cudaFree(h->slab);
     delete h;
     return LSGD_ERR_CUDA;
@@ -532,8 +552,8 @@ lsgd_status lsgd_destroy(lsgd_handle h) {
   if (!h) return LSGD_OK;
   cudaStreamSynchronize(h->stream);
   if (h->mlp_state) mlp_destroy(h);
-  cudaFree(h->d_acc64);
-  cudaFree(h->d_psd_part);
+  if (h->owns_acc64) cudaFree(h->d_acc64);
+  if (h->owns_psd_part) cudaFree(h->d_psd_part);
   cudaError_t e = cudaFree(h->slab);
   delete h;
   return e == cudaSuccess ? LSGD_OK : LSGD_ERR_CUDA;
@@ -646,6 +666,16 @@ lsgd_status lsgd_selftest_wait_timeout(lsgd_handle h, int64_t budget_cycles, int
   LSGD_CUDA(cudaStreamSynchronize(h->stream));
   LSGD_CUDA(cudaMemcpy(gave_up, h->d_selftest, sizeof(int32_t), cudaMemcpyDeviceToHost));
   return LSGD_OK;
+}
+
+uint64_t lsgd_matcomp_scratch_bytes(int32_t P, int64_t ld) {
+  if (P < 1 || ld < 1) return 0;
+  return sizeof(unsigned long long) * (uint64_t)P * (uint64_t)ld;
+}
+
+uint64_t lsgd_psd_scratch_bytes(int32_t r, int32_t P, int64_t ld) {
+  if (r < 1 || P < 1 || ld < 1 || psd_split(r) <= 1) return 0;
+  return sizeof(double) * (uint64_t)psd_split(r) * (uint64_t)P * (uint64_t)ld;
 }
 
 lsgd_status lsgd_center(lsgd_handle h, float* center) {

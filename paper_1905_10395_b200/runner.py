@@ -53,16 +53,20 @@ class Population:
             self.obs_c = torch.from_numpy(A["obs_c"]).to(dev)
             self.obs_v = torch.from_numpy(A["obs_v"]).to(dev)
             self.held = torch.from_numpy(A["heldout_pos"]).to(dev)
+            # the gradient accumulator is the caller's, like every large buffer
+            self.scratch = torch.empty(api.matcomp_scratch_bytes(w.P, w.ld), dtype=torch.uint8, device=dev)
             desc = api.MatcompDesc(m["n_rows"], m["n_cols"], m["rank"], len(A["obs_r"]), self.obs_r.data_ptr(),
                                    self.obs_c.data_ptr(), self.obs_v.data_ptr(), m["batch"], len(A["heldout_pos"]),
-                                   self.held.data_ptr())
+                                   self.held.data_ptr(), self.scratch.data_ptr(), self.scratch.numel())
             self.batches = [torch.from_numpy(np.ascontiguousarray(p)).to(dev) for p in A["batch_pos"]]
             if self.g is None:
                 self.g = torch.empty_like(self.x)
         elif w.objective == "psd":
             obj = api.OBJ_PSD_COMPLETION
             self.M = torch.from_numpy(A["M"]).to(dev)
-            desc = api.PsdDesc(w.meta["n"], w.meta["r"], self.M.data_ptr())
+            nbytes = api.psd_scratch_bytes(w.meta["r"], w.P, w.ld)
+            self.scratch = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
+            desc = api.PsdDesc(w.meta["n"], w.meta["r"], self.M.data_ptr(), self.scratch.data_ptr() if nbytes else None, nbytes)
             if self.g is None:
                 self.g = torch.empty_like(self.x)
         elif w.objective == "mlp":

@@ -73,9 +73,26 @@ def test_create_rejects_shapes_beyond_the_documented_capacities(api):
     h = C.c_void_p()
     assert api.lib().lsgd_create(C.byref(cfg), C.byref(h)) == api.ERR_UNSUPPORTED
     # matrix-completion batch beyond the range of the fixed-point accumulator
-    desc = api.MatcompDesc(10, 10, 5, 50, 4096, 4096, 4096, (1 << 15) + 1, 8, 4096)
+    desc = api.MatcompDesc(10, 10, 5, 50, 4096, 4096, 4096, (1 << 15) + 1, 8, 4096, None, 0)
     cfg, keep = _cfg(api, d=100, objective=api.OBJ_MATCOMP, desc=desc)
     assert api.lib().lsgd_create(C.byref(cfg), C.byref(h)) == api.ERR_UNSUPPORTED
+
+
+def test_caller_owned_scratch_is_validated_on_the_host(api):
+    P, ld = 4, 128
+    need = api.matcomp_scratch_bytes(P, ld)
+    assert need == 8 * P * ld
+    h = C.c_void_p()
+    for scratch, nbytes, status in [(4096 + 8, need, api.ERR_ALIGNMENT), (4096, need - 1, api.ERR_INVALID_ARG)]:
+        desc = api.MatcompDesc(10, 10, 5, 50, 4096, 4096, 4096, 16, 8, 4096, scratch, nbytes)
+        cfg, keep = _cfg(api, d=100, objective=api.OBJ_MATCOMP, desc=desc)
+        assert api.lib().lsgd_create(C.byref(cfg), C.byref(h)) == status
+    assert api.psd_scratch_bytes(100, 8, 100000) == 0                    # large ranks need none
+    need = api.psd_scratch_bytes(10, 4, 128)                             # two fp64 partial gradients at small rank
+    assert need == 16 * 4 * 128
+    desc = api.PsdDesc(10, 10, 4096, 8192, need - 8)
+    cfg, keep = _cfg(api, d=100, objective=api.OBJ_PSD_COMPLETION, desc=desc)
+    assert api.lib().lsgd_create(C.byref(cfg), C.byref(h)) == api.ERR_INVALID_ARG
 
 
 def test_device_flag_bits_match_the_header(api):
