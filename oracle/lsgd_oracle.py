@@ -26,9 +26,10 @@ Readings of the paper taken here (each is also exercised by a pin in tests/test_
   * Nesterov momentum and weight decay (Section 4.1) act on the gradient step only; the pulls stay outside
     the momentum buffer (momentum_update).
 
-Pins: see tests/test_oracle_pins.py.  Parity unpinned (self-consistent definitions only, no
-external fact fixes them): the placement of bf16 roundings in the MLP objective's "bf16emu" mode,
-and the 1/(2|B|) / 1/N constants of the observed-entry matrix-completion objective.
+Pins: see tests/test_oracle_pins.py, test_oracle_algorithm1.py, test_oracle_momentum.py, test_oracle_eagd.py.
+Parity unpinned (self-consistent definitions only, no external fact fixes them): the placement of bf16
+roundings in the backward pass of the MLP objective's "bf16emu" mode, and the 1/(2|B|) / 1/N constants of
+the observed-entry matrix-completion objective.
 """
 from __future__ import annotations
 

@@ -469,6 +469,30 @@ def test_mlp_bf16emu_is_close_to_fp32_and_rounding_matches_library():
     assert not np.array_equal(g32, g16)
 
 
+def test_mlp_bf16emu_rounds_operands_only():
+    """Where every matrix-product operand is exactly representable in bfloat16 -- small integers for the data, the
+    weights and hence the hidden activations -- rounding the operands changes nothing: the bf16-emulation mode must
+    give the fp32 mode's losses bit for bit (forward pass and held-out loss), and its gradient of the last layer,
+    whose operands are the representable activations and the rounded dZ, must be the fp32 mode's within the one
+    rounding of dZ (2^-9 relative)."""
+    w, segs, o32 = _tiny_mlp("fp32")
+    rng = np.random.default_rng(4)
+    A = w.arrays
+    A["pool_x"][...] = rng.integers(-3, 4, A["pool_x"].shape).astype(F32)
+    A["held_x"][...] = rng.integers(-3, 4, A["held_x"].shape).astype(F32)
+    x0 = w.x0.copy()
+    x0[...] = rng.integers(-2, 3, x0.shape).astype(F32)
+    o16 = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="bf16emu")
+    o32 = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="fp32")
+    assert np.array_equal(o16.loss(x0, 0), o32.loss(x0, 0))
+    g16, g32 = o16.grad(x0, 0), o32.grad(x0, 0)
+    assert np.array_equal(o16.last_train_loss, o32.last_train_loss)
+    s3 = segs[-1]
+    a, b = g16[:, s3["w"]:s3["w"] + s3["n_in"] * s3["n_out"]], g32[:, s3["w"]:s3["w"] + s3["n_in"] * s3["n_out"]]
+    assert np.abs(a - b).max() <= 2.0 ** -8 * np.abs(b).max() + 1e-12
+    assert np.abs(b).max() > 0
+
+
 # ---- center variable = plain average of the workers (Section 4.1) ---------------------------------
 def test_center_variable_is_the_average():
     rng = np.random.default_rng(8)
