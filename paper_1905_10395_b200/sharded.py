@@ -112,8 +112,16 @@ class CudaShardEngine:
     def is_pull_step(self) -> bool:
         return self.t % self.w.tau == 0
 
+    def _make_current(self) -> None:
+        # the library refuses calls on a handle while another device is current (engines of several devices may
+        # live in one process, as in run_lockstep)
+        import torch
+        if torch.cuda.current_device() != self.dev.index:
+            torch.cuda.set_device(self.dev)
+
     def begin_step(self) -> bool:
         """Gradient; on a pull step also the local election and this rank's key.  True on a pull step."""
+        self._make_current()
         batch = self.batches[self.t % len(self.batches)] if self.batches else None
         self.lsgd.grad(batch)
         if not self.is_pull_step():
@@ -137,6 +145,7 @@ class CudaShardEngine:
     def pick_global(self, keys, world: int):
         """From all ranks' keys: the winning rank and the winner's global worker index; sets this rank's global
         leader (own winner or guest row) on the device.  The one host synchronisation of a pull step."""
+        self._make_current()
         winner, gidx, self._best_local = self.lsgd.shard_pick_global(keys, world, self.shard.rank, self.shard.guest)
         self.global_leader_global = gidx
         return winner, gidx
@@ -156,6 +165,7 @@ class CudaShardEngine:
         return self.x[self.shard.guest]
 
     def finish_step(self) -> None:
+        self._make_current()
         self.lsgd.step()
         self.t += 1
 

@@ -31,7 +31,8 @@ o = orc.LsgdOracle(w.x0, orc.External(w.arrays["g"], w.arrays["loss_ring"]), w.g
 o.run(steps)
 same = bool(np.array_equal(eng.x_local().view(np.uint32), o.x[eng.shard.workers].view(np.uint32)))
 want = [h["gl"] for h in o.history]
-print(json.dumps({"rank": rank, "world": world, "rows_equal": same, "leaders": leaders, "want": want,
-                  "workers": eng.shard.workers.tolist()}), flush=True)
+sys.stdout.write(json.dumps({"rank": rank, "world": world, "rows_equal": same, "leaders": leaders, "want": want,
+                             "workers": eng.shard.workers.tolist()}) + "\n")
+sys.stdout.flush()
 dist.barrier()
 dist.destroy_process_group()

@@ -80,6 +80,21 @@ def _free_port():
         return s.getsockname()[1]
 
 
+def _json_objects(text):
+    """Every JSON object in the ranks' joint output (two ranks may write on one line)."""
+    dec, out, pos = json.JSONDecoder(), [], 0
+    while True:
+        pos = text.find("{", pos)
+        if pos < 0:
+            return out
+        try:
+            obj, end = dec.raw_decode(text, pos)
+            out.append(obj)
+            pos = end
+        except json.JSONDecodeError:
+            pos += 1
+
+
 def test_two_gloo_ranks_exchange_the_global_leader():
     for attempt in range(2):                             # the probed port can be taken before the ranks bind it
         cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2", "--master-addr",
@@ -88,7 +103,7 @@ def test_two_gloo_ranks_exchange_the_global_leader():
         if r.returncode == 0:
             break
     assert r.returncode == 0, r.stderr[-3000:]
-    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    lines = _json_objects(r.stdout)
     assert sorted(l["rank"] for l in lines) == [0, 1]
     owners = set()
     for l in lines:
