@@ -330,14 +330,20 @@ def test_election_on_the_running_mean_of_training_losses():
     pop.close()
 
 
-@pytest.mark.parametrize("fused", [False, True])
-def test_cuda_graph_replay_of_the_mlp_step_equals_the_call_by_call_run(fused):
+@pytest.mark.parametrize("fused,big", [(False, False), (True, False), (True, True)])
+def test_cuda_graph_replay_of_the_mlp_step_equals_the_call_by_call_run(fused, big):
     """Whole periods of the MLP step (tensor-core products, programmatic dependent launches, the fused step)
-    captured into a CUDA graph and replayed give the same parameters, bit for bit, as issuing the calls."""
+    captured into a CUDA graph and replayed give the same parameters, bit for bit, as issuing the calls.
+    big: 1024-wide layers and a held-out batch of 1024 for 10 workers, so that the held-out forward runs on the
+    CTA-pair kernel (cluster launches inside the capture) and decides the elections of every period."""
     import torch
     from paper_1905_10395_b200 import api
     from paper_1905_10395_b200.runner import Population
-    w = inputs.make_mlp(4, 2, dims=(64, 128, 128, 10), pool=512, heldout=128, batch=128, steps=4, tau=2, config_id=63)
+    if big:
+        w = inputs.make_mlp(10, 2, dims=(64, 1024, 1024, 10), pool=512, heldout=1024, batch=128, steps=4, tau=2,
+                            config_id=64)
+    else:
+        w = inputs.make_mlp(4, 2, dims=(64, 128, 128, 10), pool=512, heldout=128, batch=128, steps=4, tau=2, config_id=63)
     flags = api.FLAG_MLP_FUSED_STEP if fused else 0
     stream = torch.cuda.Stream()
     a = Population(w, flags=flags, stream=stream)
