@@ -439,6 +439,7 @@ def run_ours(args):
     ev0.record()
     n_launch = 0
     pull_flags = []
+    e_ev = []                                    # MLP: events around the held-out election
     for s in range(steps):
         t = pop.t
         batch = pop.batches[t % len(pop.batches)] if pop.batches else None
@@ -461,7 +462,12 @@ def run_ours(args):
                 n_launch += 1 + 2 * (int(loc) + int(glo))
             continue
         if t % spec["tau"] == 0:
+            if spec["kind"] == "mlp":
+                e_ev.append((torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)))
+                e_ev[-1][0].record()
             pop.lsgd.elect(pop.loss_ring[pop.n_elections % pop.loss_ring.shape[0]] if pop.loss_ring is not None else None)
+            if spec["kind"] == "mlp":
+                e_ev[-1][1].record()
             pop.n_elections += 1
         k_ev[s][0].record()
         pop.lsgd.step()
@@ -534,6 +540,17 @@ def run_ours(args):
                     "tensor_tflops": P * mflops / (g_ms * 1e-3) / 1e12,
                     "tensor_peak_tflops": t_peak, "tensor_peak_source": t_src,
                     "tensor_frac": P * mflops / (g_ms * 1e-3) / 1e12 / t_peak}
+        if e_ev:
+            # the held-out election: its two hidden-layer products (M = held-out batch per worker) are the
+            # tensor-bound part of this workload; their flops over the whole election call
+            d0, d1, d2, d3 = [int(v) for v in w.meta["dims"]]
+            n_h = int(w.arrays["held_y"].shape[0])
+            e_ms = float(np.mean([a.elapsed_time(b) for a, b in e_ev]))
+            e_flops = 2.0 * P * n_h * (d0 * d1 + d1 * d2 + d2 * d3)
+            roofline["election"] = {"bound": "tensor", "kernel": "bgemm_pair_kernel (two hidden-layer products) + logits + softmax + election",
+                                    "ms_per_election": e_ms, "elections": len(e_ev), "flops_per_election": e_flops,
+                                    "achieved": e_flops / (e_ms * 1e-3) / 1e12, "peak": t_peak, "peak_source": t_src,
+                                    "unit": "TFLOP/s", "frac": e_flops / (e_ms * 1e-3) / 1e12 / t_peak}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": elapsed_ms / steps, "steps_per_s": steps * world / (elapsed_ms * 1e-3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
