@@ -313,13 +313,13 @@ LSGD_API lsgd_status lsgd_get_leader_counts(lsgd_handle h, int32_t* global_count
 #define LSGD_DEVFLAG_OVERFLOW 8u
 LSGD_API lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out /* HOST, may be NULL */);
 /* Self-test of the bounded device waits (test support; the paper has no counterpart).  Every wait of the
- * copy pipelines in the update kernels is limited by a clock budget after which the kernel records
- * LSGD_DEVFLAG_WAIT_TIMEOUT and returns instead of hanging.  This call runs that same wait routine in a
- * one-warp kernel on a barrier that nothing completes (no copy is in flight), with a budget of budget_cycles
- * clock cycles (1 .. 10^8, LSGD_ERR_INVALID_ARG otherwise), synchronises the stream and stores 1 in
- * *gave_up (HOST) if the wait ran out.  The status word keeps the bit until lsgd_check_device reads it;
- * the context stays usable.                                                                          */
-LSGD_API lsgd_status lsgd_selftest_wait_timeout(lsgd_handle h, int64_t budget_cycles, int32_t* gave_up);
+ * copy pipelines in the update kernels and of the copy / tensor-core pipelines in the product kernels is limited
+ * by a clock budget after which the kernel records LSGD_DEVFLAG_WAIT_TIMEOUT and returns instead of hanging.
+ * This call runs that same wait routine (which = 0: the update kernels', 1: the product kernels') in a one-warp
+ * kernel on a barrier that nothing completes (no copy is in flight), with a budget of budget_cycles clock cycles
+ * (1 .. 10^8, LSGD_ERR_INVALID_ARG otherwise), synchronises the stream and stores 1 in *gave_up (HOST) if the
+ * wait ran out.  The status word keeps the bit until lsgd_check_device reads it; the context stays usable.  */
+LSGD_API lsgd_status lsgd_selftest_wait_timeout(lsgd_handle h, int32_t which, int64_t budget_cycles, int32_t* gave_up);
 /* The "center variable" the paper reports at test time for LSGD (Section 4.1): the average of the
  * parameters of all workers, center[k] = (1/P) sum_i x[i][k], summed in worker order in fp64 and rounded
  * once.  center: DEVICE float[ld] (columns d..ld-1 are written as the mean of the padding).  Enqueued

@@ -108,7 +108,7 @@ def lib() -> C.CDLL:
         L.lsgd_shard_pick_global.restype = C.c_int
         L.lsgd_mlp_get_activations.argtypes = [H, C.c_void_p, C.c_void_p]
         L.lsgd_mlp_get_activations.restype = C.c_int
-        L.lsgd_selftest_wait_timeout.argtypes = [H, C.c_int64, C.POINTER(C.c_int32)]
+        L.lsgd_selftest_wait_timeout.argtypes = [H, C.c_int32, C.c_int64, C.POINTER(C.c_int32)]
         L.lsgd_selftest_wait_timeout.restype = C.c_int
         L.lsgd_bgemm_check_device.argtypes = [C.POINTER(C.c_uint32)]
         L.lsgd_bgemm_check_device.restype = C.c_int
@@ -330,10 +330,12 @@ class Lsgd:
             raise LsgdError(s, "lsgd_check_device")
         return f.value
 
-    def selftest_wait_timeout(self, budget_cycles: int) -> int:
-        """Runs the update pipeline's bounded wait on a barrier nothing completes; 1 if the wait ran out."""
+    def selftest_wait_timeout(self, budget_cycles: int, which: int = 0) -> int:
+        """Runs a pipeline's bounded wait (which = 0: update kernels, 1: product kernels) on a barrier nothing
+        completes; 1 if the wait ran out."""
         out = C.c_int32(-1)
-        _check(lib().lsgd_selftest_wait_timeout(self.h, int(budget_cycles), C.byref(out)), "lsgd_selftest_wait_timeout")
+        _check(lib().lsgd_selftest_wait_timeout(self.h, int(which), int(budget_cycles), C.byref(out)),
+               "lsgd_selftest_wait_timeout")
         return out.value
 
     def set_eta(self, eta: float):

@@ -74,13 +74,14 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false after the clock budget (or when another role has aborted).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t* status,
+                                          long long budget = kWaitBudgetCycles) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitBudgetCycles) {
+    if (clock64() - t0 > budget) {
       *abort_flag = 1;
       atomicOr(status, FLAG_WAIT_TIMEOUT);
       return false;
@@ -672,6 +673,24 @@ bgemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   }
 }
 
+// Self-test of the bounded wait of the product kernels: one warp waits, with a short budget, on a barrier that
+// nothing completes (no copy or product is in flight), so the wait runs out, sets the status bit and returns.
+__global__ void __launch_bounds__(32) gemm_wait_timeout_selftest_kernel(uint32_t* status, long long budget, int* gave_up) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(&bar, 1);
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(&bar, 0, &abort_flag, status, budget);
+  __syncwarp();
+  if (threadIdx.x == 0) {
+    *gave_up = ok ? 0 : 1;
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&bar)) : "memory");
+  }
+}
+
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -719,6 +738,11 @@ bool make_tile_map_f32(CUtensorMap* map, const void* base, int64_t N, int64_t M,
 bool make_tile_map_bf16(CUtensorMap* map, const void* base, int64_t N, int64_t M, int64_t pitch_elems, int64_t batch,
                         int64_t batch_stride_elems) {
   return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, N, M, pitch_elems, batch, batch_stride_elems, 64, 128);
+}
+
+cudaError_t launch_gemm_wait_timeout_selftest(uint32_t* status, long long budget_cycles, int* gave_up, cudaStream_t s) {
+  gemm_wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status, budget_cycles, gave_up);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_bgemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmShape& p, cudaStream_t s) {

@@ -90,6 +90,8 @@ cudaError_t launch_momentum_update_chunked(const UpdateArgs& a, cudaStream_t s);
 // One warp runs the update pipeline's bounded barrier wait on a barrier nothing completes: *gave_up (DEVICE) <- 1
 // and FLAG_WAIT_TIMEOUT in *status after about budget_cycles clock cycles.
 cudaError_t launch_wait_timeout_selftest(uint32_t* status, long long budget_cycles, int* gave_up, cudaStream_t s);
+// the same for the bounded wait of the tensor-core product kernels (gemm_tc.cu)
+cudaError_t launch_gemm_wait_timeout_selftest(uint32_t* status, long long budget_cycles, int* gave_up, cudaStream_t s);
 cudaError_t launch_center(const float* x, float* center, int32_t P, int64_t d, int64_t ld, cudaStream_t s);
 
 // out[k] <- (1 - kk) center[k] + kk * mean_i x[i][k] over all ld columns (EAGD center rule, kk = P eta lambda)

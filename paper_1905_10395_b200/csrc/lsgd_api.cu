@@ -658,11 +658,15 @@ lsgd_status lsgd_check_device(lsgd_handle h, uint32_t* flag_out) {
   return f ? LSGD_ERR_DEVICE_FLAG : LSGD_OK;
 }
 
-lsgd_status lsgd_selftest_wait_timeout(lsgd_handle h, int64_t budget_cycles, int32_t* gave_up) {
+lsgd_status lsgd_selftest_wait_timeout(lsgd_handle h, int32_t which, int64_t budget_cycles, int32_t* gave_up) {
   if (!h || !gave_up) return LSGD_ERR_INVALID_ARG;
+  if (which < 0 || which > 1) return LSGD_ERR_INVALID_ARG;
   if (budget_cycles < 1 || budget_cycles > 100000000) return LSGD_ERR_INVALID_ARG;   // at most ~50 ms
   if (!on_own_device(h)) return LSGD_ERR_STATE;
-  LSGD_CUDA(launch_wait_timeout_selftest(h->d_status, (long long)budget_cycles, h->d_selftest, h->stream));
+  if (which == 0)
+    LSGD_CUDA(launch_wait_timeout_selftest(h->d_status, (long long)budget_cycles, h->d_selftest, h->stream));
+  else
+    LSGD_CUDA(launch_gemm_wait_timeout_selftest(h->d_status, (long long)budget_cycles, h->d_selftest, h->stream));
   LSGD_CUDA(cudaStreamSynchronize(h->stream));
   LSGD_CUDA(cudaMemcpy(gave_up, h->d_selftest, sizeof(int32_t), cudaMemcpyDeviceToHost));
   return LSGD_OK;

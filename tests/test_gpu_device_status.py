@@ -30,9 +30,10 @@ def test_bounded_wait_runs_out_and_is_reported_and_the_handle_still_works():
     pop = Population(w)
     pop.run(2)
     assert pop.lsgd.check_device() == 0
-    assert pop.lsgd.selftest_wait_timeout(100_000) == 1            # the wait gave up after ~50 us
-    assert pop.lsgd.check_device() == api.DEVFLAG_WAIT_TIMEOUT     # LSGD_ERR_DEVICE_FLAG with this bit
-    assert pop.lsgd.check_device() == 0                            # reading clears it
+    for which in (0, 1):                                           # the update kernels' wait, the product kernels' wait
+        assert pop.lsgd.selftest_wait_timeout(100_000, which) == 1     # the wait gave up after ~50 us
+        assert pop.lsgd.check_device() == api.DEVFLAG_WAIT_TIMEOUT     # LSGD_ERR_DEVICE_FLAG with this bit
+        assert pop.lsgd.check_device() == 0                            # reading clears it
     with pytest.raises(api.LsgdError) as e:
         pop.lsgd.selftest_wait_timeout(10 ** 9)                    # budgets are capped
     assert e.value.status == api.ERR_INVALID_ARG
