@@ -194,7 +194,9 @@ def workload_spec(args):
         r = args.rank
         return dict(kind="psd", cfg=5, P=8, G=1, d=1000 * r, n=1000, r=r, eta=5e-4, lambda_l=0.2, lambda_g=0.0,
                     tau=args.tau or 1, name=f"PSD completion (the paper's experiment): 8 workers, n=1000, rank {r}, "
-                    "eta 5e-4, lambda 1/5, tau 1", launches=(3, 2))
+                    "eta 5e-4, lambda 1/5, tau 1",
+                    # gradient (+ the combine of the two partial gradients up to rank 32), election, update
+                    launches=(4, 3) if r <= 32 else (3, 2))
     raise SystemExit("unknown workload")
 
 
