@@ -117,6 +117,14 @@ def test_null_handles(api):
     assert L.lsgd_step(None) == api.ERR_INVALID_ARG
     assert L.lsgd_destroy(None) == api.OK
     assert api.status_string(api.ERR_STATE)
+    out = (C.c_int32 * 3)()
+    assert L.lsgd_shard_best_key(None, 1, None, None) == api.ERR_INVALID_ARG
+    assert L.lsgd_shard_pick_global(None, None, 1, 0, 0, out) == api.ERR_INVALID_ARG
+    assert L.lsgd_selftest_wait_timeout(None, 0, 1000, out) == api.ERR_INVALID_ARG
+    assert L.lsgd_mlp_get_activations(None, None, None) == api.ERR_INVALID_ARG
+    assert L.lsgd_set_leaders(None, None, 0) == api.ERR_INVALID_ARG
+    assert L.lsgd_center(None, None) == api.ERR_INVALID_ARG
+    assert api.matcomp_scratch_bytes(0, 32) == 0 and api.psd_scratch_bytes(0, 1, 32) == 0
 
 
 def test_mlp_offsets_match_the_input_generator_layout(api):
