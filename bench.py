@@ -135,6 +135,14 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def host_cores() -> int:
+    """Cores this process may run on (the affinity mask where the platform has one, else the core count)."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
 def _threads_used() -> int:
     """Threads the oracle's NumPy can use: 1 for its element-wise loops; BLAS threads for matmuls."""
     try:
@@ -309,7 +317,7 @@ def oracle_all_cores(spec, steps, sample_cols, n_proc=None):
     if spec["kind"] not in ("external", "quadratic"):
         return None
     import multiprocessing as mp
-    n_proc = n_proc or os.cpu_count() or 1
+    n_proc = n_proc or host_cores()
     ctx = mp.get_context("spawn")
     barrier, out = ctx.Barrier(n_proc), ctx.Queue()
     cols = int(min(sample_cols, spec["d"]))
@@ -345,7 +353,7 @@ def cpu_baseline_record(spec, value, cores, sample, all_cores=None):
         rec = {"value": v, "unit": UNIT, "cores": n, "kind": "oracle",
                "sample": f"{n} processes, each: {sample.split(', ')[0]}; {dt:.1f} s",
                "single_core": {"value": value, "cores": cores, "sample": sample},
-               "host_cores": os.cpu_count()}
+               "host_cores": host_cores()}
     return rec
 
 
@@ -365,7 +373,7 @@ def run_reference(args):
         "config": {"workload": spec["name"], "tau": spec["tau"],
                    "sample": f"each step covers {what}"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"{steps} steps x {what}", "host_cores": os.cpu_count()},
+                         "sample": f"{steps} steps x {what}", "host_cores": host_cores()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -656,7 +664,7 @@ def run_ours(args):
         v, dt, what, osteps = oracle_sample_run(spec, osteps, 1, sample, min_seconds=10.0)
         cores = _threads_used() if spec["kind"] in ("mlp", "psd") else 1
         # fewer steps for the all-cores leg: the processes share the memory system and run about three times longer
-        allc = oracle_all_cores(spec, max(2, osteps // 3), min(sample, 1 << 20) if (os.cpu_count() or 1) > 16 else sample)
+        allc = oracle_all_cores(spec, max(2, osteps // 3), min(sample, 1 << 20) if host_cores() > 16 else sample)
         line["cpu_baseline"] = cpu_baseline_record(spec, v, cores, f"{osteps} steps x {what}, {dt:.1f} s", allc)
     if rank == 0:
         print(json.dumps(line), flush=True)
