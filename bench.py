@@ -204,7 +204,7 @@ def workload_spec(args):
                     tau=args.tau or 1, name=f"PSD completion (the paper's experiment): 8 workers, n=1000, rank {r}, "
                     "eta 5e-4, lambda 1/5, tau 1",
                     # gradient (+ the combine of the two partial gradients up to rank 32), election, update
-                    launches=(4, 3) if r <= 32 else (3, 2))
+                    launches=(4, 3) if r <= 32 else (3, 2), eagd=bool(getattr(args, "eagd", False)))
     raise SystemExit("unknown workload")
 
 
@@ -274,8 +274,11 @@ def _oracle_sample_once(spec, steps, warmup, sample_cols):
         obj = orc.Mlp(segs, A["pool_x"], A["pool_y"], A["batch_idx"], A["held_x"], A["held_y"], mode="bf16emu")
         what = f"{P} of {spec['P']} workers (one group)"
     mom = spec.get("momentum") if spec["kind"] == "external" else None
-    o = orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau, momentum=mom,
-                       weight_decay=spec.get("weight_decay", 0.0))
+    if spec.get("eagd"):
+        o = orc.EagdOracle(w.x0, obj, w.eta, w.lambda_l, tau=w.tau)
+    else:
+        o = orc.LsgdOracle(w.x0, obj, w.group_of, w.G, w.eta, w.lambda_l, w.lambda_g, w.tau, momentum=mom,
+                           weight_decay=spec.get("weight_decay", 0.0))
     for _ in range(warmup):
         o.step()
     t0 = time.perf_counter()
@@ -419,7 +422,7 @@ def run_ours(args):
                          momentum=args.momentum, weight_decay=args.weight_decay)
     elif spec["kind"] == "psd":
         w = inputs.make_psd(P=P, n=spec["n"], r=spec["r"], steps=steps)
-        pop = Population(w, device=str(dev), arithmetic=args.arith, stream=gstream)
+        pop = Population(w, device=str(dev), arithmetic=args.arith, stream=gstream, eagd=args.eagd)
     else:
         w = inputs.config(spec["cfg"], tau=spec["tau"])
         pop = Population(w, device=str(dev), fused_quadratic=True, arithmetic=args.arith, stream=gstream,
@@ -471,7 +474,7 @@ def run_ours(args):
                 pop._elect(None, False)
                 n_launch += 1 + 2 * (int(loc) + int(glo))
             continue
-        if t % spec["tau"] == 0:
+        if t % spec["tau"] == 0 and not getattr(pop, "eagd", False):
             if spec["kind"] == "mlp":
                 e_ev.append((torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)))
                 e_ev[-1][0].record()
@@ -569,7 +572,7 @@ def run_ours(args):
                    "arithmetic": ["fp64 unfused", "fp64 fma", "fp32 fma"][args.arith],
                    "l2": ("per-step inputs exceed the 126 MB L2; no flush between steps" if P * d * 8 > 3e8 else
                           "working set fits in L2; steps run back to back as in training (no flush)"),
-                   "multi_gpu": "replicas only", "schedule": args.schedule,
+                   "multi_gpu": "replicas only", "schedule": "eagd" if getattr(args, "eagd", False) else args.schedule,
                    **({"momentum": args.momentum, "weight_decay": args.weight_decay} if with_momentum else {}),
                    **({"mlp_fused_step": not args.mlp_unfused_step} if spec["kind"] == "mlp" else {})},
         "clocks": clocks,
@@ -767,6 +770,8 @@ def main():
     ap.add_argument("--momentum", type=float, default=None,
                     help="c4: Nesterov momentum of the Section 4.1 optimiser (adds the buffer v: 20 B per worker-param)")
     ap.add_argument("--weight-decay", type=float, default=0.0)
+    ap.add_argument("--eagd", action="store_true",
+                    help="psd: elastic averaging towards a center variable instead of leaders (the paper's comparison line)")
     ap.add_argument("--sharded", action="store_true",
                     help="groups sharded over the ranks with a leader broadcast per pull step (see run_sharded)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -775,6 +780,8 @@ def main():
     if args.steps <= 0:
         args.steps = 100 if args.impl == "reference" else \
             {"c4": 100, "c0": 4000, "c1": 2000, "c2": 4000, "c3": 1000, "psd": 2000}[args.workload]
+    if args.eagd and args.workload != "psd":
+        raise SystemExit("--eagd times the comparison line of the PSD completion experiment only")
     if args.impl == "reference":
         run_reference(args)
     elif args.sharded:
