@@ -411,8 +411,9 @@ def run_ours(args):
     # ---- inputs: generated on the host from the seed (C4: into pinned memory, also used by the e2e leg)
     hx = hg = None
     if spec["kind"] == "external":
-        hx = torch.empty((P, d), dtype=torch.float32, pin_memory=True)
-        hg = torch.empty((P, d), dtype=torch.float32, pin_memory=True)
+        pin = world == 1                      # pinned only where the end-to-end leg will copy from them
+        hx = torch.empty((P, d), dtype=torch.float32, pin_memory=pin)
+        hg = torch.empty((P, d), dtype=torch.float32, pin_memory=pin)
         w = inputs.make_external(P, G, d, eta=spec["eta"], lambda_l=spec["lambda_l"], lambda_g=spec["lambda_g"],
                                  tau=spec["tau"], steps=steps, config_id=4, x_out=hx.numpy(), g_out=hg.numpy())
         x = hx.to(dev, non_blocking=True)
